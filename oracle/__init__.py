@@ -1,0 +1,161 @@
+"""ctypes front end of the fp64 CPU oracle (``m2rnn_ref.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, the smoke check and the
+bench's CPU-baseline leg, never by the CUDA library's package.  Takes and
+returns numpy float64 arrays in the paper's layouts (Algorithm 1/2 I/O lists):
+q [B,T,Nq,K], k [B,T,Nk,K], v [B,T,N,V], gate [B,T,N], W [N,V,V],
+h0 [B,N,K,V], y [B,T,N,V].
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "m2rnn_ref.c")
+_LIB = os.path.join(_HERE, "libm2rnn_ref.so")
+
+GATE_VALUE, GATE_LOGIT, GATE_PSI = 0, 1, 2
+
+
+def build(force: bool = False, src: str = _SRC, out: str = _LIB) -> str:
+    """Compile the oracle with gcc (IEEE semantics: no -ffast-math)."""
+    hdr = os.path.join(_HERE, "m2rnn_ref.h")
+    stale = (not os.path.exists(out)
+             or os.path.getmtime(out) < max(os.path.getmtime(src), os.path.getmtime(hdr)))
+    if force or stale:
+        tmp = f"{out}.{os.getpid()}.tmp"
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-I", _HERE,
+                               "-o", tmp, src, "-lm"])
+        os.replace(tmp, out)
+    return out
+
+
+class _Params(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int), ("T", ctypes.c_int), ("N", ctypes.c_int),
+                ("Nq", ctypes.c_int), ("Nk", ctypes.c_int), ("K", ctypes.c_int),
+                ("V", ctypes.c_int), ("gate_kind", ctypes.c_int), ("dh_clip", ctypes.c_double)]
+
+
+_dp = ctypes.POINTER(ctypes.c_double)
+
+
+def load(path: str | None = None) -> ctypes.CDLL:
+    lib = ctypes.CDLL(path or build())
+    lib.m2rnn_ref_gate.restype = ctypes.c_double
+    lib.m2rnn_ref_gate.argtypes = [ctypes.c_int, ctypes.c_double, ctypes.c_double,
+                                   ctypes.c_double, _dp]
+    lib.m2rnn_ref_fwd.restype = ctypes.c_int
+    lib.m2rnn_ref_fwd.argtypes = [ctypes.POINTER(_Params)] + [_dp] * 12
+    lib.m2rnn_ref_bwd.restype = ctypes.c_int
+    lib.m2rnn_ref_bwd.argtypes = [ctypes.POINTER(_Params)] + [_dp] * 17
+    lib.m2rnn_ref_decode_step.restype = ctypes.c_int
+    lib.m2rnn_ref_decode_step.argtypes = [ctypes.POINTER(_Params)] + [_dp] * 10
+    return lib
+
+
+_lib = None
+
+
+def _get():
+    global _lib
+    if _lib is None:
+        _lib = load()
+    return _lib
+
+
+def _c(a, shape=None):
+    """float64, C-contiguous copy-if-needed; None stays None."""
+    if a is None:
+        return None
+    a = np.ascontiguousarray(np.asarray(a, dtype=np.float64))
+    if shape is not None and tuple(a.shape) != tuple(shape):
+        raise ValueError(f"expected shape {tuple(shape)}, got {tuple(a.shape)}")
+    return a
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(_dp)
+
+
+def _shapes(q, k, v, W):
+    B, T, Nq, K = q.shape
+    Nk = k.shape[2]
+    N, V = v.shape[2], v.shape[3]
+    assert k.shape == (B, T, Nk, K) and v.shape == (B, T, N, V) and W.shape == (N, V, V)
+    return B, T, N, Nq, Nk, K, V
+
+
+def gate_fn(x, kind=GATE_LOGIT, alpha=1.0, beta=0.0, lib=None):
+    """f and df/dx of one gate entry (scalar)."""
+    d = ctypes.c_double(0.0)
+    f = (lib or _get()).m2rnn_ref_gate(kind, float(x), float(alpha), float(beta), ctypes.byref(d))
+    return f, d.value
+
+
+def fwd(q, k, v, gate, W, h0=None, *, gate_kind=GATE_LOGIT, alpha=None, beta=None, w_r=None,
+        return_states=False, lib=None):
+    """Forward scan -> (y [B,T,N,V], hT [B,N,K,V]) (+ all states [B,N,T+1,K,V])."""
+    lib = lib or _get()
+    q, k, v, W = _c(q), _c(k), _c(v), _c(W)
+    B, T, N, Nq, Nk, K, V = _shapes(q, k, v, W)
+    gate = _c(gate, (B, T, N))
+    h0 = _c(h0, (B, N, K, V)) if h0 is not None else None
+    alpha, beta = _c(alpha, (N,)) if alpha is not None else None, _c(beta, (N,)) if beta is not None else None
+    w_r = _c(w_r, (N, V)) if w_r is not None else None
+    y = np.empty((B, T, N, V), np.float64)
+    hT = np.empty((B, N, K, V), np.float64)
+    H_all = np.empty((B, N, T + 1, K, V), np.float64) if return_states else None
+    p = _Params(B, T, N, Nq, Nk, K, V, gate_kind, 0.0)
+    rc = lib.m2rnn_ref_fwd(ctypes.byref(p), _p(q), _p(k), _p(v), _p(gate), _p(W), _p(h0),
+                           _p(alpha), _p(beta), _p(w_r), _p(y), _p(hT), _p(H_all))
+    if rc != 0:
+        raise RuntimeError(f"m2rnn_ref_fwd failed: {rc}")
+    return (y, hT, H_all) if return_states else (y, hT)
+
+
+def bwd(q, k, v, gate, W, h0, dy, d_hT=None, *, gate_kind=GATE_LOGIT, alpha=None, beta=None,
+        w_r=None, dh_clip=0.0, lib=None):
+    """Backward through time -> dict(dq, dk, dv, dgate, dW, dh0)."""
+    lib = lib or _get()
+    q, k, v, W = _c(q), _c(k), _c(v), _c(W)
+    B, T, N, Nq, Nk, K, V = _shapes(q, k, v, W)
+    gate, dy = _c(gate, (B, T, N)), _c(dy, (B, T, N, V))
+    h0 = _c(h0, (B, N, K, V)) if h0 is not None else None
+    d_hT = _c(d_hT, (B, N, K, V)) if d_hT is not None else None
+    alpha, beta = _c(alpha, (N,)) if alpha is not None else None, _c(beta, (N,)) if beta is not None else None
+    w_r = _c(w_r, (N, V)) if w_r is not None else None
+    out = dict(dq=np.empty((B, T, Nq, K)), dk=np.empty((B, T, Nk, K)), dv=np.empty((B, T, N, V)),
+               dgate=np.empty((B, T, N)), dW=np.empty((N, V, V)), dh0=np.empty((B, N, K, V)))
+    p = _Params(B, T, N, Nq, Nk, K, V, gate_kind, float(dh_clip))
+    rc = lib.m2rnn_ref_bwd(ctypes.byref(p), _p(q), _p(k), _p(v), _p(gate), _p(W), _p(h0),
+                           _p(alpha), _p(beta), _p(w_r), _p(dy), _p(d_hT), _p(out["dq"]),
+                           _p(out["dk"]), _p(out["dv"]), _p(out["dgate"]), _p(out["dW"]),
+                           _p(out["dh0"]))
+    if rc != 0:
+        raise RuntimeError(f"m2rnn_ref_bwd failed: {rc}")
+    return out
+
+
+def decode_step(q, k, v, gate, W, state, *, gate_kind=GATE_LOGIT, alpha=None, beta=None,
+                w_r=None, lib=None):
+    """One step on a cached state -> (y [B,N,V], new state [B,N,K,V]); inputs untouched."""
+    lib = lib or _get()
+    q, k, v, W = _c(q), _c(k), _c(v), _c(W)
+    B, Nq, K = q.shape
+    Nk, (N, V) = k.shape[1], v.shape[1:]
+    gate = _c(gate, (B, N))
+    state = np.array(state, dtype=np.float64, order="C", copy=True)
+    assert state.shape == (B, N, K, V)
+    alpha, beta = _c(alpha, (N,)) if alpha is not None else None, _c(beta, (N,)) if beta is not None else None
+    w_r = _c(w_r, (N, V)) if w_r is not None else None
+    y = np.empty((B, N, V), np.float64)
+    p = _Params(B, 1, N, Nq, Nk, K, V, gate_kind, 0.0)
+    rc = lib.m2rnn_ref_decode_step(ctypes.byref(p), _p(q), _p(k), _p(v), _p(gate), _p(W),
+                                   _p(alpha), _p(beta), _p(w_r), _p(state), _p(y))
+    if rc != 0:
+        raise RuntimeError(f"m2rnn_ref_decode_step failed: {rc}")
+    return y, state
