@@ -1,0 +1,136 @@
+/*
+ * m2rnn.h -- C ABI of the B200 (sm_100a) M2RNN recurrent-scan library.
+ *
+ * The library computes the sequential part of one M2RNN layer, per (batch b, head n)
+ * on a K x V matrix state H (paper, Eq. 1-3 of the M2RNN layer):
+ *
+ *     Z_t = tanh(H_{t-1} W_n + k_t v_t^T)
+ *     H_t = f_t H_{t-1} + (1 - f_t) Z_t
+ *     y_t = H_t^T q_t  (+ w_r (.) v_t)
+ *
+ * forward (Algorithm 1), backward through time (Algorithm 2) and one decoding step.
+ *
+ * Conventions for every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller, contiguous in the
+ *     stated layout and 16-byte aligned.  `params` is a HOST pointer.
+ *   - Layouts are the paper's (Algorithm 1/2 I/O lists): token-major, heads interleaved.
+ *       q [B,T,Nq,K]  k [B,T,Nk,K]  v [B,T,N,V]  gate [B,T,N]  W [N,V,V]
+ *       h0,hT [B,N,K,V]  y,dy [B,T,N,V]  alpha,beta [N]  w_r [N,V]
+ *     Head n reads q-head n/(N/Nq) and k-head n/(N/Nk) (contiguous groups);
+ *     Nq = Nk = 1 is the paper's multi-value layout, Nq = Nk = N plain multi-head.
+ *   - q,k,v,W,w_r,y,dy,dq,dk,dv have the element type `io_dtype`; gate, alpha, beta,
+ *     every state (h0,hT,ckpt,d_hT,dh0,decode state), dgate and dW are fp32.
+ *     With M2RNN_BF16 the state x W product runs on tensor cores (bf16 operands, fp32
+ *     accumulate) and the state itself stays fp32; with M2RNN_F32 everything is fp32 FMA.
+ *   - The library allocates nothing and keeps nothing between calls.  Outputs are
+ *     overwritten, never accumulated into.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = the
+ *     default stream) and never synchronise.  The return value is an m2rnn_status:
+ *     argument errors are reported before anything is launched, launch errors right
+ *     after; nothing is launched when an error is returned.
+ *   - `dev_status` (device int32, may be NULL): every wait inside a kernel is bounded;
+ *     if one runs out the kernel stores M2RNN_ERR_TIMEOUT there and returns early.
+ *     The caller zeroes it and reads it back after synchronising.
+ *   - Supported sizes: K a multiple of 16 in 16..128, V in {16,32,64,128}, B,T,N >= 1
+ *     (T = 0 or B = 0 is a valid empty call: nothing is launched, hT = h0 is NOT written).
+ */
+#ifndef M2RNN_H
+#define M2RNN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  M2RNN_OK = 0,
+  M2RNN_ERR_NULL = -1,        /* a required pointer is NULL                         */
+  M2RNN_ERR_SHAPE = -2,       /* a size is non-positive or a head count does not divide N */
+  M2RNN_ERR_UNSUPPORTED = -3, /* K, V, dtype, gate kind or ckpt_interval outside the supported set */
+  M2RNN_ERR_ALIGN = -4,       /* a pointer is not 16-byte aligned                   */
+  M2RNN_ERR_WORKSPACE = -5,   /* workspace missing or smaller than m2rnn_bwd_workspace_bytes */
+  M2RNN_ERR_CUDA = -6,        /* the CUDA runtime refused a launch or attribute     */
+  M2RNN_ERR_TIMEOUT = -7      /* device-side only: a bounded wait ran out           */
+} m2rnn_status;
+
+typedef enum { M2RNN_F32 = 0, M2RNN_BF16 = 1 } m2rnn_dtype;
+
+typedef enum {
+  M2RNN_GATE_VALUE = 0, /* gate tensor IS f_t in [0,1]                 (Algorithm 1, input F)    */
+  M2RNN_GATE_LOGIT = 1, /* f_t = 1/(1+exp(-gate))                      (forget-gate eq., alpha=1, beta=0, x=-gate) */
+  M2RNN_GATE_PSI = 2    /* f_t = (1+exp(gate+beta_n))^(-alpha_n)       (forget-gate equation)    */
+} m2rnn_gate_kind;
+
+typedef struct {
+  int32_t B, T, N;       /* batch, steps, value heads (N = N_v = N_f = N_w)                   */
+  int32_t Nq, Nk;        /* query / key heads: 1..N, each divides N                           */
+  int32_t K, V;          /* state is K x V per (b,n); the transition matrix is V x V          */
+  int32_t io_dtype;      /* m2rnn_dtype                                                       */
+  int32_t gate_kind;     /* m2rnn_gate_kind                                                   */
+  int32_t ckpt_interval; /* steps between saved states; 0 = library default for (K,V,dtype)  */
+  float dh_clip;         /* <= 0: off.  Else the state gradient carried to the previous step is
+                            clamped elementwise to [-dh_clip, dh_clip] after every reverse step
+                            (section "Gradient Clipping"; the paper gives no threshold or form) */
+} m2rnn_params;
+
+/* Library version: major*10000 + minor*100 + patch. */
+int m2rnn_version(void);
+
+/* Static text for a status code. */
+const char *m2rnn_status_string(int status);
+
+/* The checkpoint interval C the library will use for `params` (params->ckpt_interval if it is
+ * non-zero and supported, else the default); <= 0 is an m2rnn_status.  The backward kernel
+ * recomputes C states at a time from a checkpoint, so C is bounded by on-chip memory. */
+int m2rnn_ckpt_interval(const m2rnn_params *params);
+
+/* Bytes of the checkpoint tensor [B,N,ceil(T/C),K,V] (fp32). */
+size_t m2rnn_ckpt_bytes(const m2rnn_params *params);
+
+/* Forward scan (Algorithm 1; Eq. 1-3).
+ *   in : q,k,v,gate,W; h0 or NULL (= zero state); alpha,beta (GATE_PSI only, else ignored,
+ *        may be NULL); w_r or NULL (residual term of Eq. 3 omitted, as in Algorithm 1)
+ *   out: y [B,T,N,V]; hT or NULL: final state H_T (fp32);
+ *        ckpt or NULL: ckpt[b,n,c] = H_{c*C}, the state BEFORE step c*C (so ckpt[..,0] = h0),
+ *        for m2rnn_bwd. */
+int m2rnn_fwd(const m2rnn_params *params, const void *q, const void *k, const void *v,
+              const float *gate, const void *W, const float *h0, const float *alpha,
+              const float *beta, const void *w_r, void *y, float *hT, float *ckpt,
+              int32_t *dev_status, void *stream);
+
+/* Scratch the backward call needs for `params`; `have_ckpt` != 0 if the caller will pass the
+ * checkpoints written by m2rnn_fwd (otherwise the workspace also holds them). */
+size_t m2rnn_bwd_workspace_bytes(const m2rnn_params *params, int have_ckpt);
+
+/* Backward through time (Algorithm 2, with the state gradient carried across steps:
+ * G_t = C_t + q_t dy_t^T, C_{t-1} = f_t G_t + dX_t W^T, dX_t = (1-f_t) G_t (.) (1 - Z_t (.) Z_t)).
+ *   in : the forward inputs; ckpt from m2rnn_fwd with the same params, or NULL (recomputed here);
+ *        dy [B,T,N,V]; d_hT or NULL: gradient w.r.t. the final state (seed of C_T)
+ *   out: dq [B,T,Nq,K], dk [B,T,Nk,K] (summed over the heads sharing them), dv [B,T,N,V],
+ *        dgate [B,T,N] (w.r.t. the gate tensor as passed, i.e. through the gate function),
+ *        dW [N,V,V] fp32 (summed over batch, fixed order: results repeat bit for bit),
+ *        dh0 or NULL [B,N,K,V] fp32.
+ *   workspace: device scratch of at least m2rnn_bwd_workspace_bytes(params, ckpt != NULL),
+ *        256-byte aligned; contents undefined afterwards.
+ * w_r's own gradient (sum over b,t of v (.) dy) is an elementwise reduction outside the scan. */
+int m2rnn_bwd(const m2rnn_params *params, const void *q, const void *k, const void *v,
+              const float *gate, const void *W, const float *h0, const float *alpha,
+              const float *beta, const void *w_r, const float *ckpt, const void *dy,
+              const float *d_hT, void *dq, void *dk, void *dv, float *dgate, float *dW,
+              float *dh0, void *workspace, size_t workspace_bytes, int32_t *dev_status,
+              void *stream);
+
+/* One decoding step on a cached state (Eq. 1-3 once; params->T is ignored).
+ *   in : q [B,Nq,K], k [B,Nk,K], v [B,N,V], gate [B,N], W, alpha/beta/w_r as in m2rnn_fwd
+ *   io : state [B,N,K,V] fp32, updated in place
+ *   out: y [B,N,V] */
+int m2rnn_decode_step(const m2rnn_params *params, const void *q, const void *k, const void *v,
+                      const float *gate, const void *W, const float *alpha, const float *beta,
+                      const void *w_r, float *state, void *y, int32_t *dev_status, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* M2RNN_H */

@@ -1,0 +1,235 @@
+"""Thin ctypes binding of ``libm2rnn.so`` (declared in ``include/m2rnn.h``).
+
+Argument marshalling only: every step of the scan runs in the library's CUDA kernels.
+torch supplies device memory and the current stream; there is no CPU or eager fallback --
+a missing or stale library raises.
+
+    y, hT, ckpt = m2rnn_fwd(q, k, v, gate, W, h0, save_ckpt=True)
+    grads       = m2rnn_bwd(q, k, v, gate, W, h0, dy, ckpt=ckpt)
+    y1          = m2rnn_decode_step(q1, k1, v1, gate1, W, state)      # state updated in place
+
+Tensor layouts are the paper's (Algorithm 1/2): q [B,T,Nq,K], k [B,T,Nk,K], v [B,T,N,V],
+gate [B,T,N] fp32, W [N,V,V], h0 [B,N,K,V] fp32.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+GATE_VALUE, GATE_LOGIT, GATE_PSI = 0, 1, 2
+F32, BF16 = 0, 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libm2rnn.so")
+
+STATUS = {0: "M2RNN_OK", -1: "M2RNN_ERR_NULL", -2: "M2RNN_ERR_SHAPE", -3: "M2RNN_ERR_UNSUPPORTED",
+          -4: "M2RNN_ERR_ALIGN", -5: "M2RNN_ERR_WORKSPACE", -6: "M2RNN_ERR_CUDA", -7: "M2RNN_ERR_TIMEOUT"}
+
+
+class M2RNNError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = _lib().m2rnn_status_string(status).decode() if _LIB is not None else ""
+        super().__init__(f"{where}: {STATUS.get(status, status)} ({msg})")
+
+
+class Params(ctypes.Structure):
+    """Mirror of ``m2rnn_params``."""
+    _fields_ = [("B", ctypes.c_int32), ("T", ctypes.c_int32), ("N", ctypes.c_int32),
+                ("Nq", ctypes.c_int32), ("Nk", ctypes.c_int32), ("K", ctypes.c_int32),
+                ("V", ctypes.c_int32), ("io_dtype", ctypes.c_int32), ("gate_kind", ctypes.c_int32),
+                ("ckpt_interval", ctypes.c_int32), ("dh_clip", ctypes.c_float)]
+
+
+_LIB = None
+_vp = ctypes.c_void_p
+_pp = ctypes.POINTER(Params)
+
+EXPORTS = {
+    "m2rnn_version": (ctypes.c_int, []),
+    "m2rnn_status_string": (ctypes.c_char_p, [ctypes.c_int]),
+    "m2rnn_ckpt_interval": (ctypes.c_int, [_pp]),
+    "m2rnn_ckpt_bytes": (ctypes.c_size_t, [_pp]),
+    "m2rnn_fwd": (ctypes.c_int, [_pp] + [_vp] * 14),
+    "m2rnn_bwd_workspace_bytes": (ctypes.c_size_t, [_pp, ctypes.c_int]),
+    "m2rnn_bwd": (ctypes.c_int, [_pp] + [_vp] * 19 + [ctypes.c_size_t, _vp, _vp]),
+    "m2rnn_decode_step": (ctypes.c_int, [_pp] + [_vp] * 12),
+}
+
+
+def _lib() -> ctypes.CDLL:
+    global _LIB
+    if _LIB is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is not built: run `python -m paper_2603_14360_b200.build` "
+                              "(there is no fallback path)")
+        lib = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in EXPORTS.items():
+            fn = getattr(lib, name)          # AttributeError if the library is stale
+            fn.restype, fn.argtypes = res, args
+        _LIB = lib
+    return _LIB
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _io_code(dtype: torch.dtype) -> int:
+    if dtype == torch.float32:
+        return F32
+    if dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported I/O dtype {dtype}")
+
+
+def _chk(t, name, shape, dtype):
+    if t is None:
+        return
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    if tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name}: expected shape {tuple(shape)}, got {tuple(t.shape)}")
+    if t.dtype != dtype:
+        raise TypeError(f"{name}: expected {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+
+
+_status_words: dict[int, torch.Tensor] = {}
+
+
+def device_status_word(device=None) -> torch.Tensor:
+    """The int32 word kernels raise when a bounded wait runs out (one per device, zero = fine)."""
+    idx = torch.cuda.current_device() if device is None else torch.device(device).index
+    if idx not in _status_words:
+        _status_words[idx] = torch.zeros(1, dtype=torch.int32, device=f"cuda:{idx}")
+    return _status_words[idx]
+
+
+def check_device_status(device=None) -> None:
+    """Synchronises and raises if any kernel since the last check reported a timeout."""
+    w = device_status_word(device)
+    v = int(w.item())
+    if v != 0:
+        w.zero_()
+        raise M2RNNError(v, "device status")
+
+
+def _params(q, k, v, W, gate_kind, ckpt_interval=0, dh_clip=0.0, decode=False) -> Params:
+    if decode:
+        B, Nq, K = q.shape
+        T, Nk, (N, V) = 1, k.shape[1], v.shape[1:]
+    else:
+        B, T, Nq, K = q.shape
+        Nk, (N, V) = k.shape[2], v.shape[2:]
+    return Params(B, T, N, Nq, Nk, K, V, _io_code(q.dtype), gate_kind, ckpt_interval, dh_clip)
+
+
+def m2rnn_version() -> int:
+    return _lib().m2rnn_version()
+
+
+def m2rnn_ckpt_interval(p: Params) -> int:
+    c = _lib().m2rnn_ckpt_interval(ctypes.byref(p))
+    if c <= 0:
+        raise M2RNNError(c, "m2rnn_ckpt_interval")
+    return c
+
+
+def m2rnn_bwd_workspace_bytes(p: Params, have_ckpt: bool) -> int:
+    return _lib().m2rnn_bwd_workspace_bytes(ctypes.byref(p), int(have_ckpt))
+
+
+def m2rnn_fwd(q, k, v, gate, W, h0=None, *, gate_kind=GATE_LOGIT, alpha=None, beta=None, w_r=None,
+              save_ckpt=False, ckpt_interval=0, want_hT=True, out=None, stream=None):
+    """Forward scan.  Returns (y, hT, ckpt); hT / ckpt are None when not requested.
+    ``out`` may hold preallocated ``y`` / ``hT`` / ``ckpt`` tensors to write into."""
+    p = _params(q, k, v, W, gate_kind, ckpt_interval)
+    B, T, N, K, V, io = p.B, p.T, p.N, p.K, p.V, q.dtype
+    _chk(q, "q", (B, T, p.Nq, K), io); _chk(k, "k", (B, T, p.Nk, K), io); _chk(v, "v", (B, T, N, V), io)
+    _chk(gate, "gate", (B, T, N), torch.float32); _chk(W, "W", (N, V, V), io)
+    _chk(h0, "h0", (B, N, K, V), torch.float32); _chk(w_r, "w_r", (N, V), io)
+    _chk(alpha, "alpha", (N,), torch.float32); _chk(beta, "beta", (N,), torch.float32)
+    out = out or {}
+    y = out.get("y")
+    if y is None:
+        y = torch.empty((B, T, N, V), dtype=io, device=q.device)
+    hT = out.get("hT")
+    if hT is None and want_hT:
+        hT = torch.empty((B, N, K, V), dtype=torch.float32, device=q.device)
+    ckpt = out.get("ckpt")
+    if ckpt is None and save_ckpt:
+        C = m2rnn_ckpt_interval(p)
+        ckpt = torch.empty((B, N, (T + C - 1) // C, K, V), dtype=torch.float32, device=q.device)
+    _chk(y, "y", (B, T, N, V), io); _chk(hT, "hT", (B, N, K, V), torch.float32)
+    rc = _lib().m2rnn_fwd(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(gate), _ptr(W), _ptr(h0),
+                          _ptr(alpha), _ptr(beta), _ptr(w_r), _ptr(y), _ptr(hT), _ptr(ckpt),
+                          _ptr(device_status_word(q.device)), _stream(stream))
+    if rc != 0:
+        raise M2RNNError(rc, "m2rnn_fwd")
+    return y, hT, ckpt
+
+
+def m2rnn_bwd(q, k, v, gate, W, h0, dy, d_hT=None, *, ckpt=None, gate_kind=GATE_LOGIT, alpha=None,
+              beta=None, w_r=None, ckpt_interval=0, dh_clip=0.0, want_dh0=True, workspace=None,
+              out=None, stream=None):
+    """Backward through time.  Returns dict(dq, dk, dv, dgate, dW, dh0)."""
+    p = _params(q, k, v, W, gate_kind, ckpt_interval, dh_clip)
+    B, T, N, K, V, io = p.B, p.T, p.N, p.K, p.V, q.dtype
+    _chk(q, "q", (B, T, p.Nq, K), io); _chk(k, "k", (B, T, p.Nk, K), io); _chk(v, "v", (B, T, N, V), io)
+    _chk(gate, "gate", (B, T, N), torch.float32); _chk(W, "W", (N, V, V), io)
+    _chk(h0, "h0", (B, N, K, V), torch.float32); _chk(w_r, "w_r", (N, V), io)
+    _chk(alpha, "alpha", (N,), torch.float32); _chk(beta, "beta", (N,), torch.float32)
+    _chk(dy, "dy", (B, T, N, V), io); _chk(d_hT, "d_hT", (B, N, K, V), torch.float32)
+    if ckpt is not None and T > 0:
+        C = m2rnn_ckpt_interval(p)
+        _chk(ckpt, "ckpt", (B, N, (T + C - 1) // C, K, V), torch.float32)
+    dev = q.device
+    out = out or {}
+    g = dict(dq=out.get("dq"), dk=out.get("dk"), dv=out.get("dv"), dgate=out.get("dgate"),
+             dW=out.get("dW"), dh0=out.get("dh0"))
+    if g["dq"] is None: g["dq"] = torch.empty_like(q)
+    if g["dk"] is None: g["dk"] = torch.empty_like(k)
+    if g["dv"] is None: g["dv"] = torch.empty_like(v)
+    if g["dgate"] is None: g["dgate"] = torch.empty_like(gate)
+    if g["dW"] is None: g["dW"] = torch.empty((N, V, V), dtype=torch.float32, device=dev)
+    if g["dh0"] is None and want_dh0: g["dh0"] = torch.empty((B, N, K, V), dtype=torch.float32, device=dev)
+    need = m2rnn_bwd_workspace_bytes(p, ckpt is not None)
+    if workspace is None:
+        workspace = torch.empty(max(need, 1), dtype=torch.uint8, device=dev)
+    rc = _lib().m2rnn_bwd(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(gate), _ptr(W), _ptr(h0),
+                          _ptr(alpha), _ptr(beta), _ptr(w_r), _ptr(ckpt), _ptr(dy), _ptr(d_hT),
+                          _ptr(g["dq"]), _ptr(g["dk"]), _ptr(g["dv"]), _ptr(g["dgate"]), _ptr(g["dW"]),
+                          _ptr(g["dh0"]), _ptr(workspace), workspace.numel(),
+                          _ptr(device_status_word(dev)), _stream(stream))
+    if rc != 0:
+        raise M2RNNError(rc, "m2rnn_bwd")
+    return g
+
+
+def m2rnn_decode_step(q, k, v, gate, W, state, *, gate_kind=GATE_LOGIT, alpha=None, beta=None,
+                      w_r=None, y=None, stream=None):
+    """One decoding step; ``state`` [B,N,K,V] fp32 is updated in place.  Returns y [B,N,V]."""
+    p = _params(q, k, v, W, gate_kind, decode=True)
+    B, N, K, V, io = p.B, p.N, p.K, p.V, q.dtype
+    _chk(q, "q", (B, p.Nq, K), io); _chk(k, "k", (B, p.Nk, K), io); _chk(v, "v", (B, N, V), io)
+    _chk(gate, "gate", (B, N), torch.float32); _chk(W, "W", (N, V, V), io)
+    _chk(state, "state", (B, N, K, V), torch.float32); _chk(w_r, "w_r", (N, V), io)
+    _chk(alpha, "alpha", (N,), torch.float32); _chk(beta, "beta", (N,), torch.float32)
+    if y is None:
+        y = torch.empty((B, N, V), dtype=io, device=q.device)
+    _chk(y, "y", (B, N, V), io)
+    rc = _lib().m2rnn_decode_step(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(gate), _ptr(W),
+                                  _ptr(alpha), _ptr(beta), _ptr(w_r), _ptr(state), _ptr(y),
+                                  _ptr(device_status_word(q.device)), _stream(stream))
+    if rc != 0:
+        raise M2RNNError(rc, "m2rnn_decode_step")
+    return y

@@ -1,0 +1,235 @@
+// C ABI of the M2RNN scan library: argument checks, workspace layout, dispatch.
+// No allocation, no synchronisation, no state kept between calls.
+#include <cuda_runtime.h>
+
+#include "internal.h"
+#include "m2rnn.h"
+
+namespace m2rnn {
+
+int max_ckpt_interval(int K, int V, int io_dtype) {
+  if (io_dtype == M2RNN_F32) return 64;  // recomputed states live in global scratch
+  // bf16: one chunk of recomputed states (bf16, K*V*2 bytes per step) stays in shared memory
+  const int per_step = K * V * 2;
+  int c = (128 * 1024) / per_step;
+  return c < 1 ? 1 : (c > 64 ? 64 : c);
+}
+
+int default_ckpt_interval(int K, int V, int io_dtype) {
+  if (io_dtype == M2RNN_F32) return 16;
+  int c = max_ckpt_interval(K, V, io_dtype);
+  return c > 16 ? 16 : c;
+}
+
+namespace {
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_params(const m2rnn_params *p, bool need_T) {
+  if (!p) return M2RNN_ERR_NULL;
+  if (p->B < 0 || p->N <= 0 || p->K <= 0 || p->V <= 0 || (need_T && p->T < 0)) return M2RNN_ERR_SHAPE;
+  if (p->Nq <= 0 || p->Nk <= 0 || p->Nq > p->N || p->Nk > p->N || p->N % p->Nq || p->N % p->Nk)
+    return M2RNN_ERR_SHAPE;
+  if (p->io_dtype != M2RNN_F32 && p->io_dtype != M2RNN_BF16) return M2RNN_ERR_UNSUPPORTED;
+  if (p->gate_kind < M2RNN_GATE_VALUE || p->gate_kind > M2RNN_GATE_PSI) return M2RNN_ERR_UNSUPPORTED;
+  if (p->K % 16 || p->K < 16 || p->K > 128) return M2RNN_ERR_UNSUPPORTED;
+  if (p->V != 16 && p->V != 32 && p->V != 64 && p->V != 128) return M2RNN_ERR_UNSUPPORTED;
+  if (p->ckpt_interval < 0 || p->ckpt_interval > max_ckpt_interval(p->K, p->V, p->io_dtype))
+    return M2RNN_ERR_UNSUPPORTED;
+  return M2RNN_OK;
+}
+
+int interval_of(const m2rnn_params *p) {
+  return p->ckpt_interval ? p->ckpt_interval : default_ckpt_interval(p->K, p->V, p->io_dtype);
+}
+
+struct Workspace {
+  size_t ckpt, dW_part, dq_part, dk_part, chunk_states, total;
+};
+
+Workspace layout(const m2rnn_params *p, bool have_ckpt) {
+  Workspace w{};
+  const int C = interval_of(p);
+  const size_t nch = p->T > 0 ? (size_t)(p->T + C - 1) / C : 0;
+  const size_t BN = (size_t)p->B * p->N, KV = (size_t)p->K * p->V;
+  size_t off = 0;
+  w.ckpt = off;
+  if (!have_ckpt) off += align_up(BN * nch * KV * sizeof(float));
+  w.dW_part = off;
+  off += align_up(BN * p->V * p->V * sizeof(float));
+  w.dq_part = off;
+  if (p->Nq < p->N) off += align_up((size_t)p->B * p->T * p->N * p->K * sizeof(float));
+  w.dk_part = off;
+  if (p->Nk < p->N) off += align_up((size_t)p->B * p->T * p->N * p->K * sizeof(float));
+  w.chunk_states = off;
+  if (p->io_dtype == M2RNN_F32) off += align_up(BN * C * KV * sizeof(float));
+  w.total = off;
+  return w;
+}
+
+ScanArgs base_args(const m2rnn_params *p) {
+  ScanArgs a{};
+  a.B = p->B; a.T = p->T; a.N = p->N; a.Nq = p->Nq; a.Nk = p->Nk; a.K = p->K; a.V = p->V;
+  a.gate_kind = p->gate_kind;
+  a.C = interval_of(p);
+  a.nchunks = p->T > 0 ? (p->T + a.C - 1) / a.C : 0;
+  a.dh_clip = p->dh_clip;
+  return a;
+}
+
+}  // namespace
+}  // namespace m2rnn
+
+using namespace m2rnn;
+
+extern "C" {
+
+int m2rnn_version(void) { return 100; }
+
+const char *m2rnn_status_string(int status) {
+  switch (status) {
+    case M2RNN_OK: return "ok";
+    case M2RNN_ERR_NULL: return "a required pointer is NULL";
+    case M2RNN_ERR_SHAPE: return "bad size: non-positive, or a head count that does not divide N";
+    case M2RNN_ERR_UNSUPPORTED: return "unsupported K, V, dtype, gate kind or checkpoint interval";
+    case M2RNN_ERR_ALIGN: return "a pointer is not 16-byte aligned (workspace: 256-byte)";
+    case M2RNN_ERR_WORKSPACE: return "workspace missing or too small";
+    case M2RNN_ERR_CUDA: return "the CUDA runtime refused the launch";
+    case M2RNN_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    default: return "unknown status";
+  }
+}
+
+int m2rnn_ckpt_interval(const m2rnn_params *params) {
+  int rc = check_params(params, false);
+  if (rc != M2RNN_OK) return rc;
+  return interval_of(params);
+}
+
+size_t m2rnn_ckpt_bytes(const m2rnn_params *params) {
+  if (check_params(params, true) != M2RNN_OK || params->T == 0) return 0;
+  const int C = interval_of(params);
+  return (size_t)params->B * params->N * ((params->T + C - 1) / C) * params->K * params->V * sizeof(float);
+}
+
+int m2rnn_fwd(const m2rnn_params *params, const void *q, const void *k, const void *v,
+              const float *gate, const void *W, const float *h0, const float *alpha,
+              const float *beta, const void *w_r, void *y, float *hT, float *ckpt,
+              int32_t *dev_status, void *stream) {
+  int rc = check_params(params, true);
+  if (rc != M2RNN_OK) return rc;
+  if (params->B == 0 || params->T == 0) return M2RNN_OK;
+  if (!q || !k || !v || !gate || !W || !y) return M2RNN_ERR_NULL;
+  if (params->gate_kind == M2RNN_GATE_PSI && (!alpha || !beta)) return M2RNN_ERR_NULL;
+  const void *ptrs[] = {q, k, v, gate, W, h0, w_r, y, hT, ckpt};
+  for (const void *p : ptrs)
+    if (!aligned16(p)) return M2RNN_ERR_ALIGN;
+  ScanArgs a = base_args(params);
+  a.q = q; a.k = k; a.v = v; a.gate = gate; a.W = W; a.h0 = h0; a.w_r = w_r;
+  a.alpha = params->gate_kind == M2RNN_GATE_PSI ? alpha : nullptr;
+  a.beta = params->gate_kind == M2RNN_GATE_PSI ? beta : nullptr;
+  a.y = y; a.hT = hT; a.ckpt = ckpt; a.dev_status = dev_status;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = params->io_dtype == M2RNN_F32 ? launch_fwd_f32(a, s) : launch_fwd_bf16(a, s);
+  return e == cudaSuccess ? M2RNN_OK : M2RNN_ERR_CUDA;
+}
+
+size_t m2rnn_bwd_workspace_bytes(const m2rnn_params *params, int have_ckpt) {
+  if (check_params(params, true) != M2RNN_OK) return 0;
+  return layout(params, have_ckpt != 0).total;
+}
+
+int m2rnn_bwd(const m2rnn_params *params, const void *q, const void *k, const void *v,
+              const float *gate, const void *W, const float *h0, const float *alpha,
+              const float *beta, const void *w_r, const float *ckpt, const void *dy,
+              const float *d_hT, void *dq, void *dk, void *dv, float *dgate, float *dW,
+              float *dh0, void *workspace, size_t workspace_bytes, int32_t *dev_status,
+              void *stream) {
+  int rc = check_params(params, true);
+  if (rc != M2RNN_OK) return rc;
+  if (!dW) return M2RNN_ERR_NULL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (params->B == 0 || params->T == 0) {
+    // empty scan: the only defined outputs are dW = 0 and dh0 = d_hT (or 0)
+    if (!aligned16(dW) || !aligned16(dh0) || !aligned16(d_hT)) return M2RNN_ERR_ALIGN;
+    cudaError_t e = cudaMemsetAsync(dW, 0, sizeof(float) * params->N * params->V * params->V, s);
+    if (e == cudaSuccess && dh0 && params->B > 0) {
+      const size_t bytes = sizeof(float) * (size_t)params->B * params->N * params->K * params->V;
+      e = d_hT ? cudaMemcpyAsync(dh0, d_hT, bytes, cudaMemcpyDeviceToDevice, s) : cudaMemsetAsync(dh0, 0, bytes, s);
+    }
+    return e == cudaSuccess ? M2RNN_OK : M2RNN_ERR_CUDA;
+  }
+  if (!q || !k || !v || !gate || !W || !dy || !dq || !dk || !dv || !dgate) return M2RNN_ERR_NULL;
+  if (params->gate_kind == M2RNN_GATE_PSI && (!alpha || !beta)) return M2RNN_ERR_NULL;
+  const void *ptrs[] = {q, k, v, gate, W, h0, w_r, ckpt, dy, d_hT, dq, dk, dv, dgate, dW, dh0};
+  for (const void *p : ptrs)
+    if (!aligned16(p)) return M2RNN_ERR_ALIGN;
+  const Workspace w = layout(params, ckpt != nullptr);
+  if (w.total > 0 && (!workspace || workspace_bytes < w.total)) return M2RNN_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return M2RNN_ERR_ALIGN;
+  char *ws = static_cast<char *>(workspace);
+
+  ScanArgs a = base_args(params);
+  a.q = q; a.k = k; a.v = v; a.gate = gate; a.W = W; a.h0 = h0; a.w_r = w_r;
+  a.alpha = params->gate_kind == M2RNN_GATE_PSI ? alpha : nullptr;
+  a.beta = params->gate_kind == M2RNN_GATE_PSI ? beta : nullptr;
+  a.dev_status = dev_status;
+  const bool f32 = params->io_dtype == M2RNN_F32;
+  cudaError_t e = cudaSuccess;
+  if (!ckpt) {
+    // pass 1 of Algorithm 2, thinned: save the state every C steps only
+    ScanArgs f = a;
+    f.y = nullptr; f.hT = nullptr;
+    f.ckpt = reinterpret_cast<float *>(ws + w.ckpt);
+    e = f32 ? launch_fwd_f32(f, s) : launch_fwd_bf16(f, s);
+    if (e != cudaSuccess) return M2RNN_ERR_CUDA;
+    a.ckpt = f.ckpt;
+  } else {
+    a.ckpt = const_cast<float *>(ckpt);
+  }
+  a.dy = dy; a.d_hT = d_hT; a.dq = dq; a.dk = dk; a.dv = dv; a.dgate = dgate; a.dh0 = dh0;
+  a.dW_part = reinterpret_cast<float *>(ws + w.dW_part);
+  a.dq_part = params->Nq < params->N ? reinterpret_cast<float *>(ws + w.dq_part) : nullptr;
+  a.dk_part = params->Nk < params->N ? reinterpret_cast<float *>(ws + w.dk_part) : nullptr;
+  a.chunk_states = f32 ? reinterpret_cast<float *>(ws + w.chunk_states) : nullptr;
+  e = f32 ? launch_bwd_f32(a, s) : launch_bwd_bf16(a, s);
+  if (e != cudaSuccess) return M2RNN_ERR_CUDA;
+  e = launch_reduce_dW(a.dW_part, dW, params->B, params->N, params->V, s);
+  if (e != cudaSuccess) return M2RNN_ERR_CUDA;
+  const size_t BT = (size_t)params->B * params->T;
+  if (a.dq_part) {
+    e = launch_reduce_heads(a.dq_part, dq, params->io_dtype, BT, params->N, params->Nq, params->K, s);
+    if (e != cudaSuccess) return M2RNN_ERR_CUDA;
+  }
+  if (a.dk_part) {
+    e = launch_reduce_heads(a.dk_part, dk, params->io_dtype, BT, params->N, params->Nk, params->K, s);
+    if (e != cudaSuccess) return M2RNN_ERR_CUDA;
+  }
+  return M2RNN_OK;
+}
+
+int m2rnn_decode_step(const m2rnn_params *params, const void *q, const void *k, const void *v,
+                      const float *gate, const void *W, const float *alpha, const float *beta,
+                      const void *w_r, float *state, void *y, int32_t *dev_status, void *stream) {
+  int rc = check_params(params, false);
+  if (rc != M2RNN_OK) return rc;
+  if (params->B == 0) return M2RNN_OK;
+  if (!q || !k || !v || !gate || !W || !state || !y) return M2RNN_ERR_NULL;
+  if (params->gate_kind == M2RNN_GATE_PSI && (!alpha || !beta)) return M2RNN_ERR_NULL;
+  const void *ptrs[] = {q, k, v, gate, W, w_r, state, y};
+  for (const void *p : ptrs)
+    if (!aligned16(p)) return M2RNN_ERR_ALIGN;
+  ScanArgs a = base_args(params);
+  a.T = 1; a.nchunks = 1;
+  a.q = q; a.k = k; a.v = v; a.gate = gate; a.W = W; a.w_r = w_r;
+  a.alpha = params->gate_kind == M2RNN_GATE_PSI ? alpha : nullptr;
+  a.beta = params->gate_kind == M2RNN_GATE_PSI ? beta : nullptr;
+  a.h0 = state; a.hT = state; a.y = y; a.ckpt = nullptr; a.dev_status = dev_status;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // one step of Eq. 1-3: a T=1 scan whose initial and final state share storage (each CTA reads
+  // its own slice of the state completely before it writes it back)
+  cudaError_t e = params->io_dtype == M2RNN_F32 ? launch_fwd_f32(a, s) : launch_decode_bf16(a, s);
+  return e == cudaSuccess ? M2RNN_OK : M2RNN_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,59 @@
+// Internal declarations shared by the host API and the kernel translation units.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "m2rnn.h"
+
+namespace m2rnn {
+
+// Everything a kernel needs, by value.  Pointers are device pointers.
+struct ScanArgs {
+  int B, T, N, Nq, Nk, K, V;
+  int gate_kind;
+  int C;          // checkpoint interval (steps)
+  int nchunks;    // ceil(T / C)
+  float dh_clip;
+  const void *q, *k, *v, *W, *w_r;
+  const float *gate, *h0, *alpha, *beta;
+  void *y;
+  float *hT;
+  float *ckpt;    // fwd: written (may be null); bwd: read
+  // backward only
+  const void *dy;
+  const float *d_hT;
+  void *dq, *dk, *dv;  // dq/dk: final tensors when the head is not shared, else see dq_part
+  float *dgate, *dh0;
+  float *dW_part;      // [B,N,V,V] per-(b,n) partial sums of dW
+  float *dq_part;      // [B,T,N,K] fp32 per-head dq when Nq < N, else null
+  float *dk_part;      // [B,T,N,K] fp32 per-head dk when Nk < N, else null
+  float *chunk_states; // fp32 path: [B*N, C, K, V] scratch for the recomputed states
+  int32_t *dev_status;
+};
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+// Default / maximum checkpoint interval for a problem (bounded by shared memory in the
+// bf16 backward kernel, which keeps one chunk of recomputed states on chip).
+int default_ckpt_interval(int K, int V, int io_dtype);
+int max_ckpt_interval(int K, int V, int io_dtype);
+
+// fp32 FMA path (scan_f32.cu)
+cudaError_t launch_fwd_f32(const ScanArgs &a, cudaStream_t s);
+cudaError_t launch_bwd_f32(const ScanArgs &a, cudaStream_t s);
+
+// bf16 tensor-core path
+cudaError_t launch_fwd_bf16(const ScanArgs &a, cudaStream_t s);     // scan_fwd_bf16.cu
+cudaError_t launch_bwd_bf16(const ScanArgs &a, cudaStream_t s);     // scan_bwd_bf16.cu
+cudaError_t launch_decode_bf16(const ScanArgs &a, cudaStream_t s);  // decode_bf16.cu
+size_t bwd_bf16_extra_workspace(const ScanArgs &a);
+
+// reductions shared by both paths (reduce.cu)
+cudaError_t launch_reduce_dW(const float *dW_part, float *dW, int B, int N, int V, cudaStream_t s);
+cudaError_t launch_reduce_heads(const float *part, void *out, int io_dtype, size_t BT, int N,
+                                int Ng, int K, cudaStream_t s);
+
+}  // namespace m2rnn

@@ -35,6 +35,7 @@ class ScanConfig:
     gate_mean: float = 2.0       # gate pre-activations ~ N(gate_mean, 1)
     h0_std: float = 0.1          # 0 -> zero initial state (passed as NULL)
     dist: str = "baseline"       # "baseline" | "saturating" | "identity_w"
+    w_scale: float = 1.0         # W ~ N(0, w_scale^2 / V): 1 puts the recurrence at the edge of stability
     seed: int = 0
 
     @property
@@ -92,8 +93,10 @@ def make_inputs(cfg: ScanConfig, *, backward: bool = False, seed: int | None = N
     baseline:    q,k,v ~ N(0,1)/sqrt(K); W ~ N(0, 1/V) (std V^-1/2); gate ~ N(gate_mean,1);
                  h0 ~ N(0, h0_std^2) (None when h0_std == 0); dy ~ N(0,1).
     identity_w:  as baseline with W = I (the paper's initialisation of W).
-    saturating:  q,k,v ~ N(0,1); W = 1.5*I + N(0,1/V); h0 ~ U(-1,1): drives tanh well into
-                 its non-linear range so a wrong non-linearity cannot pass.
+    saturating:  q,k,v ~ N(0,1) (so k v^T has unit scale); W ~ N(0,1/V); h0 ~ U(-1,1): drives
+                 tanh well into its non-linear range so a wrong non-linearity cannot pass, while
+                 the map stays contracting (an expanding W would amplify rounding differences
+                 between any two correct implementations).
     """
     rng = np.random.Generator(np.random.PCG64(cfg.seed if seed is None else seed))
     io = torch_dtype(cfg.dtype)
@@ -108,11 +111,9 @@ def make_inputs(cfg: ScanConfig, *, backward: bool = False, seed: int | None = N
     if cfg.gate_kind == GATE_VALUE:
         gate = torch.sigmoid(gate)
     out["gate"] = gate
-    W = _normal(rng, (N, V, V), V ** -0.5)
+    W = _normal(rng, (N, V, V), cfg.w_scale * V ** -0.5)
     if cfg.dist == "identity_w":
         W = torch.eye(V).expand(N, V, V).clone()
-    elif sat:
-        W = W + 1.5 * torch.eye(V)
     out["W"] = W.to(io)
     if sat:
         out["h0"] = torch.from_numpy(rng.uniform(-1.0, 1.0, size=(B, N, K, V)).astype(np.float32))

@@ -1,0 +1,125 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol
+the header declares, and rejects bad arguments before launching anything."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2603_14360_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2603_14360_b200 import build
+    build.build()
+    return binding._lib()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    hdr = open(os.path.join(ROOT, "include", "m2rnn.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    names = set(re.findall(r"\b(m2rnn_[a-z0-9_]+)\s*\(", hdr))
+    assert {"m2rnn_fwd", "m2rnn_bwd", "m2rnn_decode_step"} <= names
+    for n in names:
+        assert hasattr(lib, n), n
+    assert names == set(binding.EXPORTS), "binding and header disagree"
+    assert lib.m2rnn_version() >= 100
+    assert b"NULL" in lib.m2rnn_status_string(-1)
+
+
+def _p(**kw):
+    base = dict(B=2, T=8, N=4, Nq=4, Nk=4, K=32, V=32, io_dtype=1, gate_kind=1, ckpt_interval=0, dh_clip=0.0)
+    base.update(kw)
+    return binding.Params(**base)
+
+
+FAKE = ctypes.c_void_p(0x10000)      # aligned, never dereferenced: every call below must fail first
+ODD = ctypes.c_void_p(0x10004)
+
+
+def _fwd(lib, p, **over):
+    a = dict(q=FAKE, k=FAKE, v=FAKE, gate=FAKE, W=FAKE, h0=None, alpha=None, beta=None, w_r=None,
+             y=FAKE, hT=None, ckpt=None, st=None, stream=None)
+    a.update(over)
+    return lib.m2rnn_fwd(ctypes.byref(p), *a.values())
+
+
+def test_fwd_rejects_bad_arguments(lib):
+    assert lib.m2rnn_fwd(None, *([FAKE] * 14)) == -1
+    assert _fwd(lib, _p(N=0)) == -2
+    assert _fwd(lib, _p(Nq=3)) == -2                  # does not divide N
+    assert _fwd(lib, _p(Nk=8)) == -2                  # more key heads than heads
+    assert _fwd(lib, _p(T=-1)) == -2
+    assert _fwd(lib, _p(K=24)) == -3                  # not a multiple of 16
+    assert _fwd(lib, _p(K=144)) == -3
+    assert _fwd(lib, _p(V=48)) == -3
+    assert _fwd(lib, _p(io_dtype=7)) == -3
+    assert _fwd(lib, _p(gate_kind=3)) == -3
+    assert _fwd(lib, _p(ckpt_interval=100000)) == -3
+    assert _fwd(lib, _p(), q=None) == -1
+    assert _fwd(lib, _p(), y=None) == -1
+    assert _fwd(lib, _p(gate_kind=2)) == -1           # psi needs alpha and beta
+    assert _fwd(lib, _p(), v=ODD) == -4
+    assert _fwd(lib, _p(), hT=ODD) == -4
+    # empty calls are fine and launch nothing
+    assert _fwd(lib, _p(T=0)) == 0
+    assert _fwd(lib, _p(B=0)) == 0
+
+
+def test_bwd_rejects_bad_arguments(lib):
+    p = _p()
+    need = lib.m2rnn_bwd_workspace_bytes(ctypes.byref(p), 0)
+    need_ck = lib.m2rnn_bwd_workspace_bytes(ctypes.byref(p), 1)
+    assert need > need_ck > 0
+    assert need - need_ck >= lib.m2rnn_ckpt_bytes(ctypes.byref(p)) > 0
+    ws = ctypes.c_void_p(0x20000)
+
+    def bwd(p, ws=ws, nbytes=need, **over):
+        a = dict(q=FAKE, k=FAKE, v=FAKE, gate=FAKE, W=FAKE, h0=None, alpha=None, beta=None, w_r=None,
+                 ckpt=None, dy=FAKE, d_hT=None, dq=FAKE, dk=FAKE, dv=FAKE, dgate=FAKE, dW=FAKE, dh0=None)
+        a.update(over)
+        return lib.m2rnn_bwd(ctypes.byref(p), *a.values(), ws, nbytes, None, None)
+
+    assert bwd(p, nbytes=need - 1) == -5
+    assert bwd(p, ws=None) == -5
+    assert bwd(p, ws=ctypes.c_void_p(0x20010)) == -4
+    assert bwd(p, dy=None) == -1
+    assert bwd(p, dW=None) == -1
+    assert bwd(p, dq=ODD) == -4
+    assert bwd(_p(V=8)) == -3
+    # shared q/k heads need per-head partial sums in the workspace
+    pm = _p(Nq=1, Nk=1)
+    assert lib.m2rnn_bwd_workspace_bytes(ctypes.byref(pm), 0) > need
+
+
+def test_decode_rejects_bad_arguments(lib):
+    def dec(p, **over):
+        a = dict(q=FAKE, k=FAKE, v=FAKE, gate=FAKE, W=FAKE, alpha=None, beta=None, w_r=None,
+                 state=FAKE, y=FAKE, st=None, stream=None)
+        a.update(over)
+        return lib.m2rnn_decode_step(ctypes.byref(p), *a.values())
+
+    assert dec(_p(), state=None) == -1
+    assert dec(_p(K=8)) == -3
+    assert dec(_p(), y=ODD) == -4
+    assert dec(_p(B=0)) == 0
+    assert dec(_p(T=-5, B=0)) == 0                    # T is ignored by the decode step
+
+
+def test_ckpt_interval_query(lib):
+    p = _p()
+    c = lib.m2rnn_ckpt_interval(ctypes.byref(p))
+    assert c >= 1
+    assert lib.m2rnn_ckpt_interval(ctypes.byref(_p(ckpt_interval=4))) == 4
+    assert lib.m2rnn_ckpt_bytes(ctypes.byref(_p(T=9, ckpt_interval=4))) == 2 * 4 * 3 * 32 * 32 * 4
+    assert lib.m2rnn_ckpt_interval(ctypes.byref(_p(V=7))) == -3
+
+
+def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
+    monkeypatch.setattr(binding, "_LIB", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "missing.so"))
+    with pytest.raises(ImportError):
+        binding.m2rnn_version()
