@@ -69,7 +69,8 @@ typedef struct {
   int32_t K, V;          /* state is K x V per (b,n); the transition matrix is V x V          */
   int32_t io_dtype;      /* m2rnn_dtype                                                       */
   int32_t gate_kind;     /* m2rnn_gate_kind                                                   */
-  int32_t ckpt_interval; /* steps between saved states; 0 = library default for (K,V,dtype)  */
+  int32_t ckpt_interval; /* steps between saved states; 0 = library default for (K,V,dtype);
+                            at most m2rnn_ckpt_interval's bound, and even for M2RNN_BF16        */
   float dh_clip;         /* <= 0: off.  Else the state gradient carried to the previous step is
                             clamped elementwise to [-dh_clip, dh_clip] after every reverse step
                             (section "Gradient Clipping"; the paper gives no threshold or form) */

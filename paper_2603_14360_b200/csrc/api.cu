@@ -18,7 +18,8 @@ int max_ckpt_interval(int K, int V, int io_dtype) {
 int default_ckpt_interval(int K, int V, int io_dtype) {
   if (io_dtype == M2RNN_F32) return 16;
   int c = max_ckpt_interval(K, V, io_dtype);
-  return c > 16 ? 16 : c;
+  c = c > 16 ? 16 : c;
+  return c < 2 ? 2 : (c & ~1);  // even: the bf16 kernels checkpoint between pairs of steps
 }
 
 namespace {
@@ -36,6 +37,8 @@ int check_params(const m2rnn_params *p, bool need_T) {
   if (p->V != 16 && p->V != 32 && p->V != 64 && p->V != 128) return M2RNN_ERR_UNSUPPORTED;
   if (p->ckpt_interval < 0 || p->ckpt_interval > max_ckpt_interval(p->K, p->V, p->io_dtype))
     return M2RNN_ERR_UNSUPPORTED;
+  // the bf16 kernels take steps in pairs and checkpoint between pairs
+  if (p->io_dtype == M2RNN_BF16 && (p->ckpt_interval & 1)) return M2RNN_ERR_UNSUPPORTED;
   return M2RNN_OK;
 }
 

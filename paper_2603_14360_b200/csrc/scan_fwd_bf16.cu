@@ -27,7 +27,7 @@ template <int V>
 struct FwdSmem {
   // Per stage (floats): q [TC][K], k [TC][K], v [TC][V], f [TC], ypart [TC][NW][V]
   __host__ __device__ static int stage_floats(int K, int TC) { return TC * (2 * K + V + 1 + (K / 16) * V); }
-  __host__ __device__ static int tc(int K) { return (V >= 128 || K > 64) ? 8 : 16; }
+  __host__ __device__ static constexpr int tc(int K) { return (V >= 128 || K > 64) ? 8 : 16; }
   __host__ static size_t bytes(int K) {
     const int TC = tc(K);
     size_t b = sizeof(float) * (size_t)kStages * stage_floats(K, TC);
@@ -36,8 +36,10 @@ struct FwdSmem {
   }
 };
 
-template <int V>
-__global__ void __launch_bounds__(288, 1) fwd_bf16_kernel(ScanArgs a) {
+// MAXW: most compute warps the instantiation is launched with (K <= 16*MAXW).  Registers are
+// granted per 4 warps: up to 4+1 warps leave 255 per thread, 8+1 warps only 168.
+template <int V, int MAXW>
+__global__ void __launch_bounds__((MAXW + 1) * 32, 1) fwd_bf16_kernel(ScanArgs a) {
   using G = TileGeom<V>;
   constexpr int NT = G::NT, KT = G::KT, SEG = G::SEG;
   constexpr bool kWInRegs = V <= 64;
@@ -45,7 +47,7 @@ __global__ void __launch_bounds__(288, 1) fwd_bf16_kernel(ScanArgs a) {
 
   const int K = a.K, N = a.N, T = a.T;
   const int NW = K >> 4;
-  const int TC = FwdSmem<V>::tc(K);
+  constexpr int TC = FwdSmem<V>::tc(MAXW * 16);   // K > 64 <=> MAXW == 8
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int bn = blockIdx.x, b = bn / N, n = bn % N;
   const int stage_floats = FwdSmem<V>::stage_floats(K, TC);
@@ -194,15 +196,6 @@ __global__ void __launch_bounds__(288, 1) fwd_bf16_kernel(ScanArgs a) {
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) H[nt][0] = H[nt][1] = H[nt][2] = H[nt][3] = 0.f;
   }
-  uint32_t A[KT][4];
-#pragma unroll
-  for (int kt = 0; kt < KT; ++kt) {
-    A[kt][0] = pack_bf16(H[2 * kt][0], H[2 * kt][1]);
-    A[kt][1] = pack_bf16(H[2 * kt][2], H[2 * kt][3]);
-    A[kt][2] = pack_bf16(H[2 * kt + 1][0], H[2 * kt + 1][1]);
-    A[kt][3] = pack_bf16(H[2 * kt + 1][2], H[2 * kt + 1][3]);
-  }
-
   auto store_state = [&](float *dst) {
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
@@ -214,97 +207,155 @@ __global__ void __launch_bounds__(288, 1) fwd_bf16_kernel(ScanArgs a) {
     }
   };
 
-  int ck_left = 0, ck_idx = 0;  // steps until the next checkpoint, index of the next checkpoint
-  for (int ch = 0; ch < nchunks; ++ch) {
-    const int s = ch % kStages, len = min(TC, T - ch * TC);
-    if (!mbar_wait(&full[s], (ch / kStages) & 1)) { report_timeout(a.dev_status); return; }
-    const float *qS = stages + (size_t)s * stage_floats, *kS = qS + TC * K, *vS = kS + TC * K, *fS = vS + TC * V;
-    float *yp = const_cast<float *>(fS) + TC;
-
-    for (int t = 0; t < len; ++t) {
-      if (a.ckpt) {
-        if (ck_left == 0) {
-          store_state(a.ckpt + ((size_t)bn * a.nchunks + ck_idx) * KV);
-          ++ck_idx;
-          ck_left = a.C;
-        }
-        --ck_left;
-      }
-      const float2 kk = *reinterpret_cast<const float2 *>(kS + t * K + row0);
-      const float f = fS[t];
-      float vv[SEG];
+  // P <- k v^T  (the outer-product term of Eq. 1 seeds the accumulators)
+  // (shared-memory operands of the hot loop are 32-bit shared addresses, in bytes)
+  auto seed = [&](float (&P)[NT][4], uint32_t krow, uint32_t vrow) {
+    const float2 kk = lds64(krow + 4 * row0);
 #pragma unroll
-      for (int x = 0; x < SEG / 4; ++x) {
-        const float4 t4 = *reinterpret_cast<const float4 *>(vS + t * V + SEG * c + 4 * x);
-        vv[4 * x] = t4.x; vv[4 * x + 1] = t4.y; vv[4 * x + 2] = t4.z; vv[4 * x + 3] = t4.w;
-      }
-      // Eq. 1: P = k v^T + H W
-      float P[NT][4];
+    for (int x = 0; x < SEG / 4; ++x) {
+      const float4 v4 = lds128(vrow + 4 * (SEG * c + 4 * x));
+      P[2 * x][0] = kk.x * v4.x; P[2 * x][1] = kk.x * v4.y; P[2 * x][2] = kk.y * v4.x; P[2 * x][3] = kk.y * v4.y;
+      P[2 * x + 1][0] = kk.x * v4.z; P[2 * x + 1][1] = kk.x * v4.w; P[2 * x + 1][2] = kk.y * v4.z; P[2 * x + 1][3] = kk.y * v4.w;
+    }
+  };
+  // P += A[kt] * W[kt][:]  : one k tile of H W
+  auto mma_ktile = [&](float (&P)[NT][4], const uint32_t (&Ak)[4], int kt) {
 #pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-        P[nt][0] = kk.x * vv[2 * nt]; P[nt][1] = kk.x * vv[2 * nt + 1];
-        P[nt][2] = kk.y * vv[2 * nt]; P[nt][3] = kk.y * vv[2 * nt + 1];
-      }
-#pragma unroll
-      for (int kt = 0; kt < KT; ++kt) {
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          if constexpr (kWInRegs) {
-            mma_bf16_16816(P[nt], A[kt], Wr[kt][nt][0], Wr[kt][nt][1]);
-          } else {
-            const uint2 w = Wf[(kt * NT + nt) * 32 + lane];
-            mma_bf16_16816(P[nt], A[kt], w.x, w.y);
-          }
-        }
-      }
-      // Eq. 2: H = Z + f (H - Z), Z = tanh(P); then the bf16 operand of the next step
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-          const float z = tanh_approx(P[nt][r]);
-          H[nt][r] = fmaf(f, H[nt][r] - z, z);
-        }
-      }
-#pragma unroll
-      for (int kt = 0; kt < KT; ++kt) {
-        A[kt][0] = pack_bf16(H[2 * kt][0], H[2 * kt][1]);
-        A[kt][1] = pack_bf16(H[2 * kt][2], H[2 * kt][3]);
-        A[kt][2] = pack_bf16(H[2 * kt + 1][0], H[2 * kt + 1][1]);
-        A[kt][3] = pack_bf16(H[2 * kt + 1][2], H[2 * kt + 1][3]);
-      }
-      // Eq. 3: this warp's share of H_t^T q_t
-      if (want_y) {
-        const float2 qq = *reinterpret_cast<const float2 *>(qS + t * K + row0);
-        float part[SEG];
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          part[2 * nt] = fmaf(qq.y, H[nt][2], qq.x * H[nt][0]);
-          part[2 * nt + 1] = fmaf(qq.y, H[nt][3], qq.x * H[nt][1]);
-        }
-        reduce_over_rows<SEG>(part, lane);
-        using RO = RowReduceOut<V>;
-        if (RO::owner(lane)) {
-          float *dst = yp + ((size_t)t * NW + warp) * V + RO::first_col(lane);
-          if constexpr (RO::CNT == 4) *reinterpret_cast<float4 *>(dst) = make_float4(part[0], part[1], part[2], part[3]);
-          else if constexpr (RO::CNT == 2) *reinterpret_cast<float2 *>(dst) = make_float2(part[0], part[1]);
-          else dst[0] = part[0];
-        }
+    for (int nt = 0; nt < NT; ++nt) {
+      if constexpr (kWInRegs) {
+        mma_bf16_16816(P[nt], Ak, Wr[kt][nt][0], Wr[kt][nt][1]);
+      } else {
+        const uint2 w = Wf[(kt * NT + nt) * 32 + lane];
+        mma_bf16_16816(P[nt], Ak, w.x, w.y);
       }
     }
+  };
+
+  // One step, software-pipelined by hand: while the MUFU works through tanh of step t, column
+  // tile pair by column tile pair, the tensor pipe already runs the k tiles of step t+1 that
+  // depend only on the pairs finished so far.  The body is branch-free (one basic block) so the
+  // instruction scheduler can interleave the MUFU, tensor and FMA streams.
+  //   Pc: H_{t-1} W + k_t v_t^T, complete (or in flight) on entry
+  //   Pn: receives H_t W + k_{t+1} v_{t+1}^T; after the last step it is fed a valid but
+  //       meaningless row and its result is never read
+  auto step = [&](float (&Pc)[NT][4], float (&Pn)[NT][4], float f, uint32_t qrow, uint32_t ydst,
+                  uint32_t krow_n, uint32_t vrow_n) {
+    seed(Pn, krow_n, vrow_n);
+    const float2 qq = lds64(qrow + 4 * row0);
+    float part[SEG];
+#pragma unroll
+    for (int kt = 0; kt < KT; ++kt) {
+#pragma unroll
+      for (int nt = 2 * kt; nt < 2 * kt + 2; ++nt) {
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          const float z = tanh_approx(Pc[nt][r]);          // Eq. 1
+          H[nt][r] = fmaf(f, H[nt][r] - z, z);             // Eq. 2: f H + (1-f) Z
+        }
+        part[2 * nt] = fmaf(qq.y, H[nt][2], qq.x * H[nt][0]);      // Eq. 3, this thread's two rows
+        part[2 * nt + 1] = fmaf(qq.y, H[nt][3], qq.x * H[nt][1]);
+      }
+      uint32_t Ak[4];
+      Ak[0] = pack_bf16(H[2 * kt][0], H[2 * kt][1]);
+      Ak[1] = pack_bf16(H[2 * kt][2], H[2 * kt][3]);
+      Ak[2] = pack_bf16(H[2 * kt + 1][0], H[2 * kt + 1][1]);
+      Ak[3] = pack_bf16(H[2 * kt + 1][2], H[2 * kt + 1][3]);
+      mma_ktile(Pn, Ak, kt);
+    }
+    reduce_over_rows<SEG>(part, lane);
+    using RO = RowReduceOut<V>;
+    if (RO::owner(lane)) {
+      const uint32_t dst = ydst + 4 * RO::first_col(lane);
+      if constexpr (RO::CNT == 4) sts128(dst, make_float4(part[0], part[1], part[2], part[3]));
+      else if constexpr (RO::CNT == 2) sts64(dst, make_float2(part[0], part[1]));
+      else sts32(dst, part[0]);
+    }
+  };
+
+  float P0[NT][4], P1[NT][4];
+  int ck_left = 0, ck_idx = 0;  // steps until the next checkpoint, index of the next checkpoint
+  auto maybe_checkpoint = [&](int steps) {   // called before an even-numbered step
+    if (a.ckpt) {
+      if (ck_left == 0) {
+        store_state(a.ckpt + ((size_t)bn * a.nchunks + ck_idx) * KV);
+        ++ck_idx;
+        ck_left = a.C;
+      }
+      ck_left -= steps;
+    }
+  };
+  const uint32_t stages_sa = smem_u32(stages);
+  auto stage_sa = [&](int s) { return stages_sa + 4u * (uint32_t)(s * stage_floats); };
+  // byte offsets of the arrays inside a stage
+  const uint32_t oK = 4u * TC * K, oV = 2 * oK, oF = oV + 4u * TC * V, oY = oF + 4u * TC;
+
+  if (T > 0) {
+    if (!mbar_wait(&full[0], 0)) { report_timeout(a.dev_status); return; }
+    // prologue: the first step's product from the initial state
+    seed(P0, stages_sa + oK, stages_sa + oV);
+#pragma unroll
+    for (int kt = 0; kt < KT; ++kt) {
+      uint32_t Ak[4];
+      Ak[0] = pack_bf16(H[2 * kt][0], H[2 * kt][1]);
+      Ak[1] = pack_bf16(H[2 * kt][2], H[2 * kt][3]);
+      Ak[2] = pack_bf16(H[2 * kt + 1][0], H[2 * kt + 1][1]);
+      Ak[3] = pack_bf16(H[2 * kt + 1][2], H[2 * kt + 1][3]);
+      mma_ktile(P0, Ak, kt);
+    }
+  }
+  // Steps are taken in pairs (P0 -> P1 -> P0); the two steps of a pair form one basic block, so
+  // the tail of the first (row reduction, last MMAs in flight) overlaps the head of the second.
+  // TC and the checkpoint interval are even: stage hand-over and checkpoints fall between pairs.
+  int ch = 0, tl = 0, s = 0;   // stage-sized chunk of the scan, step within it, its stage
+  for (int t = 0; t + 1 < T; t += 2) {
+    const uint32_t st = stage_sa(s);
+    const uint32_t yp = st + oY + 4u * ((tl * NW + warp) * V);
+    const bool cross = tl + 2 == TC, more = t + 2 < T;
+    const int sn = s + 1 == kStages ? 0 : s + 1;
+    uint32_t k2 = st + oK + 4u * ((tl + 1) * K), v2 = st + oV + 4u * ((tl + 1) * V);   // after the last step: any valid row
+    if (more) {
+      if (cross) {
+        if (!mbar_wait(&full[sn], ((ch + 1) / kStages) & 1)) { report_timeout(a.dev_status); return; }
+        k2 = stage_sa(sn) + oK;
+        v2 = stage_sa(sn) + oV;
+      } else {
+        k2 += 4u * K;
+        v2 += 4u * V;
+      }
+    }
+    maybe_checkpoint(2);
+    step(P0, P1, lds32(st + oF + 4u * tl), st + 4u * (tl * K), yp, st + oK + 4u * ((tl + 1) * K), st + oV + 4u * ((tl + 1) * V));
+    step(P1, P0, lds32(st + oF + 4u * (tl + 1)), st + 4u * ((tl + 1) * K), yp + 4u * (NW * V), k2, v2);
+    if (cross || !more) {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&done[s]);
+    }
+    tl += 2;
+    if (cross) { tl = 0; ++ch; s = sn; }
+  }
+  if (T & 1) {
+    const uint32_t st = stage_sa(s);
+    maybe_checkpoint(1);
+    step(P0, P1, lds32(st + oF + 4u * tl), st + 4u * (tl * K), st + oY + 4u * ((tl * NW + warp) * V),
+         st + oK + 4u * (tl * K), st + oV + 4u * (tl * V));
     __syncwarp();
     if (lane == 0) mbar_arrive(&done[s]);
   }
   if (a.hT) store_state(a.hT + bn * KV);
 }
 
+template <int V, int MAXW>
+cudaError_t launch_vw(const ScanArgs &a, cudaStream_t s) {
+  const size_t smem = FwdSmem<V>::bytes(a.K);
+  cudaError_t e = cudaFuncSetAttribute(fwd_bf16_kernel<V, MAXW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  fwd_bf16_kernel<V, MAXW><<<a.B * a.N, (a.K / 16 + 1) * 32, smem, s>>>(a);
+  return cudaGetLastError();
+}
+
 template <int V>
 cudaError_t launch_v(const ScanArgs &a, cudaStream_t s) {
-  const size_t smem = FwdSmem<V>::bytes(a.K);
-  cudaError_t e = cudaFuncSetAttribute(fwd_bf16_kernel<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
-  fwd_bf16_kernel<V><<<a.B * a.N, (a.K / 16 + 1) * 32, smem, s>>>(a);
-  return cudaGetLastError();
+  return a.K <= 64 ? launch_vw<V, 4>(a, s) : launch_vw<V, 8>(a, s);
 }
 
 }  // namespace
