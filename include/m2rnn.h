@@ -123,6 +123,36 @@ int m2rnn_bwd(const m2rnn_params *params, const void *q, const void *k, const vo
               float *dh0, void *workspace, size_t workspace_bytes, int32_t *dev_status,
               void *stream);
 
+/* m2rnn_bwd without a workspace argument, for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this is a convenience of the library.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a plugin inside a host
+ * application that owns the allocator and hands out only input/output buffers, a real-time or
+ * safety-reviewed service that forbids allocation after start-up, or a caller whose memory pool
+ * is exhausted or fragmented by the time the backward pass runs.  Such callers still pass every
+ * input and output tensor; only the scratch comes from the library.
+ *
+ * The scratch is a fixed array of M2RNN_STATIC_SCRATCH_BYTES inside the library's device image:
+ * every GPU that loads the library holds that much memory until the process exits, whether or
+ * not this function is ever called.  The function itself calls no allocating routine.
+ *   - A problem whose m2rnn_bwd_workspace_bytes(params, ckpt != NULL) exceeds
+ *     M2RNN_STATIC_SCRATCH_BYTES is refused with M2RNN_ERR_WORKSPACE before anything runs;
+ *     passing the checkpoints written by m2rnn_fwd lowers the need.
+ *   - The first call on each device looks up the array's device address (the device that is
+ *     current at the call); make that first call before starting any stream capture.
+ *   - All calls share the one array, which keeps whatever the last call left in it.  Nothing in
+ *     it has to start at zero (each call writes what it later reads), but two calls that overlap
+ *     on the GPU -- different streams, or different host threads -- race on it: run them one
+ *     after the other.
+ * Arguments, outputs and status codes are otherwise exactly those of m2rnn_bwd. */
+#define M2RNN_STATIC_SCRATCH_BYTES (8u << 20)
+int m2rnn_bwd_static_scratch(const m2rnn_params *params, const void *q, const void *k,
+                             const void *v, const float *gate, const void *W, const float *h0,
+                             const float *alpha, const float *beta, const void *w_r,
+                             const float *ckpt, const void *dy, const float *d_hT, void *dq,
+                             void *dk, void *dv, float *dgate, float *dW, float *dh0,
+                             int32_t *dev_status, void *stream);
+
 /* One decoding step on a cached state (Eq. 1-3 once; params->T is ignored).
  *   in : q [B,Nq,K], k [B,Nk,K], v [B,N,V], gate [B,N], W, alpha/beta/w_r as in m2rnn_fwd
  *   io : state [B,N,K,V] fp32, updated in place

@@ -55,8 +55,11 @@ EXPORTS = {
     "m2rnn_fwd": (ctypes.c_int, [_pp] + [_vp] * 14),
     "m2rnn_bwd_workspace_bytes": (ctypes.c_size_t, [_pp, ctypes.c_int]),
     "m2rnn_bwd": (ctypes.c_int, [_pp] + [_vp] * 19 + [ctypes.c_size_t, _vp, _vp]),
+    "m2rnn_bwd_static_scratch": (ctypes.c_int, [_pp] + [_vp] * 20),
     "m2rnn_decode_step": (ctypes.c_int, [_pp] + [_vp] * 12),
 }
+
+STATIC_SCRATCH_BYTES = 8 << 20   # M2RNN_STATIC_SCRATCH_BYTES
 
 
 def _lib() -> ctypes.CDLL:
@@ -213,6 +216,35 @@ def m2rnn_bwd(q, k, v, gate, W, h0, dy, d_hT=None, *, ckpt=None, gate_kind=GATE_
     if rc != 0:
         raise M2RNNError(rc, "m2rnn_bwd")
     return g
+
+
+def m2rnn_bwd_static_scratch(q, k, v, gate, W, h0, dy, d_hT=None, *, out, ckpt=None, gate_kind=GATE_LOGIT,
+                             alpha=None, beta=None, w_r=None, ckpt_interval=0, dh_clip=0.0, stream=None):
+    """Backward through time on the library's built-in scratch array, for callers that must not
+    allocate device memory (an embedding application that owns the allocator, a service that
+    forbids allocation after start-up).  Nothing is allocated here either: ``out`` must already
+    hold ``dq, dk, dv, dgate, dW`` (and ``dh0`` if wanted), which are written in place and
+    returned.  Problems that need more than ``STATIC_SCRATCH_BYTES`` of scratch raise
+    ``M2RNNError`` with ``M2RNN_ERR_WORKSPACE``; calls must not overlap on the GPU, because they
+    all share the one array."""
+    p = _params(q, k, v, W, gate_kind, ckpt_interval, dh_clip)
+    B, T, N, K, V, io = p.B, p.T, p.N, p.K, p.V, q.dtype
+    _chk(q, "q", (B, T, p.Nq, K), io); _chk(k, "k", (B, T, p.Nk, K), io); _chk(v, "v", (B, T, N, V), io)
+    _chk(gate, "gate", (B, T, N), torch.float32); _chk(W, "W", (N, V, V), io)
+    _chk(h0, "h0", (B, N, K, V), torch.float32); _chk(w_r, "w_r", (N, V), io)
+    _chk(alpha, "alpha", (N,), torch.float32); _chk(beta, "beta", (N,), torch.float32)
+    _chk(dy, "dy", (B, T, N, V), io); _chk(d_hT, "d_hT", (B, N, K, V), torch.float32)
+    _chk(out["dq"], "dq", q.shape, io); _chk(out["dk"], "dk", k.shape, io); _chk(out["dv"], "dv", v.shape, io)
+    _chk(out["dgate"], "dgate", gate.shape, torch.float32); _chk(out["dW"], "dW", (N, V, V), torch.float32)
+    _chk(out.get("dh0"), "dh0", (B, N, K, V), torch.float32)
+    rc = _lib().m2rnn_bwd_static_scratch(
+        ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(gate), _ptr(W), _ptr(h0), _ptr(alpha), _ptr(beta),
+        _ptr(w_r), _ptr(ckpt), _ptr(dy), _ptr(d_hT), _ptr(out["dq"]), _ptr(out["dk"]), _ptr(out["dv"]),
+        _ptr(out["dgate"]), _ptr(out["dW"]), _ptr(out.get("dh0")), _ptr(device_status_word(q.device)),
+        _stream(stream))
+    if rc != 0:
+        raise M2RNNError(rc, "m2rnn_bwd_static_scratch")
+    return out
 
 
 def m2rnn_decode_step(q, k, v, gate, W, state, *, gate_kind=GATE_LOGIT, alpha=None, beta=None,
