@@ -7,19 +7,30 @@
 
 namespace m2rnn {
 
-int max_ckpt_interval(int K, int V, int io_dtype) {
-  if (io_dtype == M2RNN_F32) return 64;  // recomputed states live in global scratch
-  // bf16: one chunk of recomputed states (bf16, K*V*2 bytes per step) stays in shared memory
-  const int per_step = K * V * 2;
-  int c = (128 * 1024) / per_step;
-  return c < 1 ? 1 : (c > 64 ? 64 : c);
-}
-
-int default_ckpt_interval(int K, int V, int io_dtype) {
-  if (io_dtype == M2RNN_F32) return 16;
-  int c = max_ckpt_interval(K, V, io_dtype);
-  c = c > 16 ? 16 : c;
-  return c < 2 ? 2 : (c & ~1);  // even: the bf16 kernels checkpoint between pairs of steps
+BwdPlan plan_bwd(int B, int N, int K, int V, int io_dtype) {
+  BwdPlan pl{};
+  if (io_dtype == M2RNN_F32) {  // recomputed states live in global scratch
+    pl.KC = K; pl.C = 16; pl.C_max = 64;
+    return pl;
+  }
+  // Rows per CTA: the largest slab that still spreads the problem over the SMs (rows are independent
+  // recurrences; a smaller slab only shortens the work per step).  V = 128 keeps the slab at 32 rows
+  // for the sake of registers.
+  constexpr int kSMs = 148;
+  const long units = (long)(B > 0 ? B : 1) * N;
+  const int cap = V > 64 ? 32 : 64;
+  int KC = 16;
+  for (int cand = 32; cand <= cap; cand *= 2)
+    if (K % cand == 0) KC = cand;
+  while (KC > 16 && units * (K / KC) < kSMs && units * (K / (KC / 2)) <= kSMs) KC /= 2;
+  pl.KC = KC;
+  // Checkpoint interval: as many steps as two chunk buffers fit in shared memory (even, <= 16)
+  constexpr size_t kSmemLimit = 227 * 1024;
+  int c = 16;
+  while (c > 2 && bwd_bf16_smem_bytes(KC, V, c) > kSmemLimit) c -= 2;
+  pl.C_max = c;
+  pl.C = c;
+  return pl;
 }
 
 namespace {
@@ -35,7 +46,7 @@ int check_params(const m2rnn_params *p, bool need_T) {
   if (p->gate_kind < M2RNN_GATE_VALUE || p->gate_kind > M2RNN_GATE_PSI) return M2RNN_ERR_UNSUPPORTED;
   if (p->K % 16 || p->K < 16 || p->K > 128) return M2RNN_ERR_UNSUPPORTED;
   if (p->V != 16 && p->V != 32 && p->V != 64 && p->V != 128) return M2RNN_ERR_UNSUPPORTED;
-  if (p->ckpt_interval < 0 || p->ckpt_interval > max_ckpt_interval(p->K, p->V, p->io_dtype))
+  if (p->ckpt_interval < 0 || p->ckpt_interval > plan_bwd(p->B, p->N, p->K, p->V, p->io_dtype).C_max)
     return M2RNN_ERR_UNSUPPORTED;
   // the bf16 kernels take steps in pairs and checkpoint between pairs
   if (p->io_dtype == M2RNN_BF16 && (p->ckpt_interval & 1)) return M2RNN_ERR_UNSUPPORTED;
@@ -43,11 +54,11 @@ int check_params(const m2rnn_params *p, bool need_T) {
 }
 
 int interval_of(const m2rnn_params *p) {
-  return p->ckpt_interval ? p->ckpt_interval : default_ckpt_interval(p->K, p->V, p->io_dtype);
+  return p->ckpt_interval ? p->ckpt_interval : plan_bwd(p->B, p->N, p->K, p->V, p->io_dtype).C;
 }
 
 struct Workspace {
-  size_t ckpt, dW_part, dq_part, dk_part, chunk_states, total;
+  size_t ckpt, dW_part, dq_part, dk_part, chunk_states, dv_part, dgate_part, total;
 };
 
 Workspace layout(const m2rnn_params *p, bool have_ckpt) {
@@ -58,14 +69,19 @@ Workspace layout(const m2rnn_params *p, bool have_ckpt) {
   size_t off = 0;
   w.ckpt = off;
   if (!have_ckpt) off += align_up(BN * nch * KV * sizeof(float));
+  const int RS = p->K / plan_bwd(p->B, p->N, p->K, p->V, p->io_dtype).KC;   // row slabs per state (1 on the fp32 path)
   w.dW_part = off;
-  off += align_up(BN * p->V * p->V * sizeof(float));
+  off += align_up(BN * RS * p->V * p->V * sizeof(float));
   w.dq_part = off;
   if (p->Nq < p->N) off += align_up((size_t)p->B * p->T * p->N * p->K * sizeof(float));
   w.dk_part = off;
   if (p->Nk < p->N) off += align_up((size_t)p->B * p->T * p->N * p->K * sizeof(float));
   w.chunk_states = off;
   if (p->io_dtype == M2RNN_F32) off += align_up(BN * C * KV * sizeof(float));
+  w.dv_part = off;
+  if (RS > 1) off += align_up((size_t)RS * p->B * p->T * p->N * p->V * sizeof(float));
+  w.dgate_part = off;
+  if (RS > 1) off += align_up((size_t)RS * p->B * p->T * p->N * sizeof(float));
   w.total = off;
   return w;
 }
@@ -74,6 +90,7 @@ ScanArgs base_args(const m2rnn_params *p) {
   ScanArgs a{};
   a.B = p->B; a.T = p->T; a.N = p->N; a.Nq = p->Nq; a.Nk = p->Nk; a.K = p->K; a.V = p->V;
   a.gate_kind = p->gate_kind;
+  a.KC = plan_bwd(p->B, p->N, p->K, p->V, p->io_dtype).KC;
   a.C = interval_of(p);
   a.nchunks = p->T > 0 ? (p->T + a.C - 1) / a.C : 0;
   a.dh_clip = p->dh_clip;
@@ -195,11 +212,20 @@ int m2rnn_bwd(const m2rnn_params *params, const void *q, const void *k, const vo
   a.dq_part = params->Nq < params->N ? reinterpret_cast<float *>(ws + w.dq_part) : nullptr;
   a.dk_part = params->Nk < params->N ? reinterpret_cast<float *>(ws + w.dk_part) : nullptr;
   a.chunk_states = f32 ? reinterpret_cast<float *>(ws + w.chunk_states) : nullptr;
+  const int RS = params->K / a.KC;
+  a.dv_part = RS > 1 ? reinterpret_cast<float *>(ws + w.dv_part) : nullptr;
+  a.dgate_part = RS > 1 ? reinterpret_cast<float *>(ws + w.dgate_part) : nullptr;
   e = f32 ? launch_bwd_f32(a, s) : launch_bwd_bf16(a, s);
   if (e != cudaSuccess) return M2RNN_ERR_CUDA;
-  e = launch_reduce_dW(a.dW_part, dW, params->B, params->N, params->V, s);
+  e = launch_reduce_dW(a.dW_part, dW, params->B * RS, params->N, params->V, s);
   if (e != cudaSuccess) return M2RNN_ERR_CUDA;
   const size_t BT = (size_t)params->B * params->T;
+  if (RS > 1) {
+    e = launch_reduce_slabs(a.dv_part, dv, params->io_dtype, RS, BT * params->N * params->V, s);
+    if (e != cudaSuccess) return M2RNN_ERR_CUDA;
+    e = launch_reduce_slabs(a.dgate_part, dgate, M2RNN_F32, RS, BT * params->N, s);
+    if (e != cudaSuccess) return M2RNN_ERR_CUDA;
+  }
   if (a.dq_part) {
     e = launch_reduce_heads(a.dq_part, dq, params->io_dtype, BT, params->N, params->Nq, params->K, s);
     if (e != cudaSuccess) return M2RNN_ERR_CUDA;

@@ -13,6 +13,7 @@ namespace m2rnn {
 struct ScanArgs {
   int B, T, N, Nq, Nk, K, V;
   int gate_kind;
+  int KC;         // bf16 backward: state rows per CTA (a divisor of K)
   int C;          // checkpoint interval (steps)
   int nchunks;    // ceil(T / C)
   float dh_clip;
@@ -26,7 +27,9 @@ struct ScanArgs {
   const float *d_hT;
   void *dq, *dk, *dv;  // dq/dk: final tensors when the head is not shared, else see dq_part
   float *dgate, *dh0;
-  float *dW_part;      // [B,N,V,V] per-(b,n) partial sums of dW
+  float *dW_part;      // [B*K/KC,N,V,V] per-CTA partial sums of dW
+  float *dv_part;      // [K/KC][B,T,N,V] fp32 per-row-slab dv when K/KC > 1, else null
+  float *dgate_part;   // [K/KC][B,T,N] fp32 per-row-slab dgate when K/KC > 1, else null
   float *dq_part;      // [B,T,N,K] fp32 per-head dq when Nq < N, else null
   float *dk_part;      // [B,T,N,K] fp32 per-head dk when Nk < N, else null
   float *chunk_states; // fp32 path: [B*N, C, K, V] scratch for the recomputed states
@@ -36,10 +39,15 @@ struct ScanArgs {
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
-// Default / maximum checkpoint interval for a problem (bounded by shared memory in the
-// bf16 backward kernel, which keeps one chunk of recomputed states on chip).
-int default_ckpt_interval(int K, int V, int io_dtype);
-int max_ckpt_interval(int K, int V, int io_dtype);
+// How the backward pass splits a problem: state rows per CTA and the checkpoint interval (bounded
+// by shared memory in the bf16 backward kernel, which keeps two chunks of recomputed states on chip).
+struct BwdPlan {
+  int KC;     // rows per CTA (== K on the fp32 path)
+  int C;      // default checkpoint interval
+  int C_max;  // largest supported checkpoint interval
+};
+BwdPlan plan_bwd(int B, int N, int K, int V, int io_dtype);
+size_t bwd_bf16_smem_bytes(int KC, int V, int C);  // scan_bwd_bf16.cu
 
 // fp32 FMA path (scan_f32.cu)
 cudaError_t launch_fwd_f32(const ScanArgs &a, cudaStream_t s);
@@ -49,10 +57,10 @@ cudaError_t launch_bwd_f32(const ScanArgs &a, cudaStream_t s);
 cudaError_t launch_fwd_bf16(const ScanArgs &a, cudaStream_t s);     // scan_fwd_bf16.cu
 cudaError_t launch_bwd_bf16(const ScanArgs &a, cudaStream_t s);     // scan_bwd_bf16.cu
 cudaError_t launch_decode_bf16(const ScanArgs &a, cudaStream_t s);  // decode_bf16.cu
-size_t bwd_bf16_extra_workspace(const ScanArgs &a);
 
 // reductions shared by both paths (reduce.cu)
 cudaError_t launch_reduce_dW(const float *dW_part, float *dW, int B, int N, int V, cudaStream_t s);
+cudaError_t launch_reduce_slabs(const float *part, void *out, int io_dtype, int R, size_t n, cudaStream_t s);
 cudaError_t launch_reduce_heads(const float *part, void *out, int io_dtype, size_t BT, int N,
                                 int Ng, int K, cudaStream_t s);
 

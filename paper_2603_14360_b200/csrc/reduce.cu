@@ -32,7 +32,27 @@ __global__ void reduce_heads_kernel(const float *__restrict__ part, TIO *__restr
   out[x] = from_f32<TIO>(s);
 }
 
+// out[x] = sum_r part[r][x]: sums over the row slabs of a state that were handled by different CTAs
+// (dv and dgate are sums over all K rows)
+template <typename TIO>
+__global__ void reduce_slabs_kernel(const float *__restrict__ part, TIO *__restrict__ out, int R, size_t n) {
+  const size_t x = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (x >= n) return;
+  float s = 0.f;
+  for (int r = 0; r < R; ++r) s += part[(size_t)r * n + x];
+  out[x] = from_f32<TIO>(s);
+}
+
 }  // namespace
+
+cudaError_t launch_reduce_slabs(const float *part, void *out, int io_dtype, int R, size_t n, cudaStream_t s) {
+  const unsigned grid = (unsigned)((n + 255) / 256);
+  if (io_dtype == M2RNN_F32)
+    reduce_slabs_kernel<float><<<grid, 256, 0, s>>>(part, static_cast<float *>(out), R, n);
+  else
+    reduce_slabs_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(part, static_cast<__nv_bfloat16 *>(out), R, n);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_reduce_dW(const float *dW_part, float *dW, int B, int N, int V, cudaStream_t s) {
   const size_t NVV = (size_t)N * V * V;

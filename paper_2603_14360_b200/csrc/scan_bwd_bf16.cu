@@ -1,4 +1,597 @@
+// bf16 tensor-core backward through time (Algorithm 2 with the carried state gradient) for sm_100a.
+//
+// One CTA per (b, n, row slab): the K rows of a state are independent recurrences, so a CTA owns
+// KC = 16*NWC of them.  Time is walked in chunks of C steps (the checkpoint interval), last chunk
+// first, by four kinds of warps that overlap through shared memory:
+//
+//   recompute warps (NWC)  start from the checkpoint of the chunk and redo its forward steps
+//                          (Eq. 1-2, the same arithmetic as the forward kernel), leaving for every
+//                          step H_{t-1} as a bf16 row-major tile and Z_t as fp16 fragments;
+//   reverse warps   (NWC)  carry C = dL/dH in registers and walk the chunk backwards:
+//                          G = C + q dy^T, dq, df, dX = (1-f) G (1 - Z^2), dk, dv,
+//                          C <- f G + dX W^T  (mma.sync, bf16 operands, fp32 accumulate);
+//                          dX is also left as a bf16 row-major tile;
+//   dW warps        (V/16) accumulate dW += H_{t-1}^T dX on tensor cores from the two tiles
+//                          (ldmatrix.trans operands), one 16-row slab of dW per warp, off the chain;
+//   service warp    (1)    stages q, k, v, dy and the gate for coming chunks, and reduces and writes
+//                          dq, dk, dv, dgate of finished ones.
+//
+// While the reverse warps sweep chunk c the recompute warps already work on chunk c-1 (two state
+// buffers).  Hand-over is by mbarriers; every wait is bounded and reports through dev_status.
+// Sums over rows that span CTAs (dv, dgate, dW) and over batch (dW) or shared heads (dq, dk) are
+// finished by fixed-order second-stage kernels.
+#include <cuda_fp16.h>
+
+#include "device_common.cuh"
 #include "internal.h"
+#include "mma_tile.cuh"
+#include "pipeline.cuh"
+
 namespace m2rnn {
-cudaError_t launch_bwd_bf16(const ScanArgs &, cudaStream_t) { return cudaErrorNotSupported; }
+namespace {
+
+constexpr int kRing = 4;         // chunk slots of staged inputs / outputs in flight
+constexpr int kBarBytes = 256;   // room for the mbarriers below
+
+// Byte offset of 16-byte chunk `chunk` of row `row` in a bf16 [rows][V] tile.  Chunks are
+// XOR-swizzled within 128-byte lines so that both the fragment-wise stores of the chain warps and
+// the ldmatrix reads of the dW warps (8 rows, same column chunk) spread over all banks.
+template <int V>
+__device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
+  constexpr int RB = 2 * V;
+  if constexpr (RB >= 128) {
+    return (uint32_t)(row * RB + ((chunk ^ (row & 7)) << 4));
+  } else {
+    const uint32_t lin = (uint32_t)(row * RB + (chunk << 4));
+    const uint32_t line = lin >> 7;
+    return (line << 7) | ((((lin >> 4) & 7u) ^ (line & 7u)) << 4);
+  }
 }
+
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr) : "memory");
+}
+
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ float2 unpack_f16(uint32_t x) {
+  return __half22float2(*reinterpret_cast<const __half2 *>(&x));
+}
+__device__ __forceinline__ float2 unpack_bf16(uint32_t x) {
+  return make_float2(__uint_as_float(x << 16), __uint_as_float(x & 0xffff0000u));
+}
+
+// B fragment (kt, nt) of W^T under the column relabelling of mma_tile.cuh: B[k = j][n = l] = W[l][j].
+template <int V>
+__device__ __forceinline__ void load_wt_fragment(const __nv_bfloat16 *__restrict__ Wn, int kt, int nt, int lane,
+                                                 uint32_t &b0, uint32_t &b1) {
+  using G = TileGeom<V>;
+  const int g = lane >> 2, c = lane & 3;
+  const int l = G::mem_col(8 * nt + g);
+  const int j0 = G::mem_col(16 * kt + 2 * c), j1 = G::mem_col(16 * kt + 2 * c + 1);
+  const int j2 = G::mem_col(16 * kt + 8 + 2 * c), j3 = G::mem_col(16 * kt + 8 + 2 * c + 1);
+  const uint16_t *w = reinterpret_cast<const uint16_t *>(Wn);
+  b0 = (uint32_t)w[l * V + j0] | ((uint32_t)w[l * V + j1] << 16);
+  b1 = (uint32_t)w[l * V + j2] | ((uint32_t)w[l * V + j3] << 16);
+}
+
+struct BwdLayout {
+  // all byte offsets from the start of dynamic shared memory
+  uint32_t wf, wtf, state, state_stride, ztile, dx, ring, slot_bytes, total;
+  // float offsets inside a ring slot
+  uint32_t oQ, oK, oV, oDY, oF, oDF, oDQ, oDK, oDVP, oDFP;
+};
+
+template <int V>
+__host__ __device__ inline BwdLayout bwd_layout(int KC, int C, bool w_in_smem) {
+  BwdLayout L{};
+  const int NWC = KC / 16;
+  uint32_t off = kBarBytes;
+  L.wf = off;
+  if (w_in_smem) off += (V / 16) * (V / 8) * 32 * 8;
+  L.wtf = off;
+  if (w_in_smem) off += (V / 16) * (V / 8) * 32 * 8;
+  L.state = off;                               // [2][C] x { H tile (bf16) | Z fragments (fp16) }
+  L.ztile = (uint32_t)KC * V * 2;              // offset of the Z part inside one step's block
+  L.state_stride = (uint32_t)KC * V * 4;       // bytes per step
+  off += 2u * C * L.state_stride;
+  L.dx = off;                                  // [2] dX tiles (bf16)
+  off += 2u * KC * V * 2;
+  L.ring = off;
+  L.oQ = 0; L.oK = L.oQ + C * KC; L.oV = L.oK + C * KC; L.oDY = L.oV + C * V; L.oF = L.oDY + C * V;
+  L.oDF = L.oF + C; L.oDQ = L.oDF + C; L.oDK = L.oDQ + C * KC; L.oDVP = L.oDK + C * KC;
+  L.oDFP = L.oDVP + C * NWC * V;
+  L.slot_bytes = (L.oDFP + C * NWC) * 4;
+  L.slot_bytes = (L.slot_bytes + 15u) & ~15u;
+  off += kRing * L.slot_bytes;
+  L.total = off;
+  return L;
+}
+
+template <int V, int NWC>
+__global__ void __launch_bounds__((2 * NWC + V / 16 + 1) * 32, 1) bwd_bf16_kernel(ScanArgs a) {
+  using G = TileGeom<V>;
+  constexpr int NT = G::NT, KT = G::KT, SEG = G::SEG;
+  constexpr int KC = 16 * NWC, NDW = V / 16;
+  constexpr bool kWInSmem = V > 64;
+  constexpr int CPR = SEG * 2 / 16;            // 16-byte chunks per thread-row of a tile (0 when V == 16)
+  extern __shared__ __align__(128) unsigned char smem[];
+
+  const int K = a.K, N = a.N, T = a.T, C = a.C, nch = a.nchunks;
+  const int RS = K / KC;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, c = lane & 3;
+  const int unit = blockIdx.x / RS, rs = blockIdx.x % RS;
+  const int b = unit / N, n = unit % N;
+  const int rbase = rs * KC;                   // first state row of this CTA
+  const size_t KV = (size_t)K * V;
+  const BwdLayout L = bwd_layout<V>(KC, C, kWInSmem);
+
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem);
+  uint64_t *in_full = bars;             // [kRing]
+  uint64_t *out_full = bars + kRing;    // [kRing]
+  uint64_t *st_ready = bars + 2 * kRing;      // [2]
+  uint64_t *st_free = st_ready + 2;           // [2]
+  uint64_t *dx_full = st_free + 2;            // [2]
+  uint64_t *dx_free = dx_full + 2;            // [2]
+  if (tid == 0) {
+    for (int s = 0; s < kRing; ++s) { mbar_init(&in_full[s], 1); mbar_init(&out_full[s], NWC); }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&st_ready[s], NWC); mbar_init(&st_free[s], NWC + NDW);
+      mbar_init(&dx_full[s], NWC); mbar_init(&dx_free[s], NDW);
+    }
+    fence_mbar_init();
+  }
+  const __nv_bfloat16 *Wn = static_cast<const __nv_bfloat16 *>(a.W) + (size_t)n * V * V;
+  uint2 *Wf = reinterpret_cast<uint2 *>(smem + L.wf), *WTf = reinterpret_cast<uint2 *>(smem + L.wtf);
+  if constexpr (kWInSmem) {
+    for (int x = tid; x < KT * NT * 32; x += blockDim.x) {
+      uint32_t b0, b1;
+      load_w_fragment<V>(Wn, x / (NT * 32), (x / 32) % NT, x & 31, b0, b1);
+      Wf[x] = make_uint2(b0, b1);
+      load_wt_fragment<V>(Wn, x / (NT * 32), (x / 32) % NT, x & 31, b0, b1);
+      WTf[x] = make_uint2(b0, b1);
+    }
+  }
+  __syncthreads();
+
+  const uint32_t sm0 = smem_u32(smem);
+  auto slot_f = [&](int j) { return reinterpret_cast<float *>(smem + L.ring + (uint32_t)(j & (kRing - 1)) * L.slot_bytes); };
+  auto slot_sa = [&](int j) { return sm0 + L.ring + (uint32_t)(j & (kRing - 1)) * L.slot_bytes; };
+  auto state_sa = [&](int j, int s) { return sm0 + L.state + (uint32_t)((j & 1) * C + s) * L.state_stride; };
+  // chunk j of the sweep covers steps [t0, t0 + len) of time chunk nch-1-j
+  auto chunk_t0 = [&](int j) { return (nch - 1 - j) * C; };
+  auto chunk_len = [&](int j) { return min(C, T - chunk_t0(j)); };
+
+  // Thread (g,c) of chain warp w owns state rows r0 = 16w+g and r0+8 (MMA rows g, g+8) and the
+  // SEG memory columns SEG*c .. SEG*c+SEG-1 (MMA columns 8nt+2c+e <-> memory column SEG*c+2nt+e).
+  // Pair index p = nt*2 + h names the packed pair (row r0+8h, memory columns SEG*c+2nt, +1).
+  auto tile_store = [&](uint32_t tile_sa, int w, const uint32_t (&p)[NT][2]) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int row = 16 * w + g + 8 * h;
+      if constexpr (CPR == 0) {   // V == 16: 8 bytes per thread-row
+        const uint32_t addr = tile_sa + tile_off<V>(row, c >> 1) + 8u * (c & 1);
+        asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(addr), "r"(p[0][h]), "r"(p[1][h]) : "memory");
+      } else {
+#pragma unroll
+        for (int x = 0; x < CPR; ++x) {
+          const uint32_t addr = tile_sa + tile_off<V>(row, CPR * c + x);
+          asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(p[4 * x][h]), "r"(p[4 * x + 1][h]),
+                       "r"(p[4 * x + 2][h]), "r"(p[4 * x + 3][h]) : "memory");
+        }
+      }
+    }
+  };
+  auto tile_load = [&](uint32_t tile_sa, int w, uint32_t (&p)[NT][2]) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int row = 16 * w + g + 8 * h;
+      if constexpr (CPR == 0) {
+        const uint32_t addr = tile_sa + tile_off<V>(row, c >> 1) + 8u * (c & 1);
+        asm volatile("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(p[0][h]), "=r"(p[1][h]) : "r"(addr));
+      } else {
+#pragma unroll
+        for (int x = 0; x < CPR; ++x) {
+          const uint32_t addr = tile_sa + tile_off<V>(row, CPR * c + x);
+          asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];"
+                       : "=r"(p[4 * x][h]), "=r"(p[4 * x + 1][h]), "=r"(p[4 * x + 2][h]), "=r"(p[4 * x + 3][h]) : "r"(addr));
+        }
+      }
+    }
+  };
+  // Z fragments: private to the (warp, lane) pair that wrote them, 2*NT words per thread
+  auto zfrag_sa = [&](uint32_t step_sa, int w) { return step_sa + L.ztile + (uint32_t)(w * (2 * NT) * 32 + lane) * 4u; };
+
+  if (warp < NWC) {
+    // ================================================================= recompute warps
+    const int w = warp, r0 = 16 * w + g;
+    uint32_t Wr[kWInSmem ? 1 : KT][kWInSmem ? 1 : NT][2];
+    if constexpr (!kWInSmem) {
+#pragma unroll
+      for (int kt = 0; kt < KT; ++kt)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) load_w_fragment<V>(Wn, kt, nt, lane, Wr[kt][nt][0], Wr[kt][nt][1]);
+    }
+    for (int j = 0; j < nch; ++j) {
+      const int len = chunk_len(j);
+      // the chunk's starting state: ckpt[b][n][chunk] = H before step t0 (fp32)
+      float H[NT][4];
+      const float *ck = a.ckpt + ((size_t)unit * nch + (nch - 1 - j)) * KV;
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const float *src = ck + (size_t)(rbase + r0 + 8 * h) * V + SEG * c;
+#pragma unroll
+        for (int x = 0; x < SEG / 4; ++x) {
+          const float4 t4 = *reinterpret_cast<const float4 *>(src + 4 * x);
+          H[2 * x][2 * h] = t4.x; H[2 * x][2 * h + 1] = t4.y; H[2 * x + 1][2 * h] = t4.z; H[2 * x + 1][2 * h + 1] = t4.w;
+        }
+      }
+      if (!mbar_wait(&in_full[j & (kRing - 1)], (j / kRing) & 1)) { report_timeout(a.dev_status); return; }
+      if (j >= 2 && !mbar_wait(&st_free[j & 1], ((j >> 1) - 1) & 1)) { report_timeout(a.dev_status); return; }
+      const uint32_t sl = slot_sa(j);
+      for (int s = 0; s < len; ++s) {
+        const uint32_t st = state_sa(j, s);
+        // H_{t-1} as bf16: the A operand of this step and the tile the dW and reverse warps read
+        uint32_t hp[NT][2];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) { hp[nt][0] = pack_bf16(H[nt][0], H[nt][1]); hp[nt][1] = pack_bf16(H[nt][2], H[nt][3]); }
+        tile_store(st, w, hp);
+        // P = k v^T + H W   (Eq. 1 before the non-linearity)
+        const float k0 = lds32(sl + 4u * (L.oK + s * KC + r0)), k1 = lds32(sl + 4u * (L.oK + s * KC + r0 + 8));
+        const float f = lds32(sl + 4u * (L.oF + s));
+        float P[NT][4];
+#pragma unroll
+        for (int x = 0; x < SEG / 4; ++x) {
+          const float4 v4 = lds128(sl + 4u * (L.oV + s * V + SEG * c + 4 * x));
+          P[2 * x][0] = k0 * v4.x; P[2 * x][1] = k0 * v4.y; P[2 * x][2] = k1 * v4.x; P[2 * x][3] = k1 * v4.y;
+          P[2 * x + 1][0] = k0 * v4.z; P[2 * x + 1][1] = k0 * v4.w; P[2 * x + 1][2] = k1 * v4.z; P[2 * x + 1][3] = k1 * v4.w;
+        }
+#pragma unroll
+        for (int kt = 0; kt < KT; ++kt) {
+          const uint32_t Ak[4] = {hp[2 * kt][0], hp[2 * kt][1], hp[2 * kt + 1][0], hp[2 * kt + 1][1]};
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) {
+            if constexpr (kWInSmem) {
+              const uint2 wv = Wf[(kt * NT + nt) * 32 + lane];
+              mma_bf16_16816(P[nt], Ak, wv.x, wv.y);
+            } else {
+              mma_bf16_16816(P[nt], Ak, Wr[kt][nt][0], Wr[kt][nt][1]);
+            }
+          }
+        }
+        // Z = tanh(P), kept as fp16 for the reverse sweep; H <- f H + (1-f) Z  (Eq. 2)
+        const uint32_t zs = zfrag_sa(st, w);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          float z[4];
+#pragma unroll
+          for (int r = 0; r < 4; ++r) {
+            z[r] = tanh_approx(P[nt][r]);
+            H[nt][r] = fmaf(f, H[nt][r] - z[r], z[r]);
+          }
+          asm volatile("st.shared.b32 [%0], %1;" ::"r"(zs + 4u * (2 * nt) * 32), "r"(pack_f16(z[0], z[1])) : "memory");
+          asm volatile("st.shared.b32 [%0], %1;" ::"r"(zs + 4u * (2 * nt + 1) * 32), "r"(pack_f16(z[2], z[3])) : "memory");
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&st_ready[j & 1]);
+    }
+    return;
+  }
+
+  if (warp < 2 * NWC) {
+    // ================================================================= reverse warps
+    const int w = warp - NWC, r0 = 16 * w + g;
+    uint32_t WTr[kWInSmem ? 1 : KT][kWInSmem ? 1 : NT][2];
+    if constexpr (!kWInSmem) {
+#pragma unroll
+      for (int kt = 0; kt < KT; ++kt)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) load_wt_fragment<V>(Wn, kt, nt, lane, WTr[kt][nt][0], WTr[kt][nt][1]);
+    }
+    float Cg[NT][4];   // carried dL/dH_t
+    if (a.d_hT) {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const float *src = a.d_hT + (size_t)unit * KV + (size_t)(rbase + r0 + 8 * h) * V + SEG * c;
+#pragma unroll
+        for (int x = 0; x < SEG / 4; ++x) {
+          const float4 t4 = *reinterpret_cast<const float4 *>(src + 4 * x);
+          Cg[2 * x][2 * h] = t4.x; Cg[2 * x][2 * h + 1] = t4.y; Cg[2 * x + 1][2 * h] = t4.z; Cg[2 * x + 1][2 * h + 1] = t4.w;
+        }
+      }
+    } else {
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) Cg[nt][0] = Cg[nt][1] = Cg[nt][2] = Cg[nt][3] = 0.f;
+    }
+    const float clip = a.dh_clip;
+    int nstep = 0;   // steps taken so far: picks the dX tile
+    for (int j = 0; j < nch; ++j) {
+      const int len = chunk_len(j);
+      if (!mbar_wait(&in_full[j & (kRing - 1)], (j / kRing) & 1)) { report_timeout(a.dev_status); return; }
+      if (!mbar_wait(&st_ready[j & 1], (j >> 1) & 1)) { report_timeout(a.dev_status); return; }
+      const uint32_t sl = slot_sa(j);
+      for (int s = len - 1; s >= 0; --s, ++nstep) {
+        const uint32_t st = state_sa(j, s);
+        uint32_t hp[NT][2];
+        tile_load(st, w, hp);
+        const uint32_t zs = zfrag_sa(st, w);
+        const float f = lds32(sl + 4u * (L.oF + s));
+        const float q0 = lds32(sl + 4u * (L.oQ + s * KC + r0)), q1 = lds32(sl + 4u * (L.oQ + s * KC + r0 + 8));
+        const float k0 = lds32(sl + 4u * (L.oK + s * KC + r0)), k1 = lds32(sl + 4u * (L.oK + s * KC + r0 + 8));
+        const float omf = 1.f - f;
+        float dq0 = 0.f, dq1 = 0.f, dk0 = 0.f, dk1 = 0.f, df = 0.f;
+        float dvp[SEG];
+        uint32_t xp[NT][2];   // dX as bf16 pairs: the A operand of dX W^T and the tile of the dW warps
+#pragma unroll
+        for (int x = 0; x < SEG / 4; ++x) {
+          const float4 dy4 = lds128(sl + 4u * (L.oDY + s * V + SEG * c + 4 * x));
+          const float4 v4 = lds128(sl + 4u * (L.oV + s * V + SEG * c + 4 * x));
+          const float dyv[4] = {dy4.x, dy4.y, dy4.z, dy4.w}, vv[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            const int nt = 2 * x + u;
+            uint32_t zw0, zw1;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(zw0) : "r"(zs + 4u * (2 * nt) * 32));
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(zw1) : "r"(zs + 4u * (2 * nt + 1) * 32));
+            const float2 za = unpack_f16(zw0), zb = unpack_f16(zw1);
+            const float2 ha = unpack_bf16(hp[nt][0]), hb = unpack_bf16(hp[nt][1]);
+            const float z[4] = {za.x, za.y, zb.x, zb.y}, hprev[4] = {ha.x, ha.y, hb.x, hb.y};
+            float dX[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+              const float dyc = dyv[2 * u + (r & 1)], vc = vv[2 * u + (r & 1)];
+              const float qr = (r & 2) ? q1 : q0;
+              const float Gv = fmaf(qr, dyc, Cg[nt][r]);        // G = C + q dy^T
+              const float D = hprev[r] - z[r];                  // H_{t-1} - Z
+              const float ht = fmaf(f, D, z[r]);                // H_t
+              if (r & 2) dq1 = fmaf(ht, dyc, dq1); else dq0 = fmaf(ht, dyc, dq0);   // dq = H_t dy
+              df = fmaf(Gv, D, df);                             // df = sum G (.) (H_{t-1} - Z)
+              dX[r] = omf * Gv * fmaf(-z[r], z[r], 1.f);        // through the gate and tanh
+              if (r & 2) dk1 = fmaf(dX[r], vc, dk1); else dk0 = fmaf(dX[r], vc, dk0);  // dk = dX v
+              Cg[nt][r] = f * Gv;                               // gated path into H_{t-1}
+            }
+            dvp[4 * x + 2 * u] = fmaf(dX[2], k1, dX[0] * k0);   // dv = dX^T k, this thread's two rows
+            dvp[4 * x + 2 * u + 1] = fmaf(dX[3], k1, dX[1] * k0);
+            xp[nt][0] = pack_bf16(dX[0], dX[1]);
+            xp[nt][1] = pack_bf16(dX[2], dX[3]);
+          }
+        }
+        // hand dX to the dW warps
+        const int xb = nstep & 1;
+        if (nstep >= 2 && !mbar_wait(&dx_free[xb], ((nstep >> 1) - 1) & 1)) { report_timeout(a.dev_status); return; }
+        tile_store(sm0 + L.dx + (uint32_t)xb * (KC * V * 2), w, xp);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&dx_full[xb]);
+        // C_{t-1} = f G + dX W^T
+#pragma unroll
+        for (int kt = 0; kt < KT; ++kt) {
+          const uint32_t Ak[4] = {xp[2 * kt][0], xp[2 * kt][1], xp[2 * kt + 1][0], xp[2 * kt + 1][1]};
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) {
+            if constexpr (kWInSmem) {
+              const uint2 wv = WTf[(kt * NT + nt) * 32 + lane];
+              mma_bf16_16816(Cg[nt], Ak, wv.x, wv.y);
+            } else {
+              mma_bf16_16816(Cg[nt], Ak, WTr[kt][nt][0], WTr[kt][nt][1]);
+            }
+          }
+        }
+        if (clip > 0.f) {
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int r = 0; r < 4; ++r) Cg[nt][r] = fminf(fmaxf(Cg[nt][r], -clip), clip);
+        }
+        // row sums over the 4 lanes of a row group, column sums over the 8 row groups
+        dq0 += __shfl_xor_sync(0xffffffffu, dq0, 1); dq1 += __shfl_xor_sync(0xffffffffu, dq1, 1);
+        dk0 += __shfl_xor_sync(0xffffffffu, dk0, 1); dk1 += __shfl_xor_sync(0xffffffffu, dk1, 1);
+        dq0 += __shfl_xor_sync(0xffffffffu, dq0, 2); dq1 += __shfl_xor_sync(0xffffffffu, dq1, 2);
+        dk0 += __shfl_xor_sync(0xffffffffu, dk0, 2); dk1 += __shfl_xor_sync(0xffffffffu, dk1, 2);
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) df += __shfl_xor_sync(0xffffffffu, df, off);
+        if (c == 0) {
+          sts32(sl + 4u * (L.oDQ + s * KC + r0), dq0); sts32(sl + 4u * (L.oDQ + s * KC + r0 + 8), dq1);
+          sts32(sl + 4u * (L.oDK + s * KC + r0), dk0); sts32(sl + 4u * (L.oDK + s * KC + r0 + 8), dk1);
+        }
+        if (lane == 0) sts32(sl + 4u * (L.oDFP + s * NWC + w), df);
+        reduce_over_rows<SEG>(dvp, lane);
+        using RO = RowReduceOut<V>;
+        if (RO::owner(lane)) {
+          const uint32_t dst = sl + 4u * (L.oDVP + (s * NWC + w) * V + RO::first_col(lane));
+          if constexpr (RO::CNT == 4) sts128(dst, make_float4(dvp[0], dvp[1], dvp[2], dvp[3]));
+          else if constexpr (RO::CNT == 2) sts64(dst, make_float2(dvp[0], dvp[1]));
+          else sts32(dst, dvp[0]);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(&st_free[j & 1]); mbar_arrive(&out_full[j & (kRing - 1)]); }
+    }
+    if (a.dh0) {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        float *dst = a.dh0 + (size_t)unit * KV + (size_t)(rbase + r0 + 8 * h) * V + SEG * c;
+#pragma unroll
+        for (int x = 0; x < SEG / 4; ++x)
+          *reinterpret_cast<float4 *>(dst + 4 * x) =
+              make_float4(Cg[2 * x][2 * h], Cg[2 * x][2 * h + 1], Cg[2 * x + 1][2 * h], Cg[2 * x + 1][2 * h + 1]);
+      }
+    }
+    return;
+  }
+
+  if (warp < 2 * NWC + NDW) {
+    // ================================================================= dW warps
+    // warp d owns dW rows l in [16d, 16d+16): acc += H_{t-1}[:, l]^T dX, contraction over the CTA's rows
+    const int d = warp - 2 * NWC;
+    float acc[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+    const int mi = lane >> 3, mr = lane & 7;   // ldmatrix: lane supplies row mr of matrix mi
+    int nstep = 0;
+    for (int j = 0; j < nch; ++j) {
+      const int len = chunk_len(j);
+      if (!mbar_wait(&st_ready[j & 1], (j >> 1) & 1)) { report_timeout(a.dev_status); return; }
+      for (int s = len - 1; s >= 0; --s, ++nstep) {
+        const int xb = nstep & 1;
+        if (!mbar_wait(&dx_full[xb], (nstep >> 1) & 1)) { report_timeout(a.dev_status); return; }
+        const uint32_t ht = state_sa(j, s), xt = sm0 + L.dx + (uint32_t)xb * (KC * V * 2);
+#pragma unroll
+        for (int kt = 0; kt < NWC; ++kt) {
+          // A = H_{t-1}^T: matrices (i 0-7, l 0-7), (i 0-7, l 8-15), (i 8-15, l 0-7), (i 8-15, l 8-15)
+          uint32_t A[4];
+          ldmatrix_x4_trans(ht + tile_off<V>(16 * kt + mr + 8 * (mi >> 1), 2 * d + (mi & 1)), A[0], A[1], A[2], A[3]);
+#pragma unroll
+          for (int np = 0; np < NT / 2; ++np) {
+            // B = dX: matrices (i 0-7, j-tile 2np), (i 8-15, 2np), (i 0-7, 2np+1), (i 8-15, 2np+1)
+            uint32_t b0, b1, b2, b3;
+            ldmatrix_x4_trans(xt + tile_off<V>(16 * kt + mr + 8 * (mi & 1), 2 * np + (mi >> 1)), b0, b1, b2, b3);
+            mma_bf16_16816(acc[2 * np], A, b0, b1);
+            mma_bf16_16816(acc[2 * np + 1], A, b2, b3);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&dx_free[xb]);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&st_free[j & 1]);
+    }
+    float *dWp = a.dW_part + ((size_t)(b * RS + rs) * N + n) * V * V;   // one partial per CTA, [b][slab][n]
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      *reinterpret_cast<float2 *>(dWp + (size_t)(16 * d + g) * V + 8 * nt + 2 * c) = make_float2(acc[nt][0], acc[nt][1]);
+      *reinterpret_cast<float2 *>(dWp + (size_t)(16 * d + g + 8) * V + 8 * nt + 2 * c) = make_float2(acc[nt][2], acc[nt][3]);
+    }
+    return;
+  }
+
+  // =================================================================== service warp
+  {
+    const int hq = n / (N / a.Nq), hk = n / (N / a.Nk);
+    const float al = a.alpha ? a.alpha[n] : 1.f, be = a.beta ? a.beta[n] : 0.f;
+    const __nv_bfloat16 *qg = static_cast<const __nv_bfloat16 *>(a.q), *kg = static_cast<const __nv_bfloat16 *>(a.k);
+    const __nv_bfloat16 *vg = static_cast<const __nv_bfloat16 *>(a.v), *dyg = static_cast<const __nv_bfloat16 *>(a.dy);
+    const __nv_bfloat16 *wr = static_cast<const __nv_bfloat16 *>(a.w_r);
+    const size_t BT = (size_t)a.B * T;
+    auto fill = [&](int j) {
+      float *sf = slot_f(j);
+      const int t0 = chunk_t0(j), len = chunk_len(j);
+      const size_t bt0 = (size_t)b * T + t0;
+      const int kc8 = KC / 8, v8 = V / 8;
+      for (int x = lane; x < len * kc8; x += 32) {
+        const int t = x / kc8, i = (x % kc8) * 8;
+        store8_bf16_as_f32(sf + L.oQ + t * KC + i, *reinterpret_cast<const uint4 *>(qg + ((bt0 + t) * a.Nq + hq) * K + rbase + i));
+        store8_bf16_as_f32(sf + L.oK + t * KC + i, *reinterpret_cast<const uint4 *>(kg + ((bt0 + t) * a.Nk + hk) * K + rbase + i));
+      }
+      for (int x = lane; x < len * v8; x += 32) {
+        const int t = x / v8, i = (x % v8) * 8;
+        store8_bf16_as_f32(sf + L.oV + t * V + i, *reinterpret_cast<const uint4 *>(vg + ((bt0 + t) * N + n) * V + i));
+        store8_bf16_as_f32(sf + L.oDY + t * V + i, *reinterpret_cast<const uint4 *>(dyg + ((bt0 + t) * N + n) * V + i));
+      }
+      if (lane < len) {
+        float dfdx;
+        sf[L.oF + lane] = gate_value(a.gate_kind, a.gate[(bt0 + lane) * N + n], al, be, &dfdx);
+        sf[L.oDF + lane] = dfdx;
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&in_full[j & (kRing - 1)]);
+    };
+    auto flush = [&](int j) {
+      const float *sf = slot_f(j);
+      const int t0 = chunk_t0(j), len = chunk_len(j);
+      const size_t bt0 = (size_t)b * T + t0;
+      // dq, dk: this CTA's rows
+      for (int x = lane; x < len * (KC / 2); x += 32) {
+        const int t = x / (KC / 2), i = (x % (KC / 2)) * 2;
+        const float2 dq2 = *reinterpret_cast<const float2 *>(sf + L.oDQ + t * KC + i);
+        const float2 dk2 = *reinterpret_cast<const float2 *>(sf + L.oDK + t * KC + i);
+        if (a.dq_part) *reinterpret_cast<float2 *>(a.dq_part + ((bt0 + t) * N + n) * K + rbase + i) = dq2;
+        else *reinterpret_cast<uint32_t *>(static_cast<__nv_bfloat16 *>(a.dq) + ((bt0 + t) * a.Nq + hq) * K + rbase + i) = pack_bf16(dq2.x, dq2.y);
+        if (a.dk_part) *reinterpret_cast<float2 *>(a.dk_part + ((bt0 + t) * N + n) * K + rbase + i) = dk2;
+        else *reinterpret_cast<uint32_t *>(static_cast<__nv_bfloat16 *>(a.dk) + ((bt0 + t) * a.Nk + hk) * K + rbase + i) = pack_bf16(dk2.x, dk2.y);
+      }
+      // dv: sum of the reverse warps' column sums (+ w_r (.) dy from Eq. 3, added by the first row slab only)
+      for (int x = lane; x < len * (V / 2); x += 32) {
+        const int t = x / (V / 2), jj = (x % (V / 2)) * 2;
+        float s0 = 0.f, s1 = 0.f;
+        for (int w = 0; w < NWC; ++w) {
+          const float2 p = *reinterpret_cast<const float2 *>(sf + L.oDVP + (t * NWC + w) * V + jj);
+          s0 += p.x; s1 += p.y;
+        }
+        if (wr && rs == 0) {
+          s0 = fmaf(__bfloat162float(wr[(size_t)n * V + jj]), sf[L.oDY + t * V + jj], s0);
+          s1 = fmaf(__bfloat162float(wr[(size_t)n * V + jj + 1]), sf[L.oDY + t * V + jj + 1], s1);
+        }
+        const size_t o = ((bt0 + t) * N + n) * V + jj;
+        if (a.dv_part) *reinterpret_cast<float2 *>(a.dv_part + (size_t)rs * BT * N * V + o) = make_float2(s0, s1);
+        else *reinterpret_cast<uint32_t *>(static_cast<__nv_bfloat16 *>(a.dv) + o) = pack_bf16(s0, s1);
+      }
+      if (lane < len) {
+        float s = 0.f;
+        for (int w = 0; w < NWC; ++w) s += sf[L.oDFP + lane * NWC + w];
+        s *= sf[L.oDF + lane];
+        const size_t o = (bt0 + lane) * N + n;
+        if (a.dgate_part) a.dgate_part[(size_t)rs * BT * N + o] = s;
+        else a.dgate[o] = s;
+      }
+    };
+    for (int j = 0; j < min(2, nch); ++j) fill(j);
+    for (int j = 0; j < nch; ++j) {
+      if (j + 2 < nch) fill(j + 2);
+      if (!mbar_wait(&out_full[j & (kRing - 1)], (j / kRing) & 1)) { report_timeout(a.dev_status); return; }
+      flush(j);
+      __syncwarp();
+    }
+  }
+}
+
+template <int V, int NWC>
+cudaError_t launch_bwd_t(const ScanArgs &a, cudaStream_t s) {
+  const BwdLayout L = bwd_layout<V>(16 * NWC, a.C, V > 64);
+  cudaError_t e = cudaFuncSetAttribute(bwd_bf16_kernel<V, NWC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total);
+  if (e != cudaSuccess) return e;
+  const int RS = a.K / (16 * NWC);
+  bwd_bf16_kernel<V, NWC><<<a.B * a.N * RS, (2 * NWC + V / 16 + 1) * 32, L.total, s>>>(a);
+  return cudaGetLastError();
+}
+
+template <int V>
+cudaError_t launch_bwd_v(const ScanArgs &a, cudaStream_t s) {
+  switch (a.KC) {
+    case 16: return launch_bwd_t<V, 1>(a, s);
+    case 32: return launch_bwd_t<V, 2>(a, s);
+    case 64: return launch_bwd_t<V, 4>(a, s);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+template <int V>
+size_t bwd_smem(int KC, int C) { return bwd_layout<V>(KC, C, V > 64).total; }
+
+}  // namespace
+
+size_t bwd_bf16_smem_bytes(int KC, int V, int C) {
+  switch (V) {
+    case 16: return bwd_smem<16>(KC, C);
+    case 32: return bwd_smem<32>(KC, C);
+    case 64: return bwd_smem<64>(KC, C);
+    default: return bwd_smem<128>(KC, C);
+  }
+}
+
+cudaError_t launch_bwd_bf16(const ScanArgs &a, cudaStream_t s) {
+  switch (a.V) {
+    case 16: return launch_bwd_v<16>(a, s);
+    case 32: return launch_bwd_v<32>(a, s);
+    case 64: return launch_bwd_v<64>(a, s);
+    case 128: return launch_bwd_v<128>(a, s);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+}  // namespace m2rnn
