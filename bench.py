@@ -3,11 +3,13 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
 
-One "step" is one pass of the scan over one batch of synthetic input of the named workload
-(default: the bf16 forward configuration B=8, N=16, K=V=64, T=2048).  Prints ONE JSON line:
-tokens/s with inputs resident in HBM (`value`), the same through host buffers (`e2e`), the
-achieved fraction of the tensor-core roofline for the scan kernel (`roofline`), the CPU oracle
-timed on this host (`cpu_baseline`) and the GPU clocks seen while timing.
+One "step" is one pass of the scan over one batch of synthetic input of the named workload:
+a forward scan (`fwd_bf16`, the default: B=8, N=16, K=V=64, T=2048; also `long_ctx`,
+`paper_layer`, `tiny_f32`), a forward + backward scan (`bptt_bf16`, `sweep16..128`) or one decoding
+step (`decode`).  Prints ONE JSON line: tokens/s with inputs resident in HBM (`value`), the same
+through host buffers (`e2e`), the achieved fraction of the roofline of the dominant call
+(`roofline`), the CPU oracle timed on this host (`cpu_baseline`) and the GPU clocks seen while
+timing.
 
 With N > 1 (torchrun) every rank scans its own batch of the same shape (units are independent:
 no collective on the data path); the value is all ranks' tokens over the slowest rank's time.
@@ -31,6 +33,12 @@ from paper_2603_14360_b200.inputs import CONFIGS  # noqa: E402
 
 METRIC = "m2rnn_scan_tokens_per_s"
 ROTATE = 4  # input sets cycled through so that no step finds its inputs in L2
+PASS_OF = {"fwd_bf16": "fwd", "long_ctx": "fwd", "paper_layer": "fwd", "tiny_f32": "fwd", "decode": "decode"}
+SM_COUNT, SM_HZ = 148, 1.965e9
+
+
+def workload_pass(name: str) -> str:
+    return PASS_OF.get(name, "fwd+bwd")
 
 
 def measured_peaks():
@@ -102,66 +110,111 @@ class ClockSampler:
                 "samples": len(s)}
 
 
-def oracle_sample_rate(cfg, seconds_target=12.0):
+# ------------------------------------------------------------------------------ CPU oracle leg
+def oracle_sample_rate(cfg, pas, seconds_target=12.0):
     """Times the fp64 oracle (one thread) on whole (b,n) units of the workload and scales by the
     exact ratio of units (they are independent).  Returns (tokens/s, description, seconds)."""
     import oracle
     oracle.build()
-    d = inputs.make_inputs(cfg.with_(B=1, N=min(cfg.N, 2), Nq=0, Nk=0))
     f = inputs.to_f64
-    args = [f(d[x]) for x in ("q", "k", "v", "gate", "W", "h0")]
+    nsub = min(cfg.N, 2)
+    small = cfg.with_(B=1, N=nsub, Nq=0, Nk=0)
+    if pas == "decode":
+        d = inputs.make_inputs(small.with_(B=4, T=1))
+        args = [f(d[x][:, 0]) for x in ("q", "k", "v", "gate")] + [f(d["W"]), f(d["h0"])]
+        oracle.decode_step(*args)
+        t0 = time.perf_counter()
+        reps = 0
+        while time.perf_counter() - t0 < min(seconds_target, 5.0):
+            oracle.decode_step(*args)
+            reps += 1
+        dt = time.perf_counter() - t0
+        per_unit = dt / (reps * 4 * nsub)
+        full = per_unit * cfg.B * cfg.N
+        return cfg.B / full, f"{reps} decode steps of {4 * nsub} of {cfg.B * cfg.N} (b,n) units, fp64, 1 thread, scaled by unit count", dt
+    d = inputs.make_inputs(small, backward=(pas == "fwd+bwd"))
+    names = ("q", "k", "v", "gate", "W", "h0") + (("dy",) if pas == "fwd+bwd" else ())
+    args = {x: f(d[x]) for x in names}
+
+    def run(sub):
+        oracle.fwd(sub["q"], sub["k"], sub["v"], sub["gate"], sub["W"], sub["h0"])
+        if pas == "fwd+bwd":
+            oracle.bwd(sub["q"], sub["k"], sub["v"], sub["gate"], sub["W"], sub["h0"], sub["dy"])
+
+    def cut(units, T):
+        out = {}
+        for x, a in args.items():
+            if x == "W":
+                out[x] = a[:units]
+            elif x == "h0":
+                out[x] = None if a is None else a[:, :units]
+            else:
+                out[x] = a[:, :T, :units]
+        return out
+
+    probe_T = min(cfg.T, 64)
     t0 = time.perf_counter()
-    oracle.fwd(*[a[:, :64] if i < 4 else a for i, a in enumerate(args)])
-    per_unit_step = (time.perf_counter() - t0) / (64 * args[2].shape[2])
-    # whole units, full T, as many as fit the budget
-    units = max(1, min(args[2].shape[2], int(seconds_target / (per_unit_step * cfg.T))))
-    sub = [a[:, :, :units] if i < 4 else (a[:units] if i == 4 else (None if a is None else a[:, :units]))
-           for i, a in enumerate(args)]
+    run(cut(nsub, probe_T))
+    per_unit_step = (time.perf_counter() - t0) / (probe_T * nsub)
+    # whole units where a unit fits the budget, else one unit over a prefix of the sequence
+    T_use = cfg.T
+    units = max(1, min(nsub, int(seconds_target / (per_unit_step * cfg.T))))
+    if per_unit_step * cfg.T > 2 * seconds_target:
+        T_use = max(probe_T, int(seconds_target / per_unit_step))
     t0 = time.perf_counter()
-    oracle.fwd(*sub)
+    run(cut(units, T_use))
     dt = time.perf_counter() - t0
-    full_time = dt * (cfg.B * cfg.N) / units
-    return cfg.tokens / full_time, f"{units} of {cfg.B * cfg.N} (b,n) units x T={cfg.T}, fp64, 1 thread, scaled by unit count", dt
+    full_time = dt * (cfg.B * cfg.N) / units * (cfg.T / T_use)
+    what = f"{units} of {cfg.B * cfg.N} (b,n) units x T={T_use}" + ("" if T_use == cfg.T else f" of {cfg.T}")
+    return cfg.tokens / full_time, f"{what}, {pas}, fp64, 1 thread, scaled by unit (and step) count", dt
 
 
-def run_reference(args, cfg):
+def run_reference(args, cfg, pas):
     """The reference arm: the CPU oracle as it stands, on this host's cores."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    if int(os.environ.get("RANK", "0")) != 0:
         return
-    rates, dts = [], []
+    rates = []
+    desc = ""
     for i in range(args.warmup + args.steps):
-        r, desc, dt = oracle_sample_rate(cfg, seconds_target=4.0)
+        r, desc, _ = oracle_sample_rate(cfg, pas, seconds_target=4.0)
         if i >= args.warmup:
-            rates.append(r); dts.append(dt)
+            rates.append(r)
     value = sum(rates) / len(rates)
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * cfg.tokens / value,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfg.name, "B": cfg.B, "T": cfg.T, "N": cfg.N, "K": cfg.K, "V": cfg.V,
-                       "pass": "fwd"},
+            "config": {"workload": cfg.name, "B": cfg.B, "T": cfg.T, "N": cfg.N, "K": cfg.K, "V": cfg.V, "pass": pas},
             "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": 1, "kind": "oracle", "sample": desc},
             "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------------------------------ GPU leg
+def nbytes(t):
+    return 0 if t is None else t.numel() * t.element_size()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=0, help="0: a default per workload")
+    ap.add_argument("--warmup", type=int, default=0)
     ap.add_argument("--workload", default="fwd_bf16", choices=sorted(CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     cfg = CONFIGS[args.workload]
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    pas = workload_pass(args.workload)
 
     if args.impl == "reference":
-        args.steps, args.warmup = min(args.steps, 5), min(args.warmup, 1)
-        run_reference(args, cfg)
+        args.steps, args.warmup = min(args.steps or 3, 5), min(args.warmup or 1, 1)
+        run_reference(args, cfg, pas)
         return
+    if not args.steps:
+        args.steps = {"fwd_bf16": 300, "decode": 1000, "tiny_f32": 300}.get(args.workload, 20)
+    args.warmup = max(args.warmup or (20 if pas != "fwd+bwd" else 3), 3)
 
     from paper_2603_14360_b200 import binding
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -176,22 +229,60 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    # ROTATE seeded input sets per rank, resident in HBM; the same sets pinned on the host for e2e
+    bwd = pas == "fwd+bwd"
+    io = inputs.torch_dtype(cfg.dtype)
+    B, T, N, K, V = cfg.B, cfg.T, cfg.N, cfg.K, cfg.V
+    # ROTATE seeded input sets per rank, resident in HBM; the same sets pinned on the host for e2e.
+    # The decode workload rotates its per-token inputs; its state (2 x 1 GB per step) is far above L2.
     host_sets = []
     for r in range(ROTATE):
-        d = inputs.make_inputs(cfg, seed=cfg.seed + 1000 * rank + 17 * r)
+        d = inputs.make_inputs(cfg, backward=bwd, seed=cfg.seed + 1000 * rank + 17 * r)
+        if pas == "decode":
+            d = {k: (v[:, 0].contiguous() if k in ("q", "k", "v", "gate") else v) for k, v in d.items()}
         host_sets.append({k: (v.pin_memory() if isinstance(v, torch.Tensor) else v) for k, v in d.items()})
     dev_sets = [{k: (v.to(dev) if isinstance(v, torch.Tensor) else v) for k, v in hs.items()} for hs in host_sets]
     W = dev_sets[0]["W"]
-    io = inputs.torch_dtype(cfg.dtype)
-    outs = [dict(y=torch.empty((cfg.B, cfg.T, cfg.N, cfg.V), dtype=io, device=dev),
-                 hT=torch.empty((cfg.B, cfg.N, cfg.K, cfg.V), dtype=torch.float32, device=dev)) for _ in range(ROTATE)]
     stream = torch.cuda.current_stream()
+    launches_per_step = 1
 
-    def step(i):
-        s = dev_sets[i % ROTATE]
-        binding.m2rnn_fwd(s["q"], s["k"], s["v"], s["gate"], W, s["h0"], gate_kind=cfg.gate_kind,
-                          out=outs[i % ROTATE], stream=stream)
+    if pas == "decode":
+        state = dev_sets[0]["h0"].clone()
+        y1 = torch.empty((B, N, V), dtype=io, device=dev)
+
+        def step(i, s=None):
+            s = s or dev_sets[i % ROTATE]
+            binding.m2rnn_decode_step(s["q"], s["k"], s["v"], s["gate"], W, state, gate_kind=cfg.gate_kind, y=y1,
+                                      stream=stream)
+        out_tensors = [y1]
+    else:
+        p = binding._params(dev_sets[0]["q"], dev_sets[0]["k"], dev_sets[0]["v"], W, cfg.gate_kind)
+        outs = dict(y=torch.empty((B, T, N, V), dtype=io, device=dev),
+                    hT=torch.empty((B, N, K, V), dtype=torch.float32, device=dev))
+        out_tensors = list(outs.values())
+        if bwd:
+            C = binding.m2rnn_ckpt_interval(p)
+            outs["ckpt"] = torch.empty((B, N, (T + C - 1) // C, K, V), dtype=torch.float32, device=dev)
+            s0 = dev_sets[0]
+            gouts = dict(dq=torch.empty_like(s0["q"]), dk=torch.empty_like(s0["k"]), dv=torch.empty_like(s0["v"]),
+                         dgate=torch.empty_like(s0["gate"]), dW=torch.empty((N, V, V), dtype=torch.float32, device=dev),
+                         dh0=torch.empty((B, N, K, V), dtype=torch.float32, device=dev))
+            ws = torch.empty(max(1, binding.m2rnn_bwd_workspace_bytes(p, True)), dtype=torch.uint8, device=dev)
+            out_tensors += list(gouts.values())
+            # fwd, bwd, dW reduce (+ dv and dgate reduces when a state's rows are split over CTAs)
+            launches_per_step = 3 + (2 if binding.m2rnn_bwd_row_slab(p) != K else 0)
+        ev_mid = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+
+        def step(i, s=None, mark=False):
+            s = s or dev_sets[i % ROTATE]
+            binding.m2rnn_fwd(s["q"], s["k"], s["v"], s["gate"], W, s["h0"], gate_kind=cfg.gate_kind,
+                              save_ckpt=bwd, out=outs, stream=stream)
+            if bwd:
+                if mark:
+                    ev_mid[0].record(stream)
+                binding.m2rnn_bwd(s["q"], s["k"], s["v"], s["gate"], W, s["h0"], s["dy"], ckpt=outs["ckpt"],
+                                  gate_kind=cfg.gate_kind, workspace=ws, out=gouts, stream=stream)
+                if mark:
+                    ev_mid[1].record(stream)
 
     def barrier():
         torch.cuda.synchronize()
@@ -213,80 +304,109 @@ def main():
         barrier()
     ms_total = ev[0].elapsed_time(ev[1])
     binding.check_device_status()
+    # the backward call alone (its kernels only), for the roofline of the dominant call
+    ms_bwd = 0.0
+    if bwd:
+        reps = min(args.steps, 10)
+        for i in range(reps):
+            step(i, mark=True)
+            torch.cuda.synchronize()
+            ms_bwd += ev_mid[0].elapsed_time(ev_mid[1]) / reps
 
     # end to end: host buffers in, host buffers out, every step
-    host_out = dict(y=torch.empty((cfg.B, cfg.T, cfg.N, cfg.V), dtype=io).pin_memory(),
-                    hT=torch.empty((cfg.B, cfg.N, cfg.K, cfg.V), dtype=torch.float32).pin_memory())
-    stage = {k: torch.empty_like(v) for k, v in dev_sets[0].items() if isinstance(v, torch.Tensor) and k != "W"}
-    h2d = sum(t.numel() * t.element_size() for t in stage.values())
-    d2h = sum(t.numel() * t.element_size() for t in host_out.values())
+    ms_e2e, e2e_steps, h2d, d2h = 0.0, 0, 0, 0
+    if not args.no_e2e:
+        host_out = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in out_tensors if t is not outs.get("ckpt")] \
+            if pas != "decode" else [torch.empty(y1.shape, dtype=y1.dtype).pin_memory()]
+        dev_out = [t for t in out_tensors if pas == "decode" or t is not outs.get("ckpt")]
+        stage = {k: torch.empty_like(v) for k, v in dev_sets[0].items()
+                 if isinstance(v, torch.Tensor) and k != "W" and not (pas == "decode" and k == "h0")}
+        h2d = sum(nbytes(t) for t in stage.values())
+        d2h = sum(nbytes(t) for t in host_out)
 
-    def e2e_step(i):
-        hs = host_sets[i % ROTATE]
-        for k, t in stage.items():
-            t.copy_(hs[k], non_blocking=True)
-        binding.m2rnn_fwd(stage["q"], stage["k"], stage["v"], stage["gate"], W, stage.get("h0"),
-                          gate_kind=cfg.gate_kind, out=outs[0], stream=stream)
-        host_out["y"].copy_(outs[0]["y"], non_blocking=True)
-        host_out["hT"].copy_(outs[0]["hT"], non_blocking=True)
+        def e2e_step(i):
+            hs = host_sets[i % ROTATE]
+            for k, t in stage.items():
+                t.copy_(hs[k], non_blocking=True)
+            step(i, s={**stage, "W": W, "h0": stage.get("h0", dev_sets[0].get("h0"))})
+            for h, d_ in zip(host_out, dev_out):
+                h.copy_(d_, non_blocking=True)
 
-    e2e_steps = max(3, min(args.steps, 50))
-    for i in range(3):
-        e2e_step(i)
-    barrier()
-    ev2 = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
-    ev2[0].record(stream)
-    for i in range(e2e_steps):
-        e2e_step(i)
-    ev2[1].record(stream)
-    barrier()
-    ms_e2e = ev2[0].elapsed_time(ev2[1])
+        e2e_steps = max(3, min(args.steps, 50))
+        for i in range(3):
+            e2e_step(i)
+        barrier()
+        ev2 = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        ev2[0].record(stream)
+        for i in range(e2e_steps):
+            e2e_step(i)
+        ev2[1].record(stream)
+        barrier()
+        ms_e2e = ev2[0].elapsed_time(ev2[1])
 
-    times = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
+    times = torch.tensor([ms_total, ms_e2e, ms_bwd], dtype=torch.float64, device=dev)
     if dist:
         dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e = (float(x) for x in times.tolist())
+    ms_total, ms_e2e, ms_bwd = (float(x) for x in times.tolist())
     if rank != 0:
         if dist:
             dist.destroy_process_group()
         return
 
     ms_step = ms_total / args.steps
-    tokens = cfg.tokens * world
+    tokens = (B if pas == "decode" else cfg.tokens) * world
     value = tokens / (ms_step * 1e-3)
     peaks = measured_peaks()
-    th = cfg.B * cfg.T * cfg.N                                   # token-heads per launch
-    flops = 2.0 * cfg.K * cfg.V * cfg.V * th                     # the state x W contraction
     esz = 2 if cfg.dtype == "bf16" else 4
-    bt = cfg.B * cfg.T
-    stream_bytes = (bt * (cfg.nq + cfg.nk) * cfg.K * esz + 2 * th * cfg.V * esz + th * 4      # q,k | v,y | gate
-                    + 2 * cfg.B * cfg.N * cfg.K * cfg.V * 4)                                   # h0 in, hT out
-    t_tensor = flops / (peaks["tflops_burst"] * 1e12)
-    t_hbm = stream_bytes / (peaks["hbm_gbs"] * 1e9)
-    achieved = flops / (ms_step * 1e-3) / 1e12
-    sm_clock = 1.965e9
-    mufu_s = th * cfg.K * cfg.V / (16 * 148 * sm_clock)          # one tanh per state element per step
+    Tn = 1 if pas == "decode" else T
+    th = B * Tn * N                                              # token-heads per step
+    in_bytes = B * Tn * (cfg.nq + cfg.nk) * K * esz + th * V * esz + th * 4          # q,k | v | gate
+    state_bytes = 2 * B * N * K * V * 4                                                # h0 in, hT out
+    if pas == "decode":
+        # HBM-bound: the fp32 state is read and written once per step
+        alg_bytes = state_bytes + in_bytes + th * V * esz
+        achieved = alg_bytes / (ms_step * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "call": "m2rnn_decode_step",
+                "peak_source": f"{peaks['source']} HBM copy", "algorithmic_bytes_per_step": alg_bytes}
+    else:
+        # the contraction(s): forward 2KV^2 per token-head; backward 6KV^2 (recompute, dX W^T, H^T dX)
+        call_ms = ms_bwd if bwd else ms_step
+        flops = (6.0 if bwd else 2.0) * K * V * V * th
+        alg_bytes = in_bytes + th * V * esz + state_bytes
+        if bwd:  # + dy in, dq dk dv dgate out, dh0 out (checkpoints are not algorithmic)
+            alg_bytes = 2 * in_bytes + th * V * esz + state_bytes
+        achieved = flops / (call_ms * 1e-3) / 1e12
+        t_tensor, t_hbm = flops / (peaks["tflops_burst"] * 1e12), alg_bytes / (peaks["hbm_gbs"] * 1e9)
+        passes = 2 if bwd else 1                                 # tanh per state element: recompute counts once more
+        mufu_s = th * K * V / (16 * SM_COUNT * SM_HZ)
+        roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["tflops_burst"], "unit": "TFLOP/s",
+                "frac": achieved / peaks["tflops_burst"], "traffic": None,
+                "call": "m2rnn_bwd" if bwd else "m2rnn_fwd", "call_ms": call_ms,
+                "peak_source": f"{peaks['source']} cuBLAS bf16 burst",
+                "t_tensor_ms": t_tensor * 1e3, "t_hbm_ms": t_hbm * 1e3, "t_mufu_ms": mufu_s * 1e3,
+                "frac_of_mufu_ceiling": mufu_s / (call_ms * 1e-3),
+                "ns_per_scan_step": call_ms * 1e6 / T / passes}
     line = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-        "config": {"workload": cfg.name, "pass": "fwd", "B": cfg.B, "T": cfg.T, "N": cfg.N, "K": cfg.K, "V": cfg.V,
+        "config": {"workload": cfg.name, "pass": pas, "B": B, "T": Tn, "N": N, "K": K, "V": V,
                    "Nq": cfg.nq, "Nk": cfg.nk, "gate": "logit", "state": "fp32", "accumulate": "fp32",
-                   "per_gpu_batch": cfg.B,
-                   "l2": f"{ROTATE} input/output sets cycled ({ROTATE} x {int((h2d + d2h) / 1e6)} MB > 126 MB L2)"},
-        "roofline": {"bound": "tensor", "achieved": achieved, "peak": peaks["tflops_burst"], "unit": "TFLOP/s",
-                     "frac": achieved / peaks["tflops_burst"], "traffic": None,
-                     "peak_source": f"{peaks['source']} cuBLAS bf16 burst",
-                     "t_tensor_ms": t_tensor * 1e3, "t_hbm_ms": t_hbm * 1e3,
-                     "t_mufu_ms": mufu_s * 1e3, "frac_of_mufu_ceiling": mufu_s / (ms_step * 1e-3),
-                     "ns_per_scan_step": ms_step * 1e6 / cfg.T},
-        "e2e": {"value": tokens / (ms_e2e / e2e_steps * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "steps": e2e_steps},
-        "gpu_launches": args.steps,
+                   "per_gpu_batch": B,
+                   "l2": f"{ROTATE} input sets cycled; bytes touched per step {int((alg_bytes) / 1e6)} MB"
+                         f" x {ROTATE} sets vs 126 MB L2"},
+        "roofline": roof,
+        "gpu_launches": args.steps * launches_per_step,
         "clocks": clocks.summary(),
     }
+    if bwd:
+        line["ms_fwd"], line["ms_bwd"] = ms_step - ms_bwd, ms_bwd
+    if not args.no_e2e:
+        line["e2e"] = {"value": tokens / (ms_e2e / e2e_steps * 1e-3), "unit": "tokens/s",
+                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
     if not args.no_cpu_baseline:
-        rate, desc, dt = oracle_sample_rate(cfg)
+        rate, desc, dt = oracle_sample_rate(cfg, pas)
         line["cpu_baseline"] = {"value": rate, "unit": "tokens/s", "cores": 1, "kind": "oracle", "sample": desc,
                                 "seconds": dt}
     print(json.dumps(line), flush=True)

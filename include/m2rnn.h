@@ -87,6 +87,12 @@ const char *m2rnn_status_string(int status);
  * recomputes C states at a time from a checkpoint, so C is bounded by on-chip memory. */
 int m2rnn_ckpt_interval(const m2rnn_params *params);
 
+/* Rows of a state that one CTA of the backward kernel takes for `params` (a divisor of K); <= 0
+ * is an m2rnn_status.  The K rows of a state are independent recurrences (Eq. 1-2 act row by row),
+ * so the backward pass may split them over K/rows CTAs; when it does, dv and dgate (sums over all
+ * rows) are finished by two extra reduction launches. */
+int m2rnn_bwd_row_slab(const m2rnn_params *params);
+
 /* Bytes of the checkpoint tensor [B,N,ceil(T/C),K,V] (fp32). */
 size_t m2rnn_ckpt_bytes(const m2rnn_params *params);
 

@@ -51,6 +51,7 @@ EXPORTS = {
     "m2rnn_version": (ctypes.c_int, []),
     "m2rnn_status_string": (ctypes.c_char_p, [ctypes.c_int]),
     "m2rnn_ckpt_interval": (ctypes.c_int, [_pp]),
+    "m2rnn_bwd_row_slab": (ctypes.c_int, [_pp]),
     "m2rnn_ckpt_bytes": (ctypes.c_size_t, [_pp]),
     "m2rnn_fwd": (ctypes.c_int, [_pp] + [_vp] * 14),
     "m2rnn_bwd_workspace_bytes": (ctypes.c_size_t, [_pp, ctypes.c_int]),
@@ -145,6 +146,13 @@ def m2rnn_ckpt_interval(p: Params) -> int:
     if c <= 0:
         raise M2RNNError(c, "m2rnn_ckpt_interval")
     return c
+
+
+def m2rnn_bwd_row_slab(p: Params) -> int:
+    r = _lib().m2rnn_bwd_row_slab(ctypes.byref(p))
+    if r <= 0:
+        raise M2RNNError(r, "m2rnn_bwd_row_slab")
+    return r
 
 
 def m2rnn_bwd_workspace_bytes(p: Params, have_ckpt: bool) -> int:

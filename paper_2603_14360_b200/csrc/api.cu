@@ -126,6 +126,12 @@ int m2rnn_ckpt_interval(const m2rnn_params *params) {
   return interval_of(params);
 }
 
+int m2rnn_bwd_row_slab(const m2rnn_params *params) {
+  int rc = check_params(params, false);
+  if (rc != M2RNN_OK) return rc;
+  return plan_bwd(params->B, params->N, params->K, params->V, params->io_dtype).KC;
+}
+
 size_t m2rnn_ckpt_bytes(const m2rnn_params *params) {
   if (check_params(params, true) != M2RNN_OK || params->T == 0) return 0;
   const int C = interval_of(params);
