@@ -43,6 +43,11 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, 1) fwd_bf16_kernel(ScanArgs a
   using G = TileGeom<V>;
   constexpr int NT = G::NT, KT = G::KT, SEG = G::SEG;
   constexpr bool kWInRegs = V <= 64;
+  // The product of a step is split over NSET accumulator sets (k-tile kt adds into set kt % NSET,
+  // the sets are summed where they are used): an mma.sync that accumulates onto the previous
+  // one's result waits for its whole latency (well over 100 cycles), so KT of them in a row
+  // would be most of the step.
+  constexpr int NSET = V == 128 ? 1 : (KT >= 2 ? 2 : 1);
   extern __shared__ __align__(16) unsigned char smem_raw[];
 
   const int K = a.K, N = a.N, T = a.T;
@@ -209,24 +214,27 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, 1) fwd_bf16_kernel(ScanArgs a
 
   // P <- k v^T  (the outer-product term of Eq. 1 seeds the accumulators)
   // (shared-memory operands of the hot loop are 32-bit shared addresses, in bytes)
-  auto seed = [&](float (&P)[NT][4], uint32_t krow, uint32_t vrow) {
+  auto seed = [&](float (&P)[NSET][NT][4], uint32_t krow, uint32_t vrow) {
     const float2 kk = lds64(krow + 4 * row0);
 #pragma unroll
     for (int x = 0; x < SEG / 4; ++x) {
       const float4 v4 = lds128(vrow + 4 * (SEG * c + 4 * x));
-      P[2 * x][0] = kk.x * v4.x; P[2 * x][1] = kk.x * v4.y; P[2 * x][2] = kk.y * v4.x; P[2 * x][3] = kk.y * v4.y;
-      P[2 * x + 1][0] = kk.x * v4.z; P[2 * x + 1][1] = kk.x * v4.w; P[2 * x + 1][2] = kk.y * v4.z; P[2 * x + 1][3] = kk.y * v4.w;
+      P[0][2 * x][0] = kk.x * v4.x; P[0][2 * x][1] = kk.x * v4.y; P[0][2 * x][2] = kk.y * v4.x; P[0][2 * x][3] = kk.y * v4.y;
+      P[0][2 * x + 1][0] = kk.x * v4.z; P[0][2 * x + 1][1] = kk.x * v4.w; P[0][2 * x + 1][2] = kk.y * v4.z; P[0][2 * x + 1][3] = kk.y * v4.w;
     }
   };
   // P += A[kt] * W[kt][:]  : one k tile of H W
-  auto mma_ktile = [&](float (&P)[NT][4], const uint32_t (&Ak)[4], int kt) {
+  auto mma_ktile = [&](float (&P)[NSET][NT][4], const uint32_t (&Ak)[4], int kt) {
+    const int set = kt % NSET;
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
       if constexpr (kWInRegs) {
-        mma_bf16_16816(P[nt], Ak, Wr[kt][nt][0], Wr[kt][nt][1]);
+        if (kt >= 1 && kt < NSET) mma_bf16_16816_zero(P[set][nt], Ak, Wr[kt][nt][0], Wr[kt][nt][1]);
+        else mma_bf16_16816(P[set][nt], Ak, Wr[kt][nt][0], Wr[kt][nt][1]);
       } else {
         const uint2 w = Wf[(kt * NT + nt) * 32 + lane];
-        mma_bf16_16816(P[nt], Ak, w.x, w.y);
+        if (kt >= 1 && kt < NSET) mma_bf16_16816_zero(P[set][nt], Ak, w.x, w.y);
+        else mma_bf16_16816(P[set][nt], Ak, w.x, w.y);
       }
     }
   };
@@ -238,7 +246,7 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, 1) fwd_bf16_kernel(ScanArgs a
   //   Pc: H_{t-1} W + k_t v_t^T, complete (or in flight) on entry
   //   Pn: receives H_t W + k_{t+1} v_{t+1}^T; after the last step it is fed a valid but
   //       meaningless row and its result is never read
-  auto step = [&](float (&Pc)[NT][4], float (&Pn)[NT][4], float f, uint32_t qrow, uint32_t ydst,
+  auto step = [&](float (&Pc)[NSET][NT][4], float (&Pn)[NSET][NT][4], float f, uint32_t qrow, uint32_t ydst,
                   uint32_t krow_n, uint32_t vrow_n) {
     seed(Pn, krow_n, vrow_n);
     const float2 qq = lds64(qrow + 4 * row0);
@@ -249,7 +257,9 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, 1) fwd_bf16_kernel(ScanArgs a
       for (int nt = 2 * kt; nt < 2 * kt + 2; ++nt) {
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
-          const float z = tanh_approx(Pc[nt][r]);          // Eq. 1
+          float x = Pc[0][nt][r];
+          if constexpr (NSET == 2) x += Pc[1][nt][r];
+          const float z = tanh_approx(x);                  // Eq. 1
           H[nt][r] = fmaf(f, H[nt][r] - z, z);             // Eq. 2: f H + (1-f) Z
         }
         part[2 * nt] = fmaf(qq.y, H[nt][2], qq.x * H[nt][0]);      // Eq. 3, this thread's two rows
@@ -272,7 +282,7 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, 1) fwd_bf16_kernel(ScanArgs a
     }
   };
 
-  float P0[NT][4], P1[NT][4];
+  float P0[NSET][NT][4], P1[NSET][NT][4];
   int ck_left = 0, ck_idx = 0;  // steps until the next checkpoint, index of the next checkpoint
   auto maybe_checkpoint = [&](int steps) {   // called before an even-numbered step
     if (a.ckpt) {
