@@ -204,8 +204,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--seq-len", type=int, default=0,
+                    help="shorten (or lengthen) the workload's T, for profiler captures; the line's workload name says so")
     args = ap.parse_args()
     cfg = CONFIGS[args.workload]
+    if args.seq_len and args.workload != "decode":
+        cfg = cfg.with_(T=args.seq_len, name=f"{cfg.name}@T={args.seq_len}")
     pas = workload_pass(args.workload)
 
     if args.impl == "reference":

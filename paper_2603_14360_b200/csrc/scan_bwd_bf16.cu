@@ -79,6 +79,17 @@ __device__ __forceinline__ void load_wt_fragment(const __nv_bfloat16 *__restrict
   b1 = (uint32_t)w[l * V + j2] | ((uint32_t)w[l * V + j3] << 16);
 }
 
+// Register re-balancing between warpgroups (4 aligned warps): the kernel is compiled for an even
+// split (128 per thread here), then the chain warps take registers that the dW and service warps
+// give up.  An increase waits until the CTA's own pool holds enough released registers, so the
+// increases must not ask for more than the decreases release:
+//   +40*128 (recompute) + 80*128 (reverse) = 15360  <=  56*128 (dW) + 72*128 (service group) = 16384.
+// The instruction is warpgroup-wide, so only complete warpgroups may execute it: where it is used
+// the CTA is padded to 16 warps, and the three spare warps join the service warp's decrease and
+// leave.
+template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+
 struct BwdLayout {
   // all byte offsets from the start of dynamic shared memory
   uint32_t wf, wtf, state, state_stride, ztile, dx, ring, slot_bytes, total;
@@ -113,11 +124,16 @@ __host__ __device__ inline BwdLayout bwd_layout(int KC, int C, bool w_in_smem) {
 }
 
 template <int V, int NWC>
-__global__ void __launch_bounds__((2 * NWC + V / 16 + 1) * 32, 1) bwd_bf16_kernel(ScanArgs a) {
+constexpr int bwd_threads() { return (NWC == 4 && V == 64) ? 512 : (2 * NWC + V / 16 + 1) * 32; }
+
+template <int V, int NWC>
+__global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(ScanArgs a) {
   using G = TileGeom<V>;
   constexpr int NT = G::NT, KT = G::KT, SEG = G::SEG;
   constexpr int KC = 16 * NWC, NDW = V / 16;
   constexpr bool kWInSmem = V > 64;
+  // roles coincide with warpgroups only in this shape (4 + 4 + 4 + 1 warps), the one that needs it
+  constexpr bool kRebalance = NWC == 4 && V == 64;
   constexpr int CPR = SEG * 2 / 16;            // 16-byte chunks per thread-row of a tile (0 when V == 16)
   extern __shared__ __align__(128) unsigned char smem[];
 
@@ -209,6 +225,7 @@ __global__ void __launch_bounds__((2 * NWC + V / 16 + 1) * 32, 1) bwd_bf16_kerne
 
   if (warp < NWC) {
     // ================================================================= recompute warps
+    if constexpr (kRebalance) reg_inc<168>();
     const int w = warp, r0 = 16 * w + g;
     uint32_t Wr[kWInSmem ? 1 : KT][kWInSmem ? 1 : NT][2];
     if constexpr (!kWInSmem) {
@@ -286,6 +303,7 @@ __global__ void __launch_bounds__((2 * NWC + V / 16 + 1) * 32, 1) bwd_bf16_kerne
 
   if (warp < 2 * NWC) {
     // ================================================================= reverse warps
+    if constexpr (kRebalance) reg_inc<208>();
     const int w = warp - NWC, r0 = 16 * w + g;
     uint32_t WTr[kWInSmem ? 1 : KT][kWInSmem ? 1 : NT][2];
     if constexpr (!kWInSmem) {
@@ -428,6 +446,7 @@ __global__ void __launch_bounds__((2 * NWC + V / 16 + 1) * 32, 1) bwd_bf16_kerne
   if (warp < 2 * NWC + NDW) {
     // ================================================================= dW warps
     // warp d owns dW rows l in [16d, 16d+16): acc += H_{t-1}[:, l]^T dX, contraction over the CTA's rows
+    if constexpr (kRebalance) reg_dec<72>();
     const int d = warp - 2 * NWC;
     float acc[NT][4];
 #pragma unroll
@@ -471,6 +490,10 @@ __global__ void __launch_bounds__((2 * NWC + V / 16 + 1) * 32, 1) bwd_bf16_kerne
   }
 
   // =================================================================== service warp
+  if constexpr (kRebalance) {
+    reg_dec<56>();
+    if (warp > 2 * NWC + NDW) return;   // spare warps of the padded CTA
+  }
   {
     const int hq = n / (N / a.Nq), hk = n / (N / a.Nk);
     const float al = a.alpha ? a.alpha[n] : 1.f, be = a.beta ? a.beta[n] : 0.f;
@@ -556,7 +579,7 @@ cudaError_t launch_bwd_t(const ScanArgs &a, cudaStream_t s) {
   cudaError_t e = cudaFuncSetAttribute(bwd_bf16_kernel<V, NWC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.total);
   if (e != cudaSuccess) return e;
   const int RS = a.K / (16 * NWC);
-  bwd_bf16_kernel<V, NWC><<<a.B * a.N * RS, (2 * NWC + V / 16 + 1) * 32, L.total, s>>>(a);
+  bwd_bf16_kernel<V, NWC><<<a.B * a.N * RS, bwd_threads<V, NWC>(), L.total, s>>>(a);
   return cudaGetLastError();
 }
 
