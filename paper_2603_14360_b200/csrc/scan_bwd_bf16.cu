@@ -8,11 +8,14 @@
 //                          (Eq. 1-2, the same arithmetic as the forward kernel), leaving for every
 //                          step H_{t-1} as a bf16 row-major tile and Z_t as fp16 fragments;
 //   reverse warps   (NWC)  carry C = dL/dH in registers and walk the chunk backwards:
-//                          G = C + q dy^T, dq, df, dX = (1-f) G (1 - Z^2), dk, dv,
+//                          G = C + q dy^T, df, dX = (1-f) G (1 - Z^2),
 //                          C <- f G + dX W^T  (mma.sync, bf16 operands, fp32 accumulate);
-//                          dX is also left as a bf16 row-major tile;
+//                          dq = H_t dy and dk = dX v are small MMAs on fragments that are in
+//                          registers anyway (H_t is the H_{t-1} tile of the step handled just
+//                          before); dX is also left as a bf16 row-major tile;
 //   dW warps        (V/16) accumulate dW += H_{t-1}^T dX on tensor cores from the two tiles
-//                          (ldmatrix.trans operands), one 16-row slab of dW per warp, off the chain;
+//                          (ldmatrix.trans operands), one 16-row slab of dW per warp, off the chain,
+//                          and take dv = dX^T k along as one more row of the same product;
 //   service warp    (1)    stages q, k, v, dy and the gate for coming chunks, and reduces and writes
 //                          dq, dk, dv, dgate of finished ones.
 //
@@ -92,9 +95,10 @@ template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setma
 
 struct BwdLayout {
   // all byte offsets from the start of dynamic shared memory
-  uint32_t wf, wtf, state, state_stride, ztile, dx, ring, slot_bytes, total;
-  // float offsets inside a ring slot
-  uint32_t oQ, oK, oV, oDY, oF, oDF, oDQ, oDK, oDVP, oDFP;
+  uint32_t wf, wtf, state, state_stride, ztile, dx, hfin, ring, slot_bytes, total;
+  // word offsets inside a ring slot.  In: q, k, v, dy as fp32, f and df/dgate, and k, v, dy once
+  // more as the raw bf16 pairs that serve as MMA operands.  Out: dq, dk, dv, per-lane df partials.
+  uint32_t oQ, oK, oV, oDY, oF, oDF, oKB, oVB, oDYB, oDQ, oDK, oDV, oDFP;
 };
 
 template <int V>
@@ -112,11 +116,15 @@ __host__ __device__ inline BwdLayout bwd_layout(int KC, int C, bool w_in_smem) {
   off += 2u * C * L.state_stride;
   L.dx = off;                                  // [2] dX tiles (bf16)
   off += 2u * KC * V * 2;
+  L.hfin = off;                                // H after the last step, as a tile (dq of step T-1)
+  off += (uint32_t)KC * V * 2;
   L.ring = off;
+  const uint32_t Cp = (uint32_t)((C + 3) & ~3);  // keeps every array of a slot 16-byte aligned
   L.oQ = 0; L.oK = L.oQ + C * KC; L.oV = L.oK + C * KC; L.oDY = L.oV + C * V; L.oF = L.oDY + C * V;
-  L.oDF = L.oF + C; L.oDQ = L.oDF + C; L.oDK = L.oDQ + C * KC; L.oDVP = L.oDK + C * KC;
-  L.oDFP = L.oDVP + C * NWC * V;
-  L.slot_bytes = (L.oDFP + C * NWC) * 4;
+  L.oDF = L.oF + Cp; L.oKB = L.oDF + Cp; L.oVB = L.oKB + C * KC / 2; L.oDYB = L.oVB + C * V / 2;
+  L.oDQ = L.oDYB + C * V / 2; L.oDK = L.oDQ + C * KC; L.oDV = L.oDK + C * KC;
+  L.oDFP = L.oDV + C * V;
+  L.slot_bytes = (L.oDFP + C * NWC * 32) * 4;
   L.slot_bytes = (L.slot_bytes + 15u) & ~15u;
   off += kRing * L.slot_bytes;
   L.total = off;
@@ -155,7 +163,7 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
   uint64_t *dx_full = st_free + 2;            // [2]
   uint64_t *dx_free = dx_full + 2;            // [2]
   if (tid == 0) {
-    for (int s = 0; s < kRing; ++s) { mbar_init(&in_full[s], 1); mbar_init(&out_full[s], NWC); }
+    for (int s = 0; s < kRing; ++s) { mbar_init(&in_full[s], 1); mbar_init(&out_full[s], NWC + NDW); }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&st_ready[s], NWC); mbar_init(&st_free[s], NWC + NDW);
       mbar_init(&dx_full[s], NWC); mbar_init(&dx_free[s], NDW);
@@ -220,8 +228,10 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
       }
     }
   };
-  // Z fragments: private to the (warp, lane) pair that wrote them, 2*NT words per thread
-  auto zfrag_sa = [&](uint32_t step_sa, int w) { return step_sa + L.ztile + (uint32_t)(w * (2 * NT) * 32 + lane) * 4u; };
+  // Z fragments: private to the (warp, lane) pair that wrote them, 2*NT words per thread kept as
+  // NT/2 groups of 16 bytes (group x of lane l at word ((w*NT/2 + x)*32 + l)*4)
+  constexpr int ZG = NT / 2;
+  auto zfrag_sa = [&](uint32_t step_sa, int w) { return step_sa + L.ztile + (uint32_t)(w * ZG * 32 + lane) * 16u; };
 
   if (warp < NWC) {
     // ================================================================= recompute warps
@@ -284,16 +294,28 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
         // Z = tanh(P), kept as fp16 for the reverse sweep; H <- f H + (1-f) Z  (Eq. 2)
         const uint32_t zs = zfrag_sa(st, w);
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          float z[4];
+        for (int x = 0; x < ZG; ++x) {
+          uint32_t zw[4];
 #pragma unroll
-          for (int r = 0; r < 4; ++r) {
-            z[r] = tanh_approx(P[nt][r]);
-            H[nt][r] = fmaf(f, H[nt][r] - z[r], z[r]);
+          for (int u = 0; u < 2; ++u) {
+            const int nt = 2 * x + u;
+            float z[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+              z[r] = tanh_approx(P[nt][r]);
+              H[nt][r] = fmaf(f, H[nt][r] - z[r], z[r]);
+            }
+            zw[2 * u] = pack_f16(z[0], z[1]);
+            zw[2 * u + 1] = pack_f16(z[2], z[3]);
           }
-          asm volatile("st.shared.b32 [%0], %1;" ::"r"(zs + 4u * (2 * nt) * 32), "r"(pack_f16(z[0], z[1])) : "memory");
-          asm volatile("st.shared.b32 [%0], %1;" ::"r"(zs + 4u * (2 * nt + 1) * 32), "r"(pack_f16(z[2], z[3])) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(zs + 512u * x), "r"(zw[0]), "r"(zw[1]), "r"(zw[2]), "r"(zw[3]) : "memory");
         }
+      }
+      if (j == 0) {   // the state after the last step of the scan: H_t of the first reverse step
+        uint32_t hp[NT][2];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) { hp[nt][0] = pack_bf16(H[nt][0], H[nt][1]); hp[nt][1] = pack_bf16(H[nt][2], H[nt][3]); }
+        tile_store(sm0 + L.hfin, w, hp);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&st_ready[j & 1]);
@@ -329,10 +351,37 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
     }
     const float clip = a.dh_clip;
     int nstep = 0;   // steps taken so far: picks the dX tile
+    // B operand of the small MMAs: the thread's SEG columns of a vector as bf16 pairs; every
+    // column n of B holds the same vector, so every column of the result holds the product
+    auto load_pairs = [&](uint32_t row_sa, uint32_t (&pr)[NT]) {
+      if constexpr (NT == 2) {
+        asm volatile("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(pr[0]), "=r"(pr[1]) : "r"(row_sa + 4u * (SEG / 2) * c));
+      } else {
+#pragma unroll
+        for (int x = 0; x < NT / 4; ++x)
+          asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];"
+                       : "=r"(pr[4 * x]), "=r"(pr[4 * x + 1]), "=r"(pr[4 * x + 2]), "=r"(pr[4 * x + 3])
+                       : "r"(row_sa + 4u * ((SEG / 2) * c + 4 * x)));
+      }
+    };
+    // (A . vec), A given as packed pairs in accumulator layout: rows g and g+8 end up in
+    // d[.][0] and d[.][2], split over two accumulators that the caller adds when it stores them
+    // (late in the step, so that the warp never waits on these off-chain products)
+    auto matvec = [&](const uint32_t (&Ap)[NT][2], const uint32_t (&pr)[NT], float (&d)[2][4]) {
+#pragma unroll
+      for (int kt = 0; kt < KT; ++kt) {
+        const uint32_t Ak[4] = {Ap[2 * kt][0], Ap[2 * kt][1], Ap[2 * kt + 1][0], Ap[2 * kt + 1][1]};
+        if (kt < 2) mma_bf16_16816_zero(d[kt & 1], Ak, pr[2 * kt], pr[2 * kt + 1]);
+        else mma_bf16_16816(d[kt & 1], Ak, pr[2 * kt], pr[2 * kt + 1]);
+      }
+      if constexpr (KT == 1) d[1][0] = d[1][2] = 0.f;
+    };
+    uint32_t hn[NT][2];   // H_t of the step at hand as bf16 pairs = the H_{t-1} tile of the step done before
     for (int j = 0; j < nch; ++j) {
       const int len = chunk_len(j);
       if (!mbar_wait(&in_full[j & (kRing - 1)], (j / kRing) & 1)) { report_timeout(a.dev_status); return; }
       if (!mbar_wait(&st_ready[j & 1], (j >> 1) & 1)) { report_timeout(a.dev_status); return; }
+      if (j == 0) tile_load(sm0 + L.hfin, w, hn);
       const uint32_t sl = slot_sa(j);
       for (int s = len - 1; s >= 0; --s, ++nstep) {
         const uint32_t st = state_sa(j, s);
@@ -341,41 +390,38 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
         const uint32_t zs = zfrag_sa(st, w);
         const float f = lds32(sl + 4u * (L.oF + s));
         const float q0 = lds32(sl + 4u * (L.oQ + s * KC + r0)), q1 = lds32(sl + 4u * (L.oQ + s * KC + r0 + 8));
-        const float k0 = lds32(sl + 4u * (L.oK + s * KC + r0)), k1 = lds32(sl + 4u * (L.oK + s * KC + r0 + 8));
         const float omf = 1.f - f;
-        float dq0 = 0.f, dq1 = 0.f, dk0 = 0.f, dk1 = 0.f, df = 0.f;
-        float dvp[SEG];
+        // dq = H_t dy on the tensor cores (Algorithm 2, "dq <- H . dy")
+        float dqd[2][4], dkd[2][4];
+        {
+          uint32_t dyp[NT];
+          load_pairs(sl + 4u * (L.oDYB + s * (V / 2)), dyp);
+          matvec(hn, dyp, dqd);
+        }
+        float df = 0.f;
         uint32_t xp[NT][2];   // dX as bf16 pairs: the A operand of dX W^T and the tile of the dW warps
 #pragma unroll
         for (int x = 0; x < SEG / 4; ++x) {
           const float4 dy4 = lds128(sl + 4u * (L.oDY + s * V + SEG * c + 4 * x));
-          const float4 v4 = lds128(sl + 4u * (L.oV + s * V + SEG * c + 4 * x));
-          const float dyv[4] = {dy4.x, dy4.y, dy4.z, dy4.w}, vv[4] = {v4.x, v4.y, v4.z, v4.w};
+          const float dyv[4] = {dy4.x, dy4.y, dy4.z, dy4.w};
+          uint32_t zw[4];
+          asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(zw[0]), "=r"(zw[1]), "=r"(zw[2]), "=r"(zw[3]) : "r"(zs + 512u * x));
 #pragma unroll
           for (int u = 0; u < 2; ++u) {
             const int nt = 2 * x + u;
-            uint32_t zw0, zw1;
-            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(zw0) : "r"(zs + 4u * (2 * nt) * 32));
-            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(zw1) : "r"(zs + 4u * (2 * nt + 1) * 32));
-            const float2 za = unpack_f16(zw0), zb = unpack_f16(zw1);
+            const float2 za = unpack_f16(zw[2 * u]), zb = unpack_f16(zw[2 * u + 1]);
             const float2 ha = unpack_bf16(hp[nt][0]), hb = unpack_bf16(hp[nt][1]);
             const float z[4] = {za.x, za.y, zb.x, zb.y}, hprev[4] = {ha.x, ha.y, hb.x, hb.y};
             float dX[4];
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
-              const float dyc = dyv[2 * u + (r & 1)], vc = vv[2 * u + (r & 1)];
+              const float dyc = dyv[2 * u + (r & 1)];
               const float qr = (r & 2) ? q1 : q0;
               const float Gv = fmaf(qr, dyc, Cg[nt][r]);        // G = C + q dy^T
-              const float D = hprev[r] - z[r];                  // H_{t-1} - Z
-              const float ht = fmaf(f, D, z[r]);                // H_t
-              if (r & 2) dq1 = fmaf(ht, dyc, dq1); else dq0 = fmaf(ht, dyc, dq0);   // dq = H_t dy
-              df = fmaf(Gv, D, df);                             // df = sum G (.) (H_{t-1} - Z)
+              df = fmaf(Gv, hprev[r] - z[r], df);               // df = sum G (.) (H_{t-1} - Z)
               dX[r] = omf * Gv * fmaf(-z[r], z[r], 1.f);        // through the gate and tanh
-              if (r & 2) dk1 = fmaf(dX[r], vc, dk1); else dk0 = fmaf(dX[r], vc, dk0);  // dk = dX v
               Cg[nt][r] = f * Gv;                               // gated path into H_{t-1}
             }
-            dvp[4 * x + 2 * u] = fmaf(dX[2], k1, dX[0] * k0);   // dv = dX^T k, this thread's two rows
-            dvp[4 * x + 2 * u + 1] = fmaf(dX[3], k1, dX[1] * k0);
             xp[nt][0] = pack_bf16(dX[0], dX[1]);
             xp[nt][1] = pack_bf16(dX[2], dX[3]);
           }
@@ -400,32 +446,25 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
             }
           }
         }
+        // dk = dX v on the tensor cores (Algorithm 2, "dk <- dX . v")
+        {
+          uint32_t vp[NT];
+          load_pairs(sl + 4u * (L.oVB + s * (V / 2)), vp);
+          matvec(xp, vp, dkd);
+        }
         if (clip > 0.f) {
 #pragma unroll
           for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
             for (int r = 0; r < 4; ++r) Cg[nt][r] = fminf(fmaxf(Cg[nt][r], -clip), clip);
         }
-        // row sums over the 4 lanes of a row group, column sums over the 8 row groups
-        dq0 += __shfl_xor_sync(0xffffffffu, dq0, 1); dq1 += __shfl_xor_sync(0xffffffffu, dq1, 1);
-        dk0 += __shfl_xor_sync(0xffffffffu, dk0, 1); dk1 += __shfl_xor_sync(0xffffffffu, dk1, 1);
-        dq0 += __shfl_xor_sync(0xffffffffu, dq0, 2); dq1 += __shfl_xor_sync(0xffffffffu, dq1, 2);
-        dk0 += __shfl_xor_sync(0xffffffffu, dk0, 2); dk1 += __shfl_xor_sync(0xffffffffu, dk1, 2);
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) df += __shfl_xor_sync(0xffffffffu, df, off);
+        sts32(sl + 4u * (L.oDFP + (s * NWC + w) * 32 + lane), df);   // summed by the service warp
         if (c == 0) {
-          sts32(sl + 4u * (L.oDQ + s * KC + r0), dq0); sts32(sl + 4u * (L.oDQ + s * KC + r0 + 8), dq1);
-          sts32(sl + 4u * (L.oDK + s * KC + r0), dk0); sts32(sl + 4u * (L.oDK + s * KC + r0 + 8), dk1);
+          sts32(sl + 4u * (L.oDQ + s * KC + r0), dqd[0][0] + dqd[1][0]); sts32(sl + 4u * (L.oDQ + s * KC + r0 + 8), dqd[0][2] + dqd[1][2]);
+          sts32(sl + 4u * (L.oDK + s * KC + r0), dkd[0][0] + dkd[1][0]); sts32(sl + 4u * (L.oDK + s * KC + r0 + 8), dkd[0][2] + dkd[1][2]);
         }
-        if (lane == 0) sts32(sl + 4u * (L.oDFP + s * NWC + w), df);
-        reduce_over_rows<SEG>(dvp, lane);
-        using RO = RowReduceOut<V>;
-        if (RO::owner(lane)) {
-          const uint32_t dst = sl + 4u * (L.oDVP + (s * NWC + w) * V + RO::first_col(lane));
-          if constexpr (RO::CNT == 4) sts128(dst, make_float4(dvp[0], dvp[1], dvp[2], dvp[3]));
-          else if constexpr (RO::CNT == 2) sts64(dst, make_float2(dvp[0], dvp[1]));
-          else sts32(dst, dvp[0]);
-        }
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) { hn[nt][0] = hp[nt][0]; hn[nt][1] = hp[nt][1]; }
       }
       __syncwarp();
       if (lane == 0) { mbar_arrive(&st_free[j & 1]); mbar_arrive(&out_full[j & (kRing - 1)]); }
@@ -460,6 +499,12 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
         const int xb = nstep & 1;
         if (!mbar_wait(&dx_full[xb], (nstep >> 1) & 1)) { report_timeout(a.dev_status); return; }
         const uint32_t ht = state_sa(j, s), xt = sm0 + L.dx + (uint32_t)xb * (KC * V * 2);
+        // dv = dX^T k (Algorithm 2, "dv <- dX^T . k") rides along as one more row of the product:
+        // an A tile whose row 0 is k and whose other rows are zero; this warp takes columns 16d..16d+15
+        float dvacc[2][4];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) dvacc[u][0] = dvacc[u][1] = dvacc[u][2] = dvacc[u][3] = 0.f;
+        const uint32_t kb = slot_sa(j) + 4u * (L.oKB + s * (KC / 2));
 #pragma unroll
         for (int kt = 0; kt < NWC; ++kt) {
           // A = H_{t-1}^T: matrices (i 0-7, l 0-7), (i 0-7, l 8-15), (i 8-15, l 0-7), (i 8-15, l 8-15)
@@ -474,11 +519,27 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
             mma_bf16_16816(acc[2 * np + 1], A, b2, b3);
           }
         }
+#pragma unroll
+        for (int kt = 0; kt < NWC; ++kt) {
+          uint32_t Ak[4] = {0u, 0u, 0u, 0u}, b0, b1, b2, b3;
+          if (g == 0) {
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(Ak[0]) : "r"(kb + 4u * (8 * kt + c)));
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(Ak[2]) : "r"(kb + 4u * (8 * kt + 4 + c)));
+          }
+          ldmatrix_x4_trans(xt + tile_off<V>(16 * kt + mr + 8 * (mi & 1), 2 * d + (mi >> 1)), b0, b1, b2, b3);
+          mma_bf16_16816(dvacc[0], Ak, b0, b1);
+          mma_bf16_16816(dvacc[1], Ak, b2, b3);
+        }
+        if (g == 0) {
+          const uint32_t dst = slot_sa(j) + 4u * (L.oDV + s * V + 16 * d + 2 * c);
+          sts64(dst, make_float2(dvacc[0][0], dvacc[0][1]));
+          sts64(dst + 32u, make_float2(dvacc[1][0], dvacc[1][1]));
+        }
         __syncwarp();
         if (lane == 0) mbar_arrive(&dx_free[xb]);
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(&st_free[j & 1]);
+      if (lane == 0) { mbar_arrive(&st_free[j & 1]); mbar_arrive(&out_full[j & (kRing - 1)]); }
     }
     float *dWp = a.dW_part + ((size_t)(b * RS + rs) * N + n) * V * V;   // one partial per CTA, [b][slab][n]
 #pragma unroll
@@ -506,15 +567,23 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
       const int t0 = chunk_t0(j), len = chunk_len(j);
       const size_t bt0 = (size_t)b * T + t0;
       const int kc8 = KC / 8, v8 = V / 8;
+      uint4 *kb = reinterpret_cast<uint4 *>(sf + L.oKB), *vb = reinterpret_cast<uint4 *>(sf + L.oVB);
+      uint4 *dyb = reinterpret_cast<uint4 *>(sf + L.oDYB);
       for (int x = lane; x < len * kc8; x += 32) {
         const int t = x / kc8, i = (x % kc8) * 8;
+        const uint4 kr = *reinterpret_cast<const uint4 *>(kg + ((bt0 + t) * a.Nk + hk) * K + rbase + i);
         store8_bf16_as_f32(sf + L.oQ + t * KC + i, *reinterpret_cast<const uint4 *>(qg + ((bt0 + t) * a.Nq + hq) * K + rbase + i));
-        store8_bf16_as_f32(sf + L.oK + t * KC + i, *reinterpret_cast<const uint4 *>(kg + ((bt0 + t) * a.Nk + hk) * K + rbase + i));
+        store8_bf16_as_f32(sf + L.oK + t * KC + i, kr);
+        kb[x] = kr;
       }
       for (int x = lane; x < len * v8; x += 32) {
         const int t = x / v8, i = (x % v8) * 8;
-        store8_bf16_as_f32(sf + L.oV + t * V + i, *reinterpret_cast<const uint4 *>(vg + ((bt0 + t) * N + n) * V + i));
-        store8_bf16_as_f32(sf + L.oDY + t * V + i, *reinterpret_cast<const uint4 *>(dyg + ((bt0 + t) * N + n) * V + i));
+        const uint4 vr = *reinterpret_cast<const uint4 *>(vg + ((bt0 + t) * N + n) * V + i);
+        const uint4 dr = *reinterpret_cast<const uint4 *>(dyg + ((bt0 + t) * N + n) * V + i);
+        store8_bf16_as_f32(sf + L.oV + t * V + i, vr);
+        store8_bf16_as_f32(sf + L.oDY + t * V + i, dr);
+        vb[x] = vr;
+        dyb[x] = dr;
       }
       if (lane < len) {
         float dfdx;
@@ -538,14 +607,11 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
         if (a.dk_part) *reinterpret_cast<float2 *>(a.dk_part + ((bt0 + t) * N + n) * K + rbase + i) = dk2;
         else *reinterpret_cast<uint32_t *>(static_cast<__nv_bfloat16 *>(a.dk) + ((bt0 + t) * a.Nk + hk) * K + rbase + i) = pack_bf16(dk2.x, dk2.y);
       }
-      // dv: sum of the reverse warps' column sums (+ w_r (.) dy from Eq. 3, added by the first row slab only)
+      // dv of this CTA's rows (+ w_r (.) dy from Eq. 3, added by the first row slab only)
       for (int x = lane; x < len * (V / 2); x += 32) {
         const int t = x / (V / 2), jj = (x % (V / 2)) * 2;
-        float s0 = 0.f, s1 = 0.f;
-        for (int w = 0; w < NWC; ++w) {
-          const float2 p = *reinterpret_cast<const float2 *>(sf + L.oDVP + (t * NWC + w) * V + jj);
-          s0 += p.x; s1 += p.y;
-        }
+        const float2 p = *reinterpret_cast<const float2 *>(sf + L.oDV + t * V + jj);
+        float s0 = p.x, s1 = p.y;
         if (wr && rs == 0) {
           s0 = fmaf(__bfloat162float(wr[(size_t)n * V + jj]), sf[L.oDY + t * V + jj], s0);
           s1 = fmaf(__bfloat162float(wr[(size_t)n * V + jj + 1]), sf[L.oDY + t * V + jj + 1], s1);
@@ -554,13 +620,18 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
         if (a.dv_part) *reinterpret_cast<float2 *>(a.dv_part + (size_t)rs * BT * N * V + o) = make_float2(s0, s1);
         else *reinterpret_cast<uint32_t *>(static_cast<__nv_bfloat16 *>(a.dv) + o) = pack_bf16(s0, s1);
       }
-      if (lane < len) {
-        float s = 0.f;
-        for (int w = 0; w < NWC; ++w) s += sf[L.oDFP + lane * NWC + w];
-        s *= sf[L.oDF + lane];
-        const size_t o = (bt0 + lane) * N + n;
-        if (a.dgate_part) a.dgate_part[(size_t)rs * BT * N + o] = s;
-        else a.dgate[o] = s;
+      // dgate: the reverse warps leave one df partial per lane; fixed-order sum, then the gate's slope
+      for (int t = 0; t < len; ++t) {
+        float sdf = 0.f;
+        for (int w = 0; w < NWC; ++w) sdf += sf[L.oDFP + (t * NWC + w) * 32 + lane];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) sdf += __shfl_xor_sync(0xffffffffu, sdf, off);
+        if (lane == 0) {
+          sdf *= sf[L.oDF + t];
+          const size_t o = (bt0 + t) * N + n;
+          if (a.dgate_part) a.dgate_part[(size_t)rs * BT * N + o] = sdf;
+          else a.dgate[o] = sdf;
+        }
       }
     };
     for (int j = 0; j < min(2, nch); ++j) fill(j);
