@@ -38,7 +38,8 @@ struct FwdSmem {
 
 // MAXW: most compute warps the instantiation is launched with (K <= 16*MAXW).  Registers are
 // granted per 4 warps: up to 4+1 warps leave 255 per thread, 8+1 warps only 168.
-template <int V, int MAXW>
+// CKPT: whether checkpoints are written (a compile-time switch keeps the branch out of the hot loop).
+template <int V, int MAXW, bool CKPT>
 __global__ void __launch_bounds__((MAXW + 1) * 32, 1) fwd_bf16_kernel(ScanArgs a) {
   using G = TileGeom<V>;
   constexpr int NT = G::NT, KT = G::KT, SEG = G::SEG;
@@ -285,7 +286,7 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, 1) fwd_bf16_kernel(ScanArgs a
   float P0[NSET][NT][4], P1[NSET][NT][4];
   int ck_left = 0, ck_idx = 0;  // steps until the next checkpoint, index of the next checkpoint
   auto maybe_checkpoint = [&](int steps) {   // called before an even-numbered step
-    if (a.ckpt) {
+    if constexpr (CKPT) {
       if (ck_left == 0) {
         store_state(a.ckpt + ((size_t)bn * a.nchunks + ck_idx) * KV);
         ++ck_idx;
@@ -316,51 +317,66 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, 1) fwd_bf16_kernel(ScanArgs a
   // Steps are taken in pairs (P0 -> P1 -> P0); the two steps of a pair form one basic block, so
   // the tail of the first (row reduction, last MMAs in flight) overlaps the head of the second.
   // TC and the checkpoint interval are even: stage hand-over and checkpoints fall between pairs.
-  int ch = 0, tl = 0, s = 0;   // stage-sized chunk of the scan, step within it, its stage
-  for (int t = 0; t + 1 < T; t += 2) {
-    const uint32_t st = stage_sa(s);
+  // All hand-over logic sits outside the loop over the pairs of a stage, whose body is
+  // straight-line code: a warp issues in order, and every branch in that loop used to cost the
+  // chain tens of cycles per step.
+  auto pair = [&](uint32_t st, int tl, uint32_t k2, uint32_t v2) {
     const uint32_t yp = st + oY + 4u * ((tl * NW + warp) * V);
-    const bool cross = tl + 2 == TC, more = t + 2 < T;
-    const int sn = s + 1 == kStages ? 0 : s + 1;
-    uint32_t k2 = st + oK + 4u * ((tl + 1) * K), v2 = st + oV + 4u * ((tl + 1) * V);   // after the last step: any valid row
-    if (more) {
-      if (cross) {
-        if (!mbar_wait(&full[sn], ((ch + 1) / kStages) & 1)) { report_timeout(a.dev_status); return; }
-        k2 = stage_sa(sn) + oK;
-        v2 = stage_sa(sn) + oV;
-      } else {
-        k2 += 4u * K;
-        v2 += 4u * V;
-      }
-    }
-    maybe_checkpoint(2);
     step(P0, P1, lds32(st + oF + 4u * tl), st + 4u * (tl * K), yp, st + oK + 4u * ((tl + 1) * K), st + oV + 4u * ((tl + 1) * V));
     step(P1, P0, lds32(st + oF + 4u * (tl + 1)), st + 4u * ((tl + 1) * K), yp + 4u * (NW * V), k2, v2);
-    if (cross || !more) {
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&done[s]);
-    }
-    tl += 2;
-    if (cross) { tl = 0; ++ch; s = sn; }
-  }
-  if (T & 1) {
+  };
+  for (int ch = 0, s = 0; ch < nchunks; ++ch) {
+    const int sn = s + 1 == kStages ? 0 : s + 1;
     const uint32_t st = stage_sa(s);
-    maybe_checkpoint(1);
-    step(P0, P1, lds32(st + oF + 4u * tl), st + 4u * (tl * K), st + oY + 4u * ((tl * NW + warp) * V),
-         st + oK + 4u * (tl * K), st + oV + 4u * (tl * V));
+    const int len = min(TC, T - ch * TC);
+    // the last step of a stage seeds the first step of the next one (after the last step of the
+    // scan: any valid row, the product is never read)
+    uint32_t kN = st + oK, vN = st + oV;
+    if (ch + 1 < nchunks) {
+      if (!mbar_wait(&full[sn], ((ch + 1) / kStages) & 1)) { report_timeout(a.dev_status); return; }
+      kN = stage_sa(sn) + oK;
+      vN = stage_sa(sn) + oV;
+    }
+    if (len == TC) {
+#pragma unroll 1
+      for (int tl = 0; tl < TC - 2; tl += 2) {
+        maybe_checkpoint(2);
+        pair(st, tl, st + oK + 4u * ((tl + 2) * K), st + oV + 4u * ((tl + 2) * V));
+      }
+      maybe_checkpoint(2);
+      pair(st, TC - 2, kN, vN);
+    } else {   // ragged last stage
+      int tl = 0;
+      for (; tl + 1 < len; tl += 2) {
+        maybe_checkpoint(2);
+        const int nx = tl + 2 < len ? tl + 2 : tl + 1;
+        pair(st, tl, st + oK + 4u * (nx * K), st + oV + 4u * (nx * V));
+      }
+      if (len & 1) {
+        maybe_checkpoint(1);
+        step(P0, P1, lds32(st + oF + 4u * tl), st + 4u * (tl * K), st + oY + 4u * ((tl * NW + warp) * V),
+             st + oK + 4u * (tl * K), st + oV + 4u * (tl * V));
+      }
+    }
     __syncwarp();
     if (lane == 0) mbar_arrive(&done[s]);
+    s = sn;
   }
   if (a.hT) store_state(a.hT + bn * KV);
 }
 
+template <int V, int MAXW, bool CKPT>
+cudaError_t launch_vwc(const ScanArgs &a, cudaStream_t s) {
+  const size_t smem = FwdSmem<V>::bytes(a.K);
+  cudaError_t e = cudaFuncSetAttribute(fwd_bf16_kernel<V, MAXW, CKPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  fwd_bf16_kernel<V, MAXW, CKPT><<<a.B * a.N, (a.K / 16 + 1) * 32, smem, s>>>(a);
+  return cudaGetLastError();
+}
+
 template <int V, int MAXW>
 cudaError_t launch_vw(const ScanArgs &a, cudaStream_t s) {
-  const size_t smem = FwdSmem<V>::bytes(a.K);
-  cudaError_t e = cudaFuncSetAttribute(fwd_bf16_kernel<V, MAXW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
-  fwd_bf16_kernel<V, MAXW><<<a.B * a.N, (a.K / 16 + 1) * 32, smem, s>>>(a);
-  return cudaGetLastError();
+  return a.ckpt ? launch_vwc<V, MAXW, true>(a, s) : launch_vwc<V, MAXW, false>(a, s);
 }
 
 template <int V>
