@@ -29,32 +29,13 @@
 #include "internal.h"
 #include "mma_tile.cuh"
 #include "pipeline.cuh"
+#include "tile.cuh"
 
 namespace m2rnn {
 namespace {
 
 constexpr int kRing = 4;         // chunk slots of staged inputs / outputs in flight
 constexpr int kBarBytes = 256;   // room for the mbarriers below
-
-// Byte offset of 16-byte chunk `chunk` of row `row` in a bf16 [rows][V] tile.  Chunks are
-// XOR-swizzled within 128-byte lines so that both the fragment-wise stores of the chain warps and
-// the ldmatrix reads of the dW warps (8 rows, same column chunk) spread over all banks.
-template <int V>
-__device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
-  constexpr int RB = 2 * V;
-  if constexpr (RB >= 128) {
-    return (uint32_t)(row * RB + ((chunk ^ (row & 7)) << 4));
-  } else {
-    const uint32_t lin = (uint32_t)(row * RB + (chunk << 4));
-    const uint32_t line = lin >> 7;
-    return (line << 7) | ((((lin >> 4) & 7u) ^ (line & 7u)) << 4);
-  }
-}
-
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr) : "memory");
-}
 
 __device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
   uint32_t r;
@@ -142,7 +123,6 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
   constexpr bool kWInSmem = V > 64;
   // roles coincide with warpgroups only in this shape (4 + 4 + 4 + 1 warps), the one that needs it
   constexpr bool kRebalance = NWC == 4 && V == 64;
-  constexpr int CPR = SEG * 2 / 16;            // 16-byte chunks per thread-row of a tile (0 when V == 16)
   extern __shared__ __align__(128) unsigned char smem[];
 
   const int K = a.K, N = a.N, T = a.T, C = a.C, nch = a.nchunks;
@@ -193,41 +173,8 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
 
   // Thread (g,c) of chain warp w owns state rows r0 = 16w+g and r0+8 (MMA rows g, g+8) and the
   // SEG memory columns SEG*c .. SEG*c+SEG-1 (MMA columns 8nt+2c+e <-> memory column SEG*c+2nt+e).
-  // Pair index p = nt*2 + h names the packed pair (row r0+8h, memory columns SEG*c+2nt, +1).
-  auto tile_store = [&](uint32_t tile_sa, int w, const uint32_t (&p)[NT][2]) {
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int row = 16 * w + g + 8 * h;
-      if constexpr (CPR == 0) {   // V == 16: 8 bytes per thread-row
-        const uint32_t addr = tile_sa + tile_off<V>(row, c >> 1) + 8u * (c & 1);
-        asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(addr), "r"(p[0][h]), "r"(p[1][h]) : "memory");
-      } else {
-#pragma unroll
-        for (int x = 0; x < CPR; ++x) {
-          const uint32_t addr = tile_sa + tile_off<V>(row, CPR * c + x);
-          asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(p[4 * x][h]), "r"(p[4 * x + 1][h]),
-                       "r"(p[4 * x + 2][h]), "r"(p[4 * x + 3][h]) : "memory");
-        }
-      }
-    }
-  };
-  auto tile_load = [&](uint32_t tile_sa, int w, uint32_t (&p)[NT][2]) {
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int row = 16 * w + g + 8 * h;
-      if constexpr (CPR == 0) {
-        const uint32_t addr = tile_sa + tile_off<V>(row, c >> 1) + 8u * (c & 1);
-        asm volatile("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(p[0][h]), "=r"(p[1][h]) : "r"(addr));
-      } else {
-#pragma unroll
-        for (int x = 0; x < CPR; ++x) {
-          const uint32_t addr = tile_sa + tile_off<V>(row, CPR * c + x);
-          asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];"
-                       : "=r"(p[4 * x][h]), "=r"(p[4 * x + 1][h]), "=r"(p[4 * x + 2][h]), "=r"(p[4 * x + 3][h]) : "r"(addr));
-        }
-      }
-    }
-  };
+  auto tile_store = [&](uint32_t tile_sa, int w, const uint32_t (&p)[NT][2]) { m2rnn::tile_store<V>(tile_sa, w, lane, p); };
+  auto tile_load = [&](uint32_t tile_sa, int w, uint32_t (&p)[NT][2]) { m2rnn::tile_load<V>(tile_sa, w, lane, p); };
   // Z fragments: private to the (warp, lane) pair that wrote them, 2*NT words per thread kept as
   // NT/2 groups of 16 bytes (group x of lane l at word ((w*NT/2 + x)*32 + l)*4)
   constexpr int ZG = NT / 2;
