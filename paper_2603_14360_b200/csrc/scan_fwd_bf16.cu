@@ -39,8 +39,11 @@ struct FwdSmem {
 // MAXW: most compute warps the instantiation is launched with (K <= 16*MAXW).  Registers are
 // granted per 4 warps: up to 4+1 warps leave 255 per thread, 8+1 warps only 168.
 // CKPT: whether checkpoints are written (a compile-time switch keeps the branch out of the hot loop).
-template <int V, int MAXW, bool CKPT>
-__global__ void __launch_bounds__((MAXW + 1) * 32, 1) fwd_bf16_kernel(ScanArgs a) {
+// OCC: CTAs per SM the kernel is compiled for.  With more (b,n) units than SMs, two co-resident
+// CTAs (two chain warps per scheduler) hide each other's latencies; the price is a smaller
+// register budget.
+template <int V, int MAXW, bool CKPT, int OCC>
+__global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs a) {
   using G = TileGeom<V>;
   constexpr int NT = G::NT, KT = G::KT, SEG = G::SEG;
   constexpr bool kWInRegs = V <= 64;
@@ -365,13 +368,22 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, 1) fwd_bf16_kernel(ScanArgs a
   if (a.hT) store_state(a.hT + bn * KV);
 }
 
+template <int V, int MAXW, bool CKPT, int OCC>
+cudaError_t launch_vwco(const ScanArgs &a, cudaStream_t s) {
+  const size_t smem = FwdSmem<V>::bytes(a.K);
+  cudaError_t e = cudaFuncSetAttribute(fwd_bf16_kernel<V, MAXW, CKPT, OCC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  fwd_bf16_kernel<V, MAXW, CKPT, OCC><<<a.B * a.N, (a.K / 16 + 1) * 32, smem, s>>>(a);
+  return cudaGetLastError();
+}
+
 template <int V, int MAXW, bool CKPT>
 cudaError_t launch_vwc(const ScanArgs &a, cudaStream_t s) {
-  const size_t smem = FwdSmem<V>::bytes(a.K);
-  cudaError_t e = cudaFuncSetAttribute(fwd_bf16_kernel<V, MAXW, CKPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
-  fwd_bf16_kernel<V, MAXW, CKPT><<<a.B * a.N, (a.K / 16 + 1) * 32, smem, s>>>(a);
-  return cudaGetLastError();
+  // two CTAs per SM where there are units to fill them and the slab count leaves the registers
+  if constexpr (MAXW == 4 && V <= 64) {
+    if ((long)a.B * a.N > 148) return launch_vwco<V, MAXW, CKPT, 2>(a, s);
+  }
+  return launch_vwco<V, MAXW, CKPT, 1>(a, s);
 }
 
 template <int V, int MAXW>
