@@ -263,6 +263,9 @@ def main():
         outs = dict(y=torch.empty((B, T, N, V), dtype=io, device=dev),
                     hT=torch.empty((B, N, K, V), dtype=torch.float32, device=dev))
         out_tensors = list(outs.values())
+        fws_bytes = binding.m2rnn_fwd_workspace_bytes(p)
+        fws = torch.empty(fws_bytes, dtype=torch.uint8, device=dev) if fws_bytes else None
+        launches_per_step = 2 if fws_bytes else 1          # the scan (+ the add of the row slabs' shares of y)
         if bwd:
             C = binding.m2rnn_ckpt_interval(p)
             outs["ckpt"] = torch.empty((B, N, (T + C - 1) // C, K, V), dtype=torch.float32, device=dev)
@@ -273,13 +276,13 @@ def main():
             ws = torch.empty(max(1, binding.m2rnn_bwd_workspace_bytes(p, True)), dtype=torch.uint8, device=dev)
             out_tensors += list(gouts.values())
             # fwd, bwd, dW reduce (+ dv and dgate reduces when a state's rows are split over CTAs)
-            launches_per_step = 3 + (2 if binding.m2rnn_bwd_row_slab(p) != K else 0)
+            launches_per_step += 2 + (2 if binding.m2rnn_bwd_row_slab(p) != K else 0)
         ev_mid = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
 
         def step(i, s=None, mark=False):
             s = s or dev_sets[i % ROTATE]
             binding.m2rnn_fwd(s["q"], s["k"], s["v"], s["gate"], W, s["h0"], gate_kind=cfg.gate_kind,
-                              save_ckpt=bwd, out=outs, stream=stream)
+                              save_ckpt=bwd, out=outs, workspace=fws, stream=stream)
             if bwd:
                 if mark:
                     ev_mid[0].record(stream)

@@ -96,16 +96,23 @@ int m2rnn_bwd_row_slab(const m2rnn_params *params);
 /* Bytes of the checkpoint tensor [B,N,ceil(T/C),K,V] (fp32). */
 size_t m2rnn_ckpt_bytes(const m2rnn_params *params);
 
+/* Scratch the forward call needs for `params`: 0 unless the library splits the rows of a state
+ * over several CTAs (it does when there are few (b,n) units, to fill the GPU), in which case the
+ * per-slab shares of y pass through this scratch before a second launch adds them. */
+size_t m2rnn_fwd_workspace_bytes(const m2rnn_params *params);
+
 /* Forward scan (Algorithm 1; Eq. 1-3).
  *   in : q,k,v,gate,W; h0 or NULL (= zero state); alpha,beta (GATE_PSI only, else ignored,
  *        may be NULL); w_r or NULL (residual term of Eq. 3 omitted, as in Algorithm 1)
  *   out: y [B,T,N,V]; hT or NULL: final state H_T (fp32);
  *        ckpt or NULL: ckpt[b,n,c] = H_{c*C}, the state BEFORE step c*C (so ckpt[..,0] = h0),
- *        for m2rnn_bwd. */
+ *        for m2rnn_bwd.
+ *   workspace: device scratch of at least m2rnn_fwd_workspace_bytes(params), 256-byte aligned
+ *        (NULL and 0 when that is 0); contents undefined afterwards. */
 int m2rnn_fwd(const m2rnn_params *params, const void *q, const void *k, const void *v,
               const float *gate, const void *W, const float *h0, const float *alpha,
               const float *beta, const void *w_r, void *y, float *hT, float *ckpt,
-              int32_t *dev_status, void *stream);
+              void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
 
 /* Scratch the backward call needs for `params`; `have_ckpt` != 0 if the caller will pass the
  * checkpoints written by m2rnn_fwd (otherwise the workspace also holds them). */

@@ -53,7 +53,8 @@ EXPORTS = {
     "m2rnn_ckpt_interval": (ctypes.c_int, [_pp]),
     "m2rnn_bwd_row_slab": (ctypes.c_int, [_pp]),
     "m2rnn_ckpt_bytes": (ctypes.c_size_t, [_pp]),
-    "m2rnn_fwd": (ctypes.c_int, [_pp] + [_vp] * 14),
+    "m2rnn_fwd_workspace_bytes": (ctypes.c_size_t, [_pp]),
+    "m2rnn_fwd": (ctypes.c_int, [_pp] + [_vp] * 13 + [ctypes.c_size_t, _vp, _vp]),
     "m2rnn_bwd_workspace_bytes": (ctypes.c_size_t, [_pp, ctypes.c_int]),
     "m2rnn_bwd": (ctypes.c_int, [_pp] + [_vp] * 19 + [ctypes.c_size_t, _vp, _vp]),
     "m2rnn_bwd_static_scratch": (ctypes.c_int, [_pp] + [_vp] * 20),
@@ -159,10 +160,15 @@ def m2rnn_bwd_workspace_bytes(p: Params, have_ckpt: bool) -> int:
     return _lib().m2rnn_bwd_workspace_bytes(ctypes.byref(p), int(have_ckpt))
 
 
+def m2rnn_fwd_workspace_bytes(p: Params) -> int:
+    return _lib().m2rnn_fwd_workspace_bytes(ctypes.byref(p))
+
+
 def m2rnn_fwd(q, k, v, gate, W, h0=None, *, gate_kind=GATE_LOGIT, alpha=None, beta=None, w_r=None,
-              save_ckpt=False, ckpt_interval=0, want_hT=True, out=None, stream=None):
+              save_ckpt=False, ckpt_interval=0, want_hT=True, out=None, workspace=None, stream=None):
     """Forward scan.  Returns (y, hT, ckpt); hT / ckpt are None when not requested.
-    ``out`` may hold preallocated ``y`` / ``hT`` / ``ckpt`` tensors to write into."""
+    ``out`` may hold preallocated ``y`` / ``hT`` / ``ckpt`` tensors to write into; ``workspace``
+    a preallocated uint8 tensor of at least ``m2rnn_fwd_workspace_bytes`` bytes."""
     p = _params(q, k, v, W, gate_kind, ckpt_interval)
     B, T, N, K, V, io = p.B, p.T, p.N, p.K, p.V, q.dtype
     _chk(q, "q", (B, T, p.Nq, K), io); _chk(k, "k", (B, T, p.Nk, K), io); _chk(v, "v", (B, T, N, V), io)
@@ -181,8 +187,12 @@ def m2rnn_fwd(q, k, v, gate, W, h0=None, *, gate_kind=GATE_LOGIT, alpha=None, be
         C = m2rnn_ckpt_interval(p)
         ckpt = torch.empty((B, N, (T + C - 1) // C, K, V), dtype=torch.float32, device=q.device)
     _chk(y, "y", (B, T, N, V), io); _chk(hT, "hT", (B, N, K, V), torch.float32)
+    need = m2rnn_fwd_workspace_bytes(p)
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
     rc = _lib().m2rnn_fwd(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(gate), _ptr(W), _ptr(h0),
                           _ptr(alpha), _ptr(beta), _ptr(w_r), _ptr(y), _ptr(hT), _ptr(ckpt),
+                          _ptr(workspace), 0 if workspace is None else workspace.numel(),
                           _ptr(device_status_word(q.device)), _stream(stream))
     if rc != 0:
         raise M2RNNError(rc, "m2rnn_fwd")

@@ -33,6 +33,23 @@ BwdPlan plan_bwd(int B, int N, int K, int V, int io_dtype) {
   return pl;
 }
 
+int plan_fwd_rows(int B, int N, int K, int V, int io_dtype) {
+  if (io_dtype == M2RNN_F32) return K;
+  // The smallest slab (a multiple of 16 rows that divides K) that still gives every CTA an SM of
+  // its own; with more units than SMs the whole state stays in one CTA.  V = 128 keeps the slab
+  // at 64 rows or fewer for the sake of registers.
+  constexpr int kSMs = 148;
+  const long units = (long)(B > 0 ? B : 1) * N;
+  const int cap = V > 64 ? 64 : 128;
+  int best = 0;
+  for (int kc = 16; kc <= K && kc <= cap; kc += 16) {
+    if (K % kc) continue;
+    best = kc;                                   // largest admissible slab so far
+    if (units * (K / kc) <= kSMs) break;         // first (smallest) slab that fits one wave
+  }
+  return best;
+}
+
 namespace {
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -91,6 +108,7 @@ ScanArgs base_args(const m2rnn_params *p) {
   a.B = p->B; a.T = p->T; a.N = p->N; a.Nq = p->Nq; a.Nk = p->Nk; a.K = p->K; a.V = p->V;
   a.gate_kind = p->gate_kind;
   a.KC = plan_bwd(p->B, p->N, p->K, p->V, p->io_dtype).KC;
+  a.KCf = plan_fwd_rows(p->B, p->N, p->K, p->V, p->io_dtype);
   a.C = interval_of(p);
   a.nchunks = p->T > 0 ? (p->T + a.C - 1) / a.C : 0;
   a.dh_clip = p->dh_clip;
@@ -138,10 +156,17 @@ size_t m2rnn_ckpt_bytes(const m2rnn_params *params) {
   return (size_t)params->B * params->N * ((params->T + C - 1) / C) * params->K * params->V * sizeof(float);
 }
 
+size_t m2rnn_fwd_workspace_bytes(const m2rnn_params *params) {
+  if (check_params(params, true) != M2RNN_OK) return 0;
+  const int RS = params->K / plan_fwd_rows(params->B, params->N, params->K, params->V, params->io_dtype);
+  if (RS <= 1) return 0;
+  return align_up((size_t)RS * params->B * params->T * params->N * params->V * sizeof(float));
+}
+
 int m2rnn_fwd(const m2rnn_params *params, const void *q, const void *k, const void *v,
               const float *gate, const void *W, const float *h0, const float *alpha,
               const float *beta, const void *w_r, void *y, float *hT, float *ckpt,
-              int32_t *dev_status, void *stream) {
+              void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream) {
   int rc = check_params(params, true);
   if (rc != M2RNN_OK) return rc;
   if (params->B == 0 || params->T == 0) return M2RNN_OK;
@@ -155,8 +180,17 @@ int m2rnn_fwd(const m2rnn_params *params, const void *q, const void *k, const vo
   a.alpha = params->gate_kind == M2RNN_GATE_PSI ? alpha : nullptr;
   a.beta = params->gate_kind == M2RNN_GATE_PSI ? beta : nullptr;
   a.y = y; a.hT = hT; a.ckpt = ckpt; a.dev_status = dev_status;
+  const size_t need = m2rnn_fwd_workspace_bytes(params);
+  if (need > 0) {
+    if (!workspace || workspace_bytes < need) return M2RNN_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return M2RNN_ERR_ALIGN;
+    a.y_part = static_cast<float *>(workspace);
+  }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaError_t e = params->io_dtype == M2RNN_F32 ? launch_fwd_f32(a, s) : launch_fwd_bf16(a, s);
+  if (e == cudaSuccess && a.y_part)
+    e = launch_reduce_slabs(a.y_part, y, params->io_dtype, params->K / a.KCf,
+                            (size_t)params->B * params->T * params->N * params->V, s);
   return e == cudaSuccess ? M2RNN_OK : M2RNN_ERR_CUDA;
 }
 

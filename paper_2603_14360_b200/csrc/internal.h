@@ -14,12 +14,14 @@ struct ScanArgs {
   int B, T, N, Nq, Nk, K, V;
   int gate_kind;
   int KC;         // bf16 backward: state rows per CTA (a divisor of K)
+  int KCf;        // bf16 forward: state rows per CTA (a divisor of K)
   int C;          // checkpoint interval (steps)
   int nchunks;    // ceil(T / C)
   float dh_clip;
   const void *q, *k, *v, *W, *w_r;
   const float *gate, *h0, *alpha, *beta;
   void *y;
+  float *y_part;  // bf16 forward, K/KCf > 1: [K/KCf][B,T,N,V] fp32 per-row-slab y, else null
   float *hT;
   float *ckpt;    // fwd: written (may be null); bwd: read
   // backward only
@@ -47,6 +49,7 @@ struct BwdPlan {
   int C_max;  // largest supported checkpoint interval
 };
 BwdPlan plan_bwd(int B, int N, int K, int V, int io_dtype);
+int plan_fwd_rows(int B, int N, int K, int V, int io_dtype);   // state rows per CTA of the forward kernel
 size_t bwd_bf16_smem_bytes(int KC, int V, int C);  // scan_bwd_bf16.cu
 
 // fp32 FMA path (scan_f32.cu)

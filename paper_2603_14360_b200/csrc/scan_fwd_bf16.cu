@@ -1,6 +1,8 @@
 // bf16 tensor-core forward scan (Algorithm 1) for sm_100a.
 //
-// One CTA per (b,n): K/16 compute warps, each holding a 16 x V slab of the state in registers
+// One CTA per (b, n, row slab) -- the K rows of a state are independent recurrences (Eq. 1-2 act
+// row by row), so a state may be split over several CTAs, whose partial readouts a second-stage
+// kernel adds.  Below, K is the slab's row count.  Per CTA: K/16 compute warps, each holding a 16 x V slab of the state in registers
 // for all T steps (see mma_tile.cuh), plus one service warp.  Per step a compute warp
 //   1. seeds its accumulators with the outer product k_t v_t^T (fp32 FMA),
 //   2. adds H_{t-1} W with V/16 x V/8 mma.sync.m16n8k16 (bf16 operands, fp32 accumulate),
@@ -54,11 +56,13 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
   constexpr int NSET = V == 128 ? 1 : (KT >= 2 ? 2 : 1);
   extern __shared__ __align__(16) unsigned char smem_raw[];
 
-  const int K = a.K, N = a.N, T = a.T;
+  const int Kf = a.K, K = a.KCf, N = a.N, T = a.T;   // rows of the whole state / of this CTA's slab
+  const int RS = Kf / K;
   const int NW = K >> 4;
   constexpr int TC = FwdSmem<V>::tc(MAXW * 16);   // K > 64 <=> MAXW == 8
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int bn = blockIdx.x, b = bn / N, n = bn % N;
+  const int bn = blockIdx.x / RS, rs = blockIdx.x % RS, b = bn / N, n = bn % N;
+  const int rbase = rs * K;   // first state row of this CTA
   const int stage_floats = FwdSmem<V>::stage_floats(K, TC);
 
   uint64_t *full = reinterpret_cast<uint64_t *>(smem_raw);  // [kStages]
@@ -112,8 +116,8 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
         const int x = lane + 32 * i;
         if (x < len * kq8) {
           const int t = x / kq8, j = (x % kq8) * 8;
-          rk[i] = *reinterpret_cast<const uint4 *>(kg + ((bt0 + t) * a.Nk + hk) * K + j);
-          if (want_y) rq[i] = *reinterpret_cast<const uint4 *>(qg + ((bt0 + t) * a.Nq + hq) * K + j);
+          rk[i] = *reinterpret_cast<const uint4 *>(kg + ((bt0 + t) * a.Nk + hk) * Kf + rbase + j);
+          if (want_y) rq[i] = *reinterpret_cast<const uint4 *>(qg + ((bt0 + t) * a.Nq + hq) * Kf + rbase + j);
         }
         if (x < len * v8) {
           const int t = x / v8, j = (x % v8) * 8;
@@ -160,14 +164,21 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
             acc[0] += p0.x; acc[1] += p0.y; acc[2] += p0.z; acc[3] += p0.w;
             acc[4] += p1.x; acc[5] += p1.y; acc[6] += p1.z; acc[7] += p1.w;
           }
-          if (wr) {
+          if (wr && rs == 0) {
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[e] = fmaf(__bfloat162float(wr[(size_t)n * V + j + e]), vS[t * V + j + e], acc[e]);
           }
-          uint4 o;
-          o.x = pack_bf16(acc[0], acc[1]); o.y = pack_bf16(acc[2], acc[3]);
-          o.z = pack_bf16(acc[4], acc[5]); o.w = pack_bf16(acc[6], acc[7]);
-          *reinterpret_cast<uint4 *>(yg + (((size_t)b * T + t0 + t) * N + n) * V + j) = o;
+          const size_t yo = (((size_t)b * T + t0 + t) * N + n) * V + j;
+          if (a.y_part) {   // this slab's share of y, fp32; the slabs are added by a second kernel
+            float *yp = a.y_part + (size_t)rs * a.B * T * N * V + yo;
+            *reinterpret_cast<float4 *>(yp) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+            *reinterpret_cast<float4 *>(yp + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
+          } else {
+            uint4 o;
+            o.x = pack_bf16(acc[0], acc[1]); o.y = pack_bf16(acc[2], acc[3]);
+            o.z = pack_bf16(acc[4], acc[5]); o.w = pack_bf16(acc[6], acc[7]);
+            *reinterpret_cast<uint4 *>(yg + yo) = o;
+          }
         }
         __syncwarp();
       }
@@ -179,7 +190,7 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
   // -------------------------------------------------------------------- compute warps
   const int g = lane >> 2, c = lane & 3;
   const int row0 = 16 * warp + 2 * g;   // memory rows row0, row0+1  <->  MMA rows g, g+8
-  const size_t KV = (size_t)K * V;
+  const size_t KV = (size_t)Kf * V;
 
   uint32_t Wr[kWInRegs ? KT : 1][kWInRegs ? NT : 1][2];
   if constexpr (kWInRegs) {
@@ -194,7 +205,7 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
   if (a.h0) {
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-      const float *src = a.h0 + bn * KV + (size_t)(row0 + h) * V + SEG * c;
+      const float *src = a.h0 + bn * KV + (size_t)(rbase + row0 + h) * V + SEG * c;
 #pragma unroll
       for (int x = 0; x < SEG / 4; ++x) {
         const float4 t4 = *reinterpret_cast<const float4 *>(src + 4 * x);
@@ -208,7 +219,7 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
   auto store_state = [&](float *dst) {
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-      float *p = dst + (size_t)(row0 + h) * V + SEG * c;
+      float *p = dst + (size_t)(rbase + row0 + h) * V + SEG * c;
 #pragma unroll
       for (int x = 0; x < SEG / 4; ++x)
         *reinterpret_cast<float4 *>(p + 4 * x) =
@@ -370,10 +381,10 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
 
 template <int V, int MAXW, bool CKPT, int OCC>
 cudaError_t launch_vwco(const ScanArgs &a, cudaStream_t s) {
-  const size_t smem = FwdSmem<V>::bytes(a.K);
+  const size_t smem = FwdSmem<V>::bytes(a.KCf);
   cudaError_t e = cudaFuncSetAttribute(fwd_bf16_kernel<V, MAXW, CKPT, OCC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  fwd_bf16_kernel<V, MAXW, CKPT, OCC><<<a.B * a.N, (a.K / 16 + 1) * 32, smem, s>>>(a);
+  fwd_bf16_kernel<V, MAXW, CKPT, OCC><<<a.B * a.N * (a.K / a.KCf), (a.KCf / 16 + 1) * 32, smem, s>>>(a);
   return cudaGetLastError();
 }
 
@@ -381,7 +392,7 @@ template <int V, int MAXW, bool CKPT>
 cudaError_t launch_vwc(const ScanArgs &a, cudaStream_t s) {
   // two CTAs per SM where there are units to fill them and the slab count leaves the registers
   if constexpr (MAXW == 4 && V <= 64) {
-    if ((long)a.B * a.N > 148) return launch_vwco<V, MAXW, CKPT, 2>(a, s);
+    if ((long)a.B * a.N * (a.K / a.KCf) > 148) return launch_vwco<V, MAXW, CKPT, 2>(a, s);
   }
   return launch_vwco<V, MAXW, CKPT, 1>(a, s);
 }
@@ -393,7 +404,7 @@ cudaError_t launch_vw(const ScanArgs &a, cudaStream_t s) {
 
 template <int V>
 cudaError_t launch_v(const ScanArgs &a, cudaStream_t s) {
-  return a.K <= 64 ? launch_vw<V, 4>(a, s) : launch_vw<V, 8>(a, s);
+  return a.KCf <= 64 ? launch_vw<V, 4>(a, s) : launch_vw<V, 8>(a, s);
 }
 
 }  // namespace

@@ -42,13 +42,13 @@ ODD = ctypes.c_void_p(0x10004)
 
 def _fwd(lib, p, **over):
     a = dict(q=FAKE, k=FAKE, v=FAKE, gate=FAKE, W=FAKE, h0=None, alpha=None, beta=None, w_r=None,
-             y=FAKE, hT=None, ckpt=None, st=None, stream=None)
+             y=FAKE, hT=None, ckpt=None, ws=None, ws_bytes=0, st=None, stream=None)
     a.update(over)
     return lib.m2rnn_fwd(ctypes.byref(p), *a.values())
 
 
 def test_fwd_rejects_bad_arguments(lib):
-    assert lib.m2rnn_fwd(None, *([FAKE] * 14)) == -1
+    assert lib.m2rnn_fwd(None, *([FAKE] * 13), 0, FAKE, FAKE) == -1
     assert _fwd(lib, _p(N=0)) == -2
     assert _fwd(lib, _p(Nq=3)) == -2                  # does not divide N
     assert _fwd(lib, _p(Nk=8)) == -2                  # more key heads than heads
@@ -64,6 +64,14 @@ def test_fwd_rejects_bad_arguments(lib):
     assert _fwd(lib, _p(gate_kind=2)) == -1           # psi needs alpha and beta
     assert _fwd(lib, _p(), v=ODD) == -4
     assert _fwd(lib, _p(), hT=ODD) == -4
+    # few units: the rows of a state are split over CTAs and y passes through a workspace
+    small = _p(B=1, N=2, Nq=2, Nk=2, K=64, V=64)
+    need = lib.m2rnn_fwd_workspace_bytes(ctypes.byref(small))
+    assert need >= 2 * 1 * 8 * 2 * 64 * 4
+    assert _fwd(lib, small) == -5
+    assert _fwd(lib, small, ws=ctypes.c_void_p(0x20000), ws_bytes=need - 1) == -5
+    assert _fwd(lib, small, ws=ctypes.c_void_p(0x20010), ws_bytes=need) == -4
+    assert lib.m2rnn_fwd_workspace_bytes(ctypes.byref(_p(B=64, N=16))) == 0
     # empty calls are fine and launch nothing
     assert _fwd(lib, _p(T=0)) == 0
     assert _fwd(lib, _p(B=0)) == 0
