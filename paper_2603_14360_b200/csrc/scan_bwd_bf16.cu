@@ -67,7 +67,8 @@ __device__ __forceinline__ void load_wt_fragment(const __nv_bfloat16 *__restrict
 // split (128 per thread here), then the chain warps take registers that the dW and service warps
 // give up.  An increase waits until the CTA's own pool holds enough released registers, so the
 // increases must not ask for more than the decreases release:
-//   +40*128 (recompute) + 80*128 (reverse) = 15360  <=  56*128 (dW) + 72*128 (service group) = 16384.
+//   V = 64:  +40*128 (recompute) + 80*128 (reverse) = 15360  <=  56*128 (dW) + 72*128 (service group) = 16384
+//   V = 128: +120*128 (both kinds of chain warps)   = 15360  <=  24*256 (dW) + 72*128 (service group) = 15360.
 // The instruction is warpgroup-wide, so only complete warpgroups may execute it: where it is used
 // the CTA is padded to 16 warps, and the three spare warps join the service warp's decrease and
 // leave.
@@ -112,8 +113,12 @@ __host__ __device__ inline BwdLayout bwd_layout(int KC, int C, bool w_in_smem) {
   return L;
 }
 
+// Shapes whose warp roles fill whole warpgroups and whose chain warps need more than an even share
+// of the registers: 4+4 chain warps + 4 dW warps (V = 64), 2+2 chain warps + 8 dW warps (V = 128).
 template <int V, int NWC>
-constexpr int bwd_threads() { return (NWC == 4 && V == 64) ? 512 : (2 * NWC + V / 16 + 1) * 32; }
+__host__ __device__ constexpr bool bwd_rebalance() { return (NWC == 4 && V == 64) || (NWC == 2 && V == 128); }
+template <int V, int NWC>
+__host__ __device__ constexpr int bwd_threads() { return bwd_rebalance<V, NWC>() ? 512 : (2 * NWC + V / 16 + 1) * 32; }
 
 template <int V, int NWC>
 __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(ScanArgs a) {
@@ -122,7 +127,7 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
   constexpr int KC = 16 * NWC, NDW = V / 16;
   constexpr bool kWInSmem = V > 64;
   // roles coincide with warpgroups only in this shape (4 + 4 + 4 + 1 warps), the one that needs it
-  constexpr bool kRebalance = NWC == 4 && V == 64;
+  constexpr bool kRebalance = bwd_rebalance<V, NWC>();
   extern __shared__ __align__(128) unsigned char smem[];
 
   const int K = a.K, N = a.N, T = a.T, C = a.C, nch = a.nchunks;
@@ -180,9 +185,14 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
   constexpr int ZG = NT / 2;
   auto zfrag_sa = [&](uint32_t step_sa, int w) { return step_sa + L.ztile + (uint32_t)(w * ZG * 32 + lane) * 16u; };
 
+  // (each setmaxnreg below is one instruction executed by every warp of its warpgroup, at the top
+  // of the code it governs)
+  if constexpr (kRebalance && V == 128) {
+    if (warp < 2 * NWC) reg_inc<248>();
+  }
   if (warp < NWC) {
     // ================================================================= recompute warps
-    if constexpr (kRebalance) reg_inc<168>();
+    if constexpr (kRebalance && V == 64) reg_inc<168>();
     const int w = warp, r0 = 16 * w + g;
     uint32_t Wr[kWInSmem ? 1 : KT][kWInSmem ? 1 : NT][2];
     if constexpr (!kWInSmem) {
@@ -272,7 +282,7 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
 
   if (warp < 2 * NWC) {
     // ================================================================= reverse warps
-    if constexpr (kRebalance) reg_inc<208>();
+    if constexpr (kRebalance && V == 64) reg_inc<208>();
     const int w = warp - NWC, r0 = 16 * w + g;
     uint32_t WTr[kWInSmem ? 1 : KT][kWInSmem ? 1 : NT][2];
     if constexpr (!kWInSmem) {
@@ -432,7 +442,7 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
   if (warp < 2 * NWC + NDW) {
     // ================================================================= dW warps
     // warp d owns dW rows l in [16d, 16d+16): acc += H_{t-1}[:, l]^T dX, contraction over the CTA's rows
-    if constexpr (kRebalance) reg_dec<72>();
+    if constexpr (kRebalance) { if constexpr (V == 64) reg_dec<72>(); else reg_dec<104>(); }
     const int d = warp - 2 * NWC;
     float acc[NT][4];
 #pragma unroll
@@ -498,10 +508,8 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
   }
 
   // =================================================================== service warp
-  if constexpr (kRebalance) {
-    reg_dec<56>();
-    if (warp > 2 * NWC + NDW) return;   // spare warps of the padded CTA
-  }
+  if constexpr (kRebalance) reg_dec<56>();
+  if (warp > 2 * NWC + NDW) return;   // spare warps of a padded CTA
   {
     const int hq = n / (N / a.Nq), hk = n / (N / a.Nk);
     const float al = a.alpha ? a.alpha[n] : 1.f, be = a.beta ? a.beta[n] : 0.f;
