@@ -128,6 +128,7 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
   constexpr bool kWInSmem = V > 64;
   // roles coincide with warpgroups only in this shape (4 + 4 + 4 + 1 warps), the one that needs it
   constexpr bool kRebalance = bwd_rebalance<V, NWC>();
+  constexpr int NSET = V == 128 ? 1 : (KT >= 2 ? 2 : 1);   // accumulator sets of the state x W product, as in the forward kernel
   extern __shared__ __align__(128) unsigned char smem[];
 
   const int K = a.K, N = a.N, T = a.T, C = a.C, nch = a.nchunks;
@@ -228,24 +229,26 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
         // P = k v^T + H W   (Eq. 1 before the non-linearity)
         const float k0 = lds32(sl + 4u * (L.oK + s * KC + r0)), k1 = lds32(sl + 4u * (L.oK + s * KC + r0 + 8));
         const float f = lds32(sl + 4u * (L.oF + s));
-        float P[NT][4];
+        // (the same accumulator sets, in the same order, as the forward kernel: the recomputed
+        // states repeat the forward pass bit for bit)
+        float P[NSET][NT][4];
 #pragma unroll
         for (int x = 0; x < SEG / 4; ++x) {
           const float4 v4 = lds128(sl + 4u * (L.oV + s * V + SEG * c + 4 * x));
-          P[2 * x][0] = k0 * v4.x; P[2 * x][1] = k0 * v4.y; P[2 * x][2] = k1 * v4.x; P[2 * x][3] = k1 * v4.y;
-          P[2 * x + 1][0] = k0 * v4.z; P[2 * x + 1][1] = k0 * v4.w; P[2 * x + 1][2] = k1 * v4.z; P[2 * x + 1][3] = k1 * v4.w;
+          P[0][2 * x][0] = k0 * v4.x; P[0][2 * x][1] = k0 * v4.y; P[0][2 * x][2] = k1 * v4.x; P[0][2 * x][3] = k1 * v4.y;
+          P[0][2 * x + 1][0] = k0 * v4.z; P[0][2 * x + 1][1] = k0 * v4.w; P[0][2 * x + 1][2] = k1 * v4.z; P[0][2 * x + 1][3] = k1 * v4.w;
         }
 #pragma unroll
         for (int kt = 0; kt < KT; ++kt) {
           const uint32_t Ak[4] = {hp[2 * kt][0], hp[2 * kt][1], hp[2 * kt + 1][0], hp[2 * kt + 1][1]};
+          const int set = kt % NSET;
 #pragma unroll
           for (int nt = 0; nt < NT; ++nt) {
-            if constexpr (kWInSmem) {
-              const uint2 wv = Wf[(kt * NT + nt) * 32 + lane];
-              mma_bf16_16816(P[nt], Ak, wv.x, wv.y);
-            } else {
-              mma_bf16_16816(P[nt], Ak, Wr[kt][nt][0], Wr[kt][nt][1]);
-            }
+            uint2 wv;
+            if constexpr (kWInSmem) wv = Wf[(kt * NT + nt) * 32 + lane];
+            else wv = make_uint2(Wr[kt][nt][0], Wr[kt][nt][1]);
+            if (kt >= 1 && kt < NSET) mma_bf16_16816_zero(P[set][nt], Ak, wv.x, wv.y);
+            else mma_bf16_16816(P[set][nt], Ak, wv.x, wv.y);
           }
         }
         // Z = tanh(P), kept as fp16 for the reverse sweep; H <- f H + (1-f) Z  (Eq. 2)
@@ -259,7 +262,9 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
             float z[4];
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
-              z[r] = tanh_approx(P[nt][r]);
+              float xin = P[0][nt][r];
+              if constexpr (NSET == 2) xin += P[1][nt][r];
+              z[r] = tanh_approx(xin);
               H[nt][r] = fmaf(f, H[nt][r] - z[r], z[r]);
             }
             zw[2 * u] = pack_f16(z[0], z[1]);
