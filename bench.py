@@ -190,6 +190,27 @@ def run_reference(args, cfg, pas):
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------------------------------ multi-rank plumbing
+# The scan has no exchange step: with N ranks every rank scans its own batch (replicas), and the
+# only communication is the barrier around the timed region and the max of the ranks' timings.
+def rank_input_seed(base_seed: int, rank: int, rotation: int) -> int:
+    """Seed of input set `rotation` on `rank`: distinct per rank so the replicas do not share data."""
+    return base_seed + 1000 * rank + 17 * rotation
+
+
+def max_over_ranks(values, dist, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.tolist()]
+
+
+def whole_job_tokens_per_s(tokens_per_rank: int, world: int, ms_step: float) -> float:
+    """All ranks' tokens over the slowest rank's time per step."""
+    return tokens_per_rank * world / (ms_step * 1e-3)
+
+
 # ------------------------------------------------------------------------------ GPU leg
 def nbytes(t):
     return 0 if t is None else t.numel() * t.element_size()
@@ -240,7 +261,7 @@ def main():
     # The decode workload rotates its per-token inputs; its state (2 x 1 GB per step) is far above L2.
     host_sets = []
     for r in range(ROTATE):
-        d = inputs.make_inputs(cfg, backward=bwd, seed=cfg.seed + 1000 * rank + 17 * r)
+        d = inputs.make_inputs(cfg, backward=bwd, seed=rank_input_seed(cfg.seed, rank, r))
         if pas == "decode":
             d = {k: (v[:, 0].contiguous() if k in ("q", "k", "v", "gate") else v) for k, v in d.items()}
         host_sets.append({k: (v.pin_memory() if isinstance(v, torch.Tensor) else v) for k, v in d.items()})
@@ -351,10 +372,7 @@ def main():
         barrier()
         ms_e2e = ev2[0].elapsed_time(ev2[1])
 
-    times = torch.tensor([ms_total, ms_e2e, ms_bwd], dtype=torch.float64, device=dev)
-    if dist:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e, ms_bwd = (float(x) for x in times.tolist())
+    ms_total, ms_e2e, ms_bwd = max_over_ranks([ms_total, ms_e2e, ms_bwd], dist, dev)
     if rank != 0:
         if dist:
             dist.destroy_process_group()
@@ -362,7 +380,7 @@ def main():
 
     ms_step = ms_total / args.steps
     tokens = (B if pas == "decode" else cfg.tokens) * world
-    value = tokens / (ms_step * 1e-3)
+    value = whole_job_tokens_per_s(tokens // world, world, ms_step)
     peaks = measured_peaks()
     esz = 2 if cfg.dtype == "bf16" else 4
     Tn = 1 if pas == "decode" else T
