@@ -3,14 +3,17 @@
 // The step streams the whole state through the chip once (read + write, fp32), so the kernel is
 // laid out around HBM: persistent CTAs walk a contiguous range of (head, batch) units in
 // head-major order, keep the head's transition matrix as MMA fragments in shared memory (re-read
-// only when the head changes), and every warp takes 16 state rows straight from global memory
-// into accumulator-layout registers with fully used 32-byte sectors, runs the state x W product
+// only when the head changes), and prefetch the states of the next units with the bulk async-copy
+// engine (cp.async.bulk into a two-stage shared-memory buffer, completion on an mbarrier) while
+// the current ones are computed.  Every warp takes 16 state rows from the staged copy into
+// accumulator-layout registers, runs the state x W product
 // on tensor cores (mma.sync, bf16 operands, fp32 accumulate), applies the outer product, tanh
 // and the gate in registers, writes the rows back in place and leaves its share of the readout
 // in shared memory, where the unit's warps are summed.
 #include "device_common.cuh"
 #include "internal.h"
 #include "mma_tile.cuh"
+#include "pipeline.cuh"
 
 namespace m2rnn {
 namespace {
@@ -34,12 +37,22 @@ __device__ __forceinline__ uint2 dec_w_fragment(const uint16_t *__restrict__ w, 
                     (uint32_t)w[r2 * V + col] | ((uint32_t)w[r3 * V + col] << 16));
 }
 
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+  asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// global -> shared bulk copy (no multicast); both addresses 16-byte aligned, size a multiple of 16
+__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
 template <int V>
 __global__ void __launch_bounds__(256, 1) decode_bf16_kernel(ScanArgs a, int WPU, int GPI, int tasks_per_head) {
   constexpr int NT = V / 8, KT = V / 16, SEG = V / 4, NX = V == 16 ? 1 : V / 16;
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  uint2 *Wf = reinterpret_cast<uint2 *>(smem_raw);                        // [KT][NT][32]
-  float *ypart = reinterpret_cast<float *>(smem_raw + KT * NT * 32 * 8);  // [2][GPI][WPU][V]
+  uint64_t *full = reinterpret_cast<uint64_t *>(smem_raw);                // [2] stage landed
+  uint2 *Wf = reinterpret_cast<uint2 *>(smem_raw + 16);                   // [KT][NT][32]
+  float *ypart = reinterpret_cast<float *>(smem_raw + 16 + KT * NT * 32 * 8);  // [2][GPI][WPU][V]
 
   const int K = a.K, N = a.N, B = a.B;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, c = lane & 3;
@@ -51,13 +64,37 @@ __global__ void __launch_bounds__(256, 1) decode_bf16_kernel(ScanArgs a, int WPU
   __nv_bfloat16 *yg = static_cast<__nv_bfloat16 *>(a.y);
   float *state = a.hT;   // == a.h0: updated in place
 
+  const size_t unit_floats = KV;                                          // one unit's state
+  float *stage = ypart + 2 * GPI * WPU * V;                               // [2][GPI][K][V] fp32
+  if (tid == 0) {
+    mbar_init(&full[0], 1);
+    mbar_init(&full[1], 1);
+    fence_mbar_init();
+  }
+  __syncthreads();
+
   const long ntasks = (long)N * tasks_per_head;
   const long t_begin = ntasks * blockIdx.x / gridDim.x, t_end = ntasks * (blockIdx.x + 1) / gridDim.x;
+  // one thread streams the states of a task's units into a stage, 16 KB per copy
+  auto prefetch = [&](long task, int st) {
+    const int n = (int)(task / tasks_per_head), b0 = (int)(task % tasks_per_head) * GPI;
+    const int units = min(GPI, B - b0);
+    const uint32_t bytes = (uint32_t)(unit_floats * 4);
+    mbar_expect_tx(&full[st], bytes * units);
+    for (int u = 0; u < units; ++u) {
+      const char *src = reinterpret_cast<const char *>(state + ((size_t)(b0 + u) * N + n) * unit_floats);
+      char *dst = reinterpret_cast<char *>(stage + ((size_t)st * GPI + u) * unit_floats);
+      for (uint32_t off = 0; off < bytes; off += 16384u) bulk_g2s(dst + off, src + off, min(16384u, bytes - off), &full[st]);
+    }
+  };
+  if (tid == 0 && t_begin < t_end) prefetch(t_begin, 0);
   int cur_head = -1;
   int it = 0;
   for (long task = t_begin; task < t_end; ++task, ++it) {
     const int n = (int)(task / tasks_per_head);
     const int b = (int)(task % tasks_per_head) * GPI + grp;
+    // the other stage was last read before the barrier that closed the previous iteration
+    if (tid == 0 && task + 1 < t_end) prefetch(task + 1, (it + 1) & 1);
     if (n != cur_head) {
       __syncthreads();   // everyone is done with the previous head's fragments
       const uint16_t *w = reinterpret_cast<const uint16_t *>(a.W) + (size_t)n * V * V;
@@ -66,6 +103,7 @@ __global__ void __launch_bounds__(256, 1) decode_bf16_kernel(ScanArgs a, int WPU
       __syncthreads();
     }
     const bool live = active_warp && b < B;
+    if (!mbar_wait(&full[it & 1], (it >> 1) & 1)) { report_timeout(a.dev_status); return; }
     float *yp = ypart + (size_t)(((it & 1) * GPI + (active_warp ? grp : 0)) * WPU + wu) * V;
     if (live) {
       const size_t bn = (size_t)b * N + n;
@@ -74,10 +112,11 @@ __global__ void __launch_bounds__(256, 1) decode_bf16_kernel(ScanArgs a, int WPU
       // state rows r0 and r0+8 in accumulator layout
       float H[NT][4];
       float *hrow0 = state + bn * KV + (size_t)r0 * V, *hrow1 = hrow0 + 8 * V;
+      const float *srow0 = stage + ((size_t)(it & 1) * GPI + grp) * unit_floats + (size_t)r0 * V, *srow1 = srow0 + 8 * V;
 #pragma unroll
       for (int x = 0; x < NX; ++x) {
-        const float4 t0 = *reinterpret_cast<const float4 *>(hrow0 + 16 * x + 4 * c);
-        const float4 t1 = *reinterpret_cast<const float4 *>(hrow1 + 16 * x + 4 * c);
+        const float4 t0 = *reinterpret_cast<const float4 *>(srow0 + 16 * x + 4 * c);
+        const float4 t1 = *reinterpret_cast<const float4 *>(srow1 + 16 * x + 4 * c);
         H[2 * x][0] = t0.x; H[2 * x][1] = t0.y; H[2 * x + 1][0] = t0.z; H[2 * x + 1][1] = t0.w;
         H[2 * x][2] = t1.x; H[2 * x][3] = t1.y; H[2 * x + 1][2] = t1.z; H[2 * x + 1][3] = t1.w;
       }
@@ -159,7 +198,8 @@ cudaError_t launch_decode_v(const ScanArgs &a, cudaStream_t s) {
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int grid = (int)(ntasks < sms ? ntasks : sms);
-  const size_t smem = (size_t)(V / 16) * (V / 8) * 32 * 8 + sizeof(float) * 2 * GPI * WPU * V;
+  const size_t smem = 16 + (size_t)(V / 16) * (V / 8) * 32 * 8 + sizeof(float) * 2 * GPI * WPU * V   // barriers, W, y partials
+                      + sizeof(float) * 2 * (size_t)GPI * a.K * V;                                   // two stages of states
   cudaError_t e = cudaFuncSetAttribute(decode_bf16_kernel<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   decode_bf16_kernel<V><<<grid, 256, smem, s>>>(a, WPU, GPI, tasks_per_head);
