@@ -10,6 +10,9 @@
 // on tensor cores (mma.sync, bf16 operands, fp32 accumulate), applies the outer product, tanh
 // and the gate in registers, writes the rows back in place and leaves its share of the readout
 // in shared memory, where the unit's warps are summed.
+#include <cstdlib>
+#include <cstring>
+
 #include "device_common.cuh"
 #include "internal.h"
 #include "mma_tile.cuh"
@@ -208,7 +211,11 @@ cudaError_t launch_decode_v(const ScanArgs &a, cudaStream_t s) {
 
 }  // namespace
 
+// The tcgen05 kernel takes the shapes whose states stack into a 128-row tile; the mma.sync kernel
+// above covers the rest.  M2RNN_DECODE_VARIANT=legacy forces the latter (benchmarking only).
 cudaError_t launch_decode_bf16(const ScanArgs &a, cudaStream_t s) {
+  const char *variant = getenv("M2RNN_DECODE_VARIANT");
+  if (decode_tc_supported(a) && !(variant && !strcmp(variant, "legacy"))) return launch_decode_tc_bf16(a, s);
   switch (a.V) {
     case 16: return launch_decode_v<16>(a, s);
     case 32: return launch_decode_v<32>(a, s);

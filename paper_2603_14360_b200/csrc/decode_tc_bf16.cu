@@ -1,0 +1,401 @@
+// bf16 decoding step (Eq. 1-3 once on a cached fp32 state) on the 5th-generation tensor cores.
+//
+// At decode time the K rows of every (b,n) state are independent rows of one product per head:
+// [B*K, V] x [V, V].  A CTA stacks the states of 128/K units of one head into an M = 128 tile and
+// runs H W as tcgen05.mma (kind::f16, bf16 operands from shared memory, fp32 accumulator in tensor
+// memory), which leaves the SM's issue slots and register file to the streaming part of the step:
+//   - the states of the next task arrive by TMA (cp.async.bulk.tensor, 32-column boxes landing in
+//     128-byte-swizzled rows, completion on an mbarrier) while the current task is computed;
+//   - all warps convert the staged fp32 rows to the bf16, 128-byte-swizzled K-major A tile;
+//   - one thread issues the V/16 MMAs and commits them to an mbarrier;
+//   - every thread then owns one state row and half of its columns: tcgen05.ld, + k_i v^T, tanh,
+//     gate against the staged fp32 row, write H_t back in place (global) and into the stage;
+//   - the readout y = H_t^T q is a column sum over the stage.
+// Persistent CTAs walk (head, batch) tasks in head-major order; W_n^T is rebuilt in shared memory
+// (K-major B tile) only when the head changes.  Every wait is bounded; a wait that runs out ends
+// the CTA through the common exit, which frees the tensor memory.
+#include <cuda.h>
+
+#include "device_common.cuh"
+#include "internal.h"
+#include "mma_tile.cuh"
+#include "pipeline.cuh"
+
+namespace m2rnn {
+namespace {
+
+constexpr int kM = 128;   // rows of the MMA tile = threads that own a row each
+
+__device__ __forceinline__ void mbar_expect_tx_tc(uint64_t *bar, uint32_t bytes) {
+  asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// One box of a tiled (2-D) tensor map, global -> shared, no multicast.  x (innermost) times the
+// element size must be a multiple of 16 bytes.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst_sa, const CUtensorMap *map, int x, int y, uint64_t *bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(dst_sa), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+
+// One box, shared -> global; completion is tracked by the issuing thread's bulk-async group.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int x, int y, uint32_t src_sa) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(x), "r"(y), "r"(src_sa) : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 operand in the 128-byte-swizzled canonical
+// layout: rows of 64 elements (128 bytes), groups of 8 rows 1024 bytes apart, 16-byte chunks of a
+// row XOR-ed with the row index modulo 8.
+//   bits  0-13 start address >> 4     bits 32-45 stride between 8-row groups >> 4
+//   bits 16-29 leading offset >> 4 (not used by swizzled K-major layouts)
+//   bits 46-47 descriptor version 1   bits 61-63 swizzle mode (2 = 128 bytes)
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t sa) {
+  return (uint64_t)((sa & 0x3ffffu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
+         ((uint64_t)2 << 61);
+}
+// Instruction descriptor of kind::f16: fp32 accumulator (bits 4-5 = 1), bf16 A and B (bits 7-9 and
+// 10-12 = 1), both K-major (bits 15, 16 = 0), N >> 3 in bits 17-22, M >> 4 in bits 24-28.
+__host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=f"(r[0]), "=f"(r[1]), "=f"(r[2]), "=f"(r[3]), "=f"(r[4]), "=f"(r[5]), "=f"(r[6]), "=f"(r[7]), "=f"(r[8]),
+        "=f"(r[9]), "=f"(r[10]), "=f"(r[11]), "=f"(r[12]), "=f"(r[13]), "=f"(r[14]), "=f"(r[15]), "=f"(r[16]),
+        "=f"(r[17]), "=f"(r[18]), "=f"(r[19]), "=f"(r[20]), "=f"(r[21]), "=f"(r[22]), "=f"(r[23]), "=f"(r[24]),
+        "=f"(r[25]), "=f"(r[26]), "=f"(r[27]), "=f"(r[28]), "=f"(r[29]), "=f"(r[30]), "=f"(r[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// A staged fp32 state tile: V/32 blocks of [128 rows][32 columns = 128 bytes], the 16-byte chunks of
+// a row XOR-ed with the row index modulo 8 (what the tensor map's 128-byte swizzle writes), so
+// that a thread walking along its own row and a warp walking down a column both spread over all
+// banks.  Offset in floats of element (i, j):
+template <int V>
+__device__ __forceinline__ uint32_t stage_off(int i, int j) {
+  return (uint32_t)(j >> 5) * (kM * 32) + (uint32_t)i * 32 + (uint32_t)(((((j & 31) >> 2) ^ (i & 7)) << 2) | (j & 3));
+}
+
+template <int V>
+struct TcSmem {
+  static constexpr uint32_t a_bytes = kM * V * 2;             // A tile: V/64 blocks of [128 rows][128 bytes]
+  static constexpr uint32_t b_bytes = V * V * 2;              // B tile (W^T): V/64 blocks of [V rows][128 bytes]
+  static constexpr uint32_t stage_bytes = kM * V * 4;
+  // offsets from the 1024-byte aligned base
+  static constexpr uint32_t oA = 0, oB = oA + a_bytes, oStage = oB + b_bytes, oVec = oStage + 2 * stage_bytes;
+  // vectors (two buffers, the next task's are fetched a task ahead): k [128], q [128], f [128] per
+  // row, v [128/K <= 8][V]; then the warps' readout partials [8][V]
+  static constexpr uint32_t vec_floats = 3 * kM + 8 * V;
+  static constexpr uint32_t vec_bytes = (2 * vec_floats + 8 * V) * 4;
+  static constexpr uint32_t oBar = oVec + vec_bytes;          // full[2], mma_done, tmem slot
+  static constexpr uint32_t total = oBar + 64 + 1024;         // + slack for the alignment of the base
+};
+
+template <int V>
+__global__ void __launch_bounds__(256, 1) decode_tc_kernel(ScanArgs a, int GPI, int tasks_per_head,
+                                                           const __grid_constant__ CUtensorMap state_map) {
+  using S = TcSmem<V>;
+  constexpr int HC = V / 2;             // columns per thread in the epilogue
+  extern __shared__ unsigned char smem_dyn[];
+  // the swizzled tiles want a 1024-byte aligned base
+  const uint32_t base_sa = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char *base = smem_dyn + (base_sa - smem_u32(smem_dyn));
+  float *stage = reinterpret_cast<float *>(base + S::oStage);
+  float *vecs = reinterpret_cast<float *>(base + S::oVec);
+  float *ypart = vecs + 2 * S::vec_floats;                  // [8 warps][V]
+  uint64_t *full = reinterpret_cast<uint64_t *>(base + S::oBar);   // [2]
+  uint64_t *mma_done = full + 2;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(mma_done + 1);
+
+  const int K = a.K, N = a.N, B = a.B;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const size_t KV = (size_t)K * V;
+  const __nv_bfloat16 *qg = static_cast<const __nv_bfloat16 *>(a.q), *kg = static_cast<const __nv_bfloat16 *>(a.k);
+  const __nv_bfloat16 *vg = static_cast<const __nv_bfloat16 *>(a.v), *wr = static_cast<const __nv_bfloat16 *>(a.w_r);
+  __nv_bfloat16 *yg = static_cast<__nv_bfloat16 *>(a.y);
+  float *state = a.hT;   // == a.h0: updated in place
+
+  if (tid == 0) {
+    mbar_init(&full[0], 1);
+    mbar_init(&full[1], 1);
+    mbar_init(mma_done, 1);
+    fence_mbar_init();
+  }
+  if (warp == 0) {   // V columns of tensor memory for the accumulator
+    __syncwarp();
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(V) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  const long ntasks = (long)N * tasks_per_head;
+  const long t_begin = ntasks * blockIdx.x / gridDim.x, t_end = ntasks * (blockIdx.x + 1) / gridDim.x;
+  // the last warp streams the states of a task's units into a stage: per unit and 32-column block
+  // one box of [K rows][32 columns] of the state viewed as a [B*N*K, V] matrix
+  auto prefetch = [&](long task, int st) {
+    const int n = (int)(task / tasks_per_head), b0 = (int)(task % tasks_per_head) * GPI;
+    const int units = min(GPI, B - b0);
+    if (lane == 0) mbar_expect_tx_tc(&full[st], (uint32_t)(units * K) * (uint32_t)(V * 4));
+    __syncwarp();
+    const uint32_t dst0 = base_sa + S::oStage + (uint32_t)st * S::stage_bytes;
+    for (int x = lane; x < units * (V / 32); x += 32) {
+      const int u = x / (V / 32), cb = x % (V / 32);
+      tma_load_2d(dst0 + (uint32_t)cb * (kM * 128) + (uint32_t)(u * K) * 128, &state_map, 32 * cb,
+                  (int)(((size_t)(b0 + u) * N + n) * K), &full[st]);
+    }
+  };
+  if (warp == 7 && t_begin < t_end) prefetch(t_begin, 0);
+  // Per-row scalars (threads 0..127: k_i, q_i, f of the row's unit) and the units' v vectors
+  // (threads 128..255) of a task, fetched into registers a task ahead and parked in shared memory
+  // when the current task no longer reads that buffer.
+  constexpr int kVPer = 8 * V / 128;   // v entries per thread at most (8 units)
+  // raw values only: nothing may depend on a load before the task that issued it is over
+  struct VecRegs { uint16_t k, q; float gate; uint16_t v[kVPer]; int n; };
+  auto fetch_vecs = [&](long task, VecRegs &o) {
+    const int n = (int)(task / tasks_per_head), b0 = (int)(task % tasks_per_head) * GPI;
+    const int hq = n / (N / a.Nq), hk = n / (N / a.Nk);
+    o.n = n;
+    o.k = o.q = 0; o.gate = 0.f;
+    if (tid < kM) {
+      const int i = tid, u = i / K, r = i % K, bb = b0 + u;
+      if (u < GPI && bb < B) {
+        o.k = reinterpret_cast<const uint16_t *>(kg)[((size_t)bb * a.Nk + hk) * K + r];
+        o.q = reinterpret_cast<const uint16_t *>(qg)[((size_t)bb * a.Nq + hq) * K + r];
+        o.gate = a.gate[(size_t)bb * N + n];
+      }
+    } else {
+#pragma unroll
+      for (int m = 0; m < kVPer; ++m) {
+        const int x = tid - kM + m * kM, u = x / V, bb = b0 + u;
+        o.v[m] = (x < GPI * V && bb < B) ? reinterpret_cast<const uint16_t *>(vg)[((size_t)bb * N + n) * V + (x % V)] : (uint16_t)0;
+      }
+    }
+  };
+  auto park_vecs = [&](int buf, const VecRegs &o) {
+    float *vb = vecs + (size_t)buf * S::vec_floats;
+    if (tid < kM) {
+      vb[tid] = __uint_as_float((uint32_t)o.k << 16);
+      vb[kM + tid] = __uint_as_float((uint32_t)o.q << 16);
+      // rows of absent units carry gate 0 -> some f; their results are never used
+      vb[2 * kM + tid] = gate_value(a.gate_kind, o.gate, a.alpha ? a.alpha[o.n] : 1.f, a.beta ? a.beta[o.n] : 0.f, nullptr);
+    } else {
+#pragma unroll
+      for (int m = 0; m < kVPer; ++m) {
+        const int x = tid - kM + m * kM;
+        if (x < GPI * V) vb[3 * kM + x] = __uint_as_float((uint32_t)o.v[m] << 16);
+      }
+    }
+  };
+  if (t_begin < t_end) {
+    VecRegs first;
+    fetch_vecs(t_begin, first);
+    park_vecs(0, first);
+  }
+
+  constexpr uint32_t idesc = umma_idesc_bf16(kM, V);
+  int cur_head = -1, it = 0;
+  bool failed = false;
+  for (long task = t_begin; task < t_end; ++task, ++it) {
+    const int n = (int)(task / tasks_per_head), b0 = (int)(task % tasks_per_head) * GPI;
+    const int rows = min(GPI, B - b0) * K;     // live rows of the tile
+    VecRegs next;
+    if (task + 1 < t_end) fetch_vecs(task + 1, next);   // lands while this task is computed
+    if (n != cur_head) {
+      // B tile = W_n^T, K-major: row j holds W[:, j]; element (j, l) sits in block l/64 at
+      // row j, 16-byte chunk ((l%64)/8) ^ (j%8), like the A tile
+      const uint16_t *w = reinterpret_cast<const uint16_t *>(a.W) + (size_t)n * V * V;
+      for (int x = tid; x < V * V / 8; x += blockDim.x) {
+        const int j = x % V, l0 = (x / V) * 8;
+        uint32_t p[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) p[e] = (uint32_t)w[(l0 + 2 * e) * V + j] | ((uint32_t)w[(l0 + 2 * e + 1) * V + j] << 16);
+        const uint32_t off = S::oB + (uint32_t)(l0 / 64) * (V * 128) + (uint32_t)j * 128 + ((((l0 % 64) / 8) ^ (j & 7)) << 4);
+        *reinterpret_cast<uint4 *>(base + off) = make_uint4(p[0], p[1], p[2], p[3]);
+      }
+      cur_head = n;
+    }
+    const float *kvec = vecs + (size_t)(it & 1) * S::vec_floats, *qvec = kvec + kM, *fvec = qvec + kM, *vvec = fvec + kM;
+    if (!__syncthreads_and(mbar_wait(&full[it & 1], (it >> 1) & 1))) { failed = true; break; }
+    float *sg = stage + (size_t)(it & 1) * (kM * V);
+
+    // fp32 rows -> bf16 A tile (rows past the live ones are zero: their results are never used)
+    for (int x = tid; x < kM * V / 8; x += blockDim.x) {
+      const int i = x / (V / 8), ch = x % (V / 8);
+      uint4 o = make_uint4(0u, 0u, 0u, 0u);
+      if (i < rows) {
+        const float4 lo = *reinterpret_cast<const float4 *>(sg + stage_off<V>(i, 8 * ch));
+        const float4 hi = *reinterpret_cast<const float4 *>(sg + stage_off<V>(i, 8 * ch + 4));
+        o = make_uint4(pack_bf16(lo.x, lo.y), pack_bf16(lo.z, lo.w), pack_bf16(hi.x, hi.y), pack_bf16(hi.z, hi.w));
+      }
+      const uint32_t off = S::oA + (uint32_t)(ch / 8) * (kM * 128) + (uint32_t)i * 128 + (((ch & 7) ^ (i & 7)) << 4);
+      *reinterpret_cast<uint4 *>(base + off) = o;
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the tensor core
+    __syncthreads();
+    if (tid == 0) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+      for (int ks = 0; ks < V / 16; ++ks) {
+        // 16 elements (32 bytes) per step inside a 128-byte block, then the next block
+        const uint32_t koff = (uint32_t)(ks / 4) * 128u * kM + (uint32_t)(ks % 4) * 32u;
+        const uint32_t koffb = (uint32_t)(ks / 4) * 128u * V + (uint32_t)(ks % 4) * 32u;
+        umma_bf16(tmem_base, umma_desc_sw128(base_sa + S::oA + koff), umma_desc_sw128(base_sa + S::oB + koffb), idesc, ks > 0);
+      }
+      umma_commit(mma_done);
+    }
+    if (warp == 7 && task + 1 < t_end) {
+      // the other stage: its rows were stored by the last task (wait until that store has read
+      // them) and written through the generic proxy before; the loads write through the async proxy
+      asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      prefetch(task + 1, (it + 1) & 1);
+    }
+    if (!__syncthreads_and(mbar_wait(mma_done, it & 1))) { failed = true; break; }
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+
+    // epilogue: thread = (row i, column half)
+    {
+      const int i = 32 * (warp & 3) + lane, half = warp >> 2;
+      const int u = i / K;
+      const bool live = i < rows;
+      const float ki = kvec[i], f = fvec[i];
+      const float *vrow = vvec + (size_t)(live ? u : 0) * V + half * HC;
+#pragma unroll
+      for (int cb = 0; cb < HC / 32; ++cb) {
+        float P[32];
+        tmem_ld32(tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(half * HC + 32 * cb), P);
+        if (live) {
+#pragma unroll
+          for (int x = 0; x < 8; ++x) {
+            float4 *sp = reinterpret_cast<float4 *>(sg + stage_off<V>(i, half * HC + 32 * cb + 4 * x));
+            const float4 h4 = *sp;
+            const float4 v4 = *reinterpret_cast<const float4 *>(vrow + 32 * cb + 4 * x);
+            float hn[4];
+            const float hv[4] = {h4.x, h4.y, h4.z, h4.w}, vv[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float z = tanh_approx(fmaf(ki, vv[e], P[4 * x + e]));   // Eq. 1
+              hn[e] = fmaf(f, hv[e] - z, z);                               // Eq. 2
+            }
+            *sp = make_float4(hn[0], hn[1], hn[2], hn[3]);
+          }
+        }
+      }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // H_t in the stage -> visible to the TMA store
+    __syncthreads();
+    if (warp == 7) {   // H_t back to global memory, in place, one box per unit and 32-column block
+      const int units = rows / K;
+      const uint32_t src0 = base_sa + S::oStage + (uint32_t)(it & 1) * S::stage_bytes;
+      for (int x = lane; x < units * (V / 32); x += 32) {
+        const int u = x / (V / 32), cb = x % (V / 32);
+        tma_store_2d(&state_map, 32 * cb, (int)(((size_t)(b0 + u) * N + n) * K), src0 + (uint32_t)cb * (kM * 128) + (uint32_t)(u * K) * 128);
+      }
+      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    }
+    // readout (Eq. 3): y[u][j] = sum over the unit's rows of q_i H_t[i][j].  Each warp sums 16 rows
+    // (all of one unit, K >= 16), a lane takes the columns lane, lane+32, ...; then the warps of a
+    // unit are added.
+    {
+      float acc[V / 32];
+#pragma unroll
+      for (int m = 0; m < V / 32; ++m) acc[m] = 0.f;
+#pragma unroll
+      for (int rr = 0; rr < 16; ++rr) {
+        const int i = 16 * warp + rr;
+        const float qi = qvec[i];
+#pragma unroll
+        for (int m = 0; m < V / 32; ++m) acc[m] = fmaf(qi, sg[stage_off<V>(i, lane + 32 * m)], acc[m]);
+      }
+#pragma unroll
+      for (int m = 0; m < V / 32; ++m) ypart[warp * V + lane + 32 * m] = acc[m];
+    }
+    __syncthreads();
+    for (int x = tid; x < GPI * V; x += blockDim.x) {
+      const int u = x / V, j = x % V, bb = b0 + u;
+      if (bb < B) {
+        float s = 0.f;
+        for (int w = u * K / 16; w < (u + 1) * K / 16; ++w) s += ypart[w * V + j];
+        if (wr) s = fmaf(__bfloat162float(wr[(size_t)n * V + j]), vvec[x], s);
+        yg[((size_t)bb * N + n) * V + j] = __float2bfloat16_rn(s);
+      }
+    }
+    if (task + 1 < t_end) park_vecs((it + 1) & 1, next);
+    __syncthreads();   // stage, vectors and tiles are free again
+  }
+  if (warp == 7) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // the last stores
+  if (failed) report_timeout(a.dev_status);
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(V) : "memory");
+  }
+}
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda)
+using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+template <int V>
+cudaError_t launch_tc(const ScanArgs &a, cudaStream_t s) {
+  // the state as a [B*N*K, V] fp32 matrix, boxes of [K rows][32 columns], 128-byte swizzle
+  EncodeTiledFn encode = encode_tiled_fn();
+  if (!encode) return cudaErrorNotSupported;
+  CUtensorMap map;
+  const cuuint64_t dims[2] = {(cuuint64_t)V, (cuuint64_t)a.B * a.N * a.K};
+  const cuuint64_t strides[1] = {(cuuint64_t)V * 4};
+  const cuuint32_t box[2] = {32u, (cuuint32_t)a.K}, estr[2] = {1u, 1u};
+  if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, a.hT, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return cudaErrorInvalidValue;
+  const int GPI = kM / a.K;
+  const int tasks_per_head = (a.B + GPI - 1) / GPI;
+  const long ntasks = (long)a.N * tasks_per_head;
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int grid = (int)(ntasks < sms ? ntasks : sms);
+  const size_t smem = TcSmem<V>::total;
+  cudaError_t e = cudaFuncSetAttribute(decode_tc_kernel<V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  decode_tc_kernel<V><<<grid, 256, smem, s>>>(a, GPI, tasks_per_head, map);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool decode_tc_supported(const ScanArgs &a) {
+  return (a.V == 64 || a.V == 128) && (a.K == 16 || a.K == 32 || a.K == 64 || a.K == 128);
+}
+
+cudaError_t launch_decode_tc_bf16(const ScanArgs &a, cudaStream_t s) {
+  return a.V == 64 ? launch_tc<64>(a, s) : launch_tc<128>(a, s);
+}
+
+}  // namespace m2rnn

@@ -59,7 +59,9 @@ cudaError_t launch_bwd_f32(const ScanArgs &a, cudaStream_t s);
 // bf16 tensor-core path
 cudaError_t launch_fwd_bf16(const ScanArgs &a, cudaStream_t s);     // scan_fwd_bf16.cu
 cudaError_t launch_bwd_bf16(const ScanArgs &a, cudaStream_t s);     // scan_bwd_bf16.cu
-cudaError_t launch_decode_bf16(const ScanArgs &a, cudaStream_t s);  // decode_bf16.cu
+cudaError_t launch_decode_bf16(const ScanArgs &a, cudaStream_t s);  // decode_bf16.cu: picks a kernel
+bool decode_tc_supported(const ScanArgs &a);                         // decode_tc_bf16.cu
+cudaError_t launch_decode_tc_bf16(const ScanArgs &a, cudaStream_t s);  // decode_tc_bf16.cu: tcgen05 path
 
 // reductions shared by both paths (reduce.cu)
 cudaError_t launch_reduce_dW(const float *dW_part, float *dW, int B, int N, int V, cudaStream_t s);
