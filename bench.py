@@ -405,10 +405,14 @@ def main():
         t_tensor, t_hbm = flops / (peaks["tflops_burst"] * 1e12), alg_bytes / (peaks["hbm_gbs"] * 1e9)
         passes = 2 if bwd else 1                                 # tanh per state element: recompute counts once more
         mufu_s = th * K * V / (16 * SM_COUNT * SM_HZ)
-        roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["tflops_burst"], "unit": "TFLOP/s",
-                "frac": achieved / peaks["tflops_burst"], "traffic": None,
+        if cfg.dtype == "f32":   # the fp32 path is plain FMA: 148 SMs x 128 FMA lanes x 2 flop x 1.965 GHz
+            bound, peak, psrc = "alu", SM_COUNT * 128 * 2 * SM_HZ / 1e12, "derived: 148 SMs x 128 fp32 FMA/clk x 1.965 GHz"
+        else:
+            bound, peak, psrc = "tensor", peaks["tflops_burst"], f"{peaks['source']} cuBLAS bf16 burst"
+        roof = {"bound": bound, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak, "traffic": None,
                 "call": "m2rnn_bwd" if bwd else "m2rnn_fwd", "call_ms": call_ms,
-                "peak_source": f"{peaks['source']} cuBLAS bf16 burst",
+                "peak_source": psrc,
                 "t_tensor_ms": t_tensor * 1e3, "t_hbm_ms": t_hbm * 1e3, "t_mufu_ms": mufu_s * 1e3,
                 "frac_of_mufu_ceiling": mufu_s / (call_ms * 1e-3),
                 "ns_per_scan_step": call_ms * 1e6 / T / passes}
