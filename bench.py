@@ -35,6 +35,10 @@ METRIC = "m2rnn_scan_tokens_per_s"
 ROTATE = 4  # input sets cycled through so that no step finds its inputs in L2
 PASS_OF = {"fwd_bf16": "fwd", "long_ctx": "fwd", "paper_layer": "fwd", "tiny_f32": "fwd", "decode": "decode"}
 SM_COUNT, SM_HZ = 148, 1.965e9
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
+# captures summarised under profiles/ (bptt_bf16: captured at T=512, scaled by 8 -- traffic is per
+# token-head).  None for workloads without a capture of the current kernel.
+NCU_TRAFFIC_BYTES = {"fwd_bf16": 117.8e6, "bptt_bf16": 8 * 658.6e6, "decode": 2.108e9}
 
 
 def workload_pass(name: str) -> str:
@@ -117,21 +121,22 @@ def oracle_sample_rate(cfg, pas, seconds_target=12.0):
     import oracle
     oracle.build()
     f = inputs.to_f64
-    nsub = min(cfg.N, 2)
-    small = cfg.with_(B=1, N=nsub, Nq=0, Nk=0)
+    nmax, bmax = min(cfg.N, 16), min(cfg.B, 4)
+    small = cfg.with_(B=bmax, N=nmax, Nq=0, Nk=0)
     if pas == "decode":
-        d = inputs.make_inputs(small.with_(B=4, T=1))
+        d = inputs.make_inputs(small.with_(T=1))
         args = [f(d[x][:, 0]) for x in ("q", "k", "v", "gate")] + [f(d["W"]), f(d["h0"])]
         oracle.decode_step(*args)
         t0 = time.perf_counter()
         reps = 0
-        while time.perf_counter() - t0 < min(seconds_target, 5.0):
+        while time.perf_counter() - t0 < seconds_target:
             oracle.decode_step(*args)
             reps += 1
         dt = time.perf_counter() - t0
-        per_unit = dt / (reps * 4 * nsub)
+        per_unit = dt / (reps * bmax * nmax)
         full = per_unit * cfg.B * cfg.N
-        return cfg.B / full, f"{reps} decode steps of {4 * nsub} of {cfg.B * cfg.N} (b,n) units, fp64, 1 thread, scaled by unit count", dt
+        return cfg.B / full, (f"{reps} decode steps of {bmax * nmax} of {cfg.B * cfg.N} (b,n) units, fp64, 1 thread, "
+                              "scaled by unit count"), dt
     d = inputs.make_inputs(small, backward=(pas == "fwd+bwd"))
     names = ("q", "k", "v", "gate", "W", "h0") + (("dy",) if pas == "fwd+bwd" else ())
     args = {x: f(d[x]) for x in names}
@@ -141,29 +146,36 @@ def oracle_sample_rate(cfg, pas, seconds_target=12.0):
         if pas == "fwd+bwd":
             oracle.bwd(sub["q"], sub["k"], sub["v"], sub["gate"], sub["W"], sub["h0"], sub["dy"])
 
-    def cut(units, T):
+    def cut(nb, nn, T):
         out = {}
         for x, a in args.items():
             if x == "W":
-                out[x] = a[:units]
+                out[x] = a[:nn]
             elif x == "h0":
-                out[x] = None if a is None else a[:, :units]
+                out[x] = None if a is None else a[:nb, :nn]
             else:
-                out[x] = a[:, :T, :units]
+                out[x] = a[:nb, :T, :nn]
         return out
 
     probe_T = min(cfg.T, 64)
     t0 = time.perf_counter()
-    run(cut(nsub, probe_T))
-    per_unit_step = (time.perf_counter() - t0) / (probe_T * nsub)
+    run(cut(1, min(nmax, 2), probe_T))
+    per_unit_step = (time.perf_counter() - t0) / (probe_T * min(nmax, 2))
     # whole units where a unit fits the budget, else one unit over a prefix of the sequence
     T_use = cfg.T
-    units = max(1, min(nsub, int(seconds_target / (per_unit_step * cfg.T))))
-    if per_unit_step * cfg.T > 2 * seconds_target:
+    budget_units = seconds_target / (per_unit_step * cfg.T)
+    if budget_units < 1:
+        nb, nn = 1, 1
         T_use = max(probe_T, int(seconds_target / per_unit_step))
+    elif budget_units < nmax:
+        nb, nn = 1, max(1, int(budget_units))
+    else:
+        nn = nmax
+        nb = max(1, min(bmax, int(budget_units / nmax)))
     t0 = time.perf_counter()
-    run(cut(units, T_use))
+    run(cut(nb, nn, T_use))
     dt = time.perf_counter() - t0
+    units = nb * nn
     full_time = dt * (cfg.B * cfg.N) / units * (cfg.T / T_use)
     what = f"{units} of {cfg.B * cfg.N} (b,n) units x T={T_use}" + ("" if T_use == cfg.T else f" of {cfg.T}")
     return cfg.tokens / full_time, f"{what}, {pas}, fp64, 1 thread, scaled by unit (and step) count", dt
@@ -392,7 +404,8 @@ def main():
         alg_bytes = state_bytes + in_bytes + th * V * esz
         achieved = alg_bytes / (ms_step * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "call": "m2rnn_decode_step",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if not args.seq_len else None,
+                "call": "m2rnn_decode_step",
                 "peak_source": f"{peaks['source']} HBM copy", "algorithmic_bytes_per_step": alg_bytes}
     else:
         # the contraction(s): forward 2KV^2 per token-head; backward 6KV^2 (recompute, dX W^T, H^T dX)
@@ -410,7 +423,7 @@ def main():
         else:
             bound, peak, psrc = "tensor", peaks["tflops_burst"], f"{peaks['source']} cuBLAS bf16 burst"
         roof = {"bound": bound, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": None,
+                "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if not args.seq_len else None,
                 "call": "m2rnn_bwd" if bwd else "m2rnn_fwd", "call_ms": call_ms,
                 "peak_source": psrc,
                 "t_tensor_ms": t_tensor * 1e3, "t_hbm_ms": t_hbm * 1e3, "t_mufu_ms": mufu_s * 1e3,
