@@ -229,8 +229,7 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
         // P = k v^T + H W   (Eq. 1 before the non-linearity)
         const float k0 = lds32(sl + 4u * (L.oK + s * KC + r0)), k1 = lds32(sl + 4u * (L.oK + s * KC + r0 + 8));
         const float f = lds32(sl + 4u * (L.oF + s));
-        // (the same accumulator sets, in the same order, as the forward kernel: the recomputed
-        // states repeat the forward pass bit for bit)
+        // (two accumulator sets, as in the one-warp-per-slab forward kernel)
         float P[NSET][NT][4];
 #pragma unroll
         for (int x = 0; x < SEG / 4; ++x) {

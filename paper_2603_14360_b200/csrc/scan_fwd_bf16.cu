@@ -14,6 +14,9 @@
 // stage of steps from global memory, converts them to fp32, evaluates the forget gate, and,
 // once a stage is done, adds the warps' readout partials and writes y with 16-byte stores.
 // Stages are handed over with mbarriers; every wait is bounded and reports through dev_status.
+#include <cstdlib>
+#include <cstring>
+
 #include "device_common.cuh"
 #include "internal.h"
 #include "mma_tile.cuh"
@@ -409,7 +412,12 @@ cudaError_t launch_v(const ScanArgs &a, cudaStream_t s) {
 
 }  // namespace
 
+// The column-split variant (two chain warps per 16-row slab) takes the shapes it supports; the
+// environment variable M2RNN_FWD_VARIANT=wide forces the one-warp-per-slab kernel of this file
+// (benchmarking only).
 cudaError_t launch_fwd_bf16(const ScanArgs &a, cudaStream_t s) {
+  const char *variant = getenv("M2RNN_FWD_VARIANT");
+  if (fwd_cs_supported(a) && !(variant && !strcmp(variant, "wide"))) return launch_fwd_bf16_cs(a, s);
   switch (a.V) {
     case 16: return launch_v<16>(a, s);
     case 32: return launch_v<32>(a, s);

@@ -1,0 +1,418 @@
+// bf16 tensor-core forward scan (Algorithm 1), column-split variant, for sm_100a.
+//
+// Same CTA layout, staging and service warp as scan_fwd_bf16.cu, but every 16-row slab of the state
+// is shared by TWO chain warps, each owning half of the V columns.  A warp's step needs the whole
+// slab as the A operand of H W, so the two exchange their freshly packed bf16 fragments through
+// shared memory once per step (one named barrier for the pair).  The exchange hides behind the
+// MMAs a warp can already issue from its own fragments, and the scheduler now holds two chain warps
+// whose stalls interleave -- a single in-order warp per scheduler spends more than half of the step
+// waiting on its own dependency chain.  Each warp also holds only its half of W (V x V/2) in
+// registers, which keeps W out of shared memory up to V = 128.
+//
+// Accumulator element map of warp (slab s, half hf), lane (g = lane/4, c = lane%4):
+//   rows 16s+g and 16s+g+8; MMA column m of the half  <->  memory column hf*V/2 + (V/8)*c' + 2*(m>>3) + (m&1)
+//   with c' = (m&7)>>1, i.e. a thread holds V/8 adjacent columns of two rows.
+#include "device_common.cuh"
+#include "internal.h"
+#include "mma_tile.cuh"
+#include "pipeline.cuh"
+
+namespace m2rnn {
+namespace {
+
+constexpr int kStages = 3;
+constexpr int kBarrierBytes = 64;
+
+template <int V>
+struct CsSmem {
+  // Per stage (floats): q [TC][K], k [TC][K], v [TC][V], f [TC], ypart [TC][K/16][V]
+  __host__ __device__ static int stage_floats(int K, int TC) { return TC * (2 * K + V + 1 + (K / 16) * V); }
+  __host__ __device__ static constexpr int tc() { return V >= 128 ? 8 : 16; }
+  // fragment exchange: [2 parities][K/16 slabs][2 halves][V/32 k-tiles][32 lanes] x 16 bytes
+  __host__ __device__ static int xchg_bytes(int K) { return 2 * (K / 16) * 2 * (V / 32) * 32 * 16; }
+  __host__ static size_t bytes(int K) {
+    return sizeof(float) * (size_t)kStages * stage_floats(K, tc()) + xchg_bytes(K) + kBarrierBytes;
+  }
+};
+
+// memory column (inside a half) of MMA column m of that half
+template <int V>
+__host__ __device__ constexpr int half_col(int m) { return (V / 8) * ((m & 7) >> 1) + 2 * (m >> 3) + (m & 1); }
+
+template <int V, int MAXS, bool CKPT, int OCC>
+__global__ void __launch_bounds__((2 * MAXS + 1) * 32, OCC) fwd_bf16_cs_kernel(ScanArgs a) {
+  constexpr int VH = V / 2;          // columns of a half
+  constexpr int NTH = VH / 8;        // accumulator tiles of a warp
+  constexpr int KT = V / 16;         // k-tiles of the product
+  constexpr int KTH = KT / 2;        // k-tiles a warp produces itself
+  constexpr int SEGH = V / 8;        // adjacent memory columns per thread
+  constexpr int TC = CsSmem<V>::tc();
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+
+  const int Kf = a.K, K = a.KCf, N = a.N, T = a.T;   // rows of the whole state / of this CTA's slab group
+  const int RS = Kf / K;
+  const int NW = K >> 4;                               // 16-row slabs of this CTA
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int bn = blockIdx.x / RS, rs = blockIdx.x % RS, b = bn / N, n = bn % N;
+  const int rbase = rs * K;
+  const int stage_floats = CsSmem<V>::stage_floats(K, TC);
+
+  uint64_t *full = reinterpret_cast<uint64_t *>(smem_raw);  // [kStages]
+  uint64_t *done = full + kStages;                          // [kStages]
+  float *stages = reinterpret_cast<float *>(smem_raw + kBarrierBytes);
+  const uint32_t xchg_sa = smem_u32(stages + (size_t)kStages * stage_floats);
+
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&done[s], 2 * NW);
+    }
+    fence_mbar_init();
+  }
+  const __nv_bfloat16 *Wn = static_cast<const __nv_bfloat16 *>(a.W) + (size_t)n * V * V;
+  __syncthreads();
+
+  const int nchunks = (T + TC - 1) / TC;
+  const bool want_y = a.y != nullptr;
+
+  if (warp == 2 * NW) {
+    // ------------------------------------------------------------------ service warp
+    const int hq = n / (N / a.Nq), hk = n / (N / a.Nk);
+    const float al = a.alpha ? a.alpha[n] : 1.f, be = a.beta ? a.beta[n] : 0.f;
+    const __nv_bfloat16 *qg = static_cast<const __nv_bfloat16 *>(a.q);
+    const __nv_bfloat16 *kg = static_cast<const __nv_bfloat16 *>(a.k);
+    const __nv_bfloat16 *vg = static_cast<const __nv_bfloat16 *>(a.v);
+    const __nv_bfloat16 *wr = static_cast<const __nv_bfloat16 *>(a.w_r);
+    __nv_bfloat16 *yg = static_cast<__nv_bfloat16 *>(a.y);
+
+    // A stage holds at most 16 x 128 / 8 = 128 (TC = 8, K or V = 128) or 16 x 64 / 8 = 128 rows of
+    // 16 bytes per tensor: 4 per lane.  All loads of a stage are issued before the first use so
+    // that one global round trip covers the whole stage.
+    constexpr int kPerLane = 4;
+    auto fill = [&](int ch) {
+      const int s = ch % kStages, t0 = ch * TC, len = min(TC, T - t0);
+      float *qS = stages + (size_t)s * stage_floats, *kS = qS + TC * K, *vS = kS + TC * K, *fS = vS + TC * V;
+      const size_t bt0 = (size_t)b * T + t0;
+      const int kq8 = K / 8, v8 = V / 8;
+      uint4 rk[kPerLane], rq[kPerLane], rv[kPerLane];
+      float gt = 0.f;
+#pragma unroll
+      for (int i = 0; i < kPerLane; ++i) {
+        const int x = lane + 32 * i;
+        if (x < len * kq8) {
+          const int t = x / kq8, j = (x % kq8) * 8;
+          rk[i] = *reinterpret_cast<const uint4 *>(kg + ((bt0 + t) * a.Nk + hk) * Kf + rbase + j);
+          if (want_y) rq[i] = *reinterpret_cast<const uint4 *>(qg + ((bt0 + t) * a.Nq + hq) * Kf + rbase + j);
+        }
+        if (x < len * v8) {
+          const int t = x / v8, j = (x % v8) * 8;
+          rv[i] = *reinterpret_cast<const uint4 *>(vg + ((bt0 + t) * N + n) * V + j);
+        }
+      }
+      if (lane < len) gt = a.gate[(bt0 + lane) * N + n];
+#pragma unroll
+      for (int i = 0; i < kPerLane; ++i) {
+        const int x = lane + 32 * i;
+        if (x < len * kq8) {
+          const int t = x / kq8, j = (x % kq8) * 8;
+          store8_bf16_as_f32(kS + t * K + j, rk[i]);
+          if (want_y) store8_bf16_as_f32(qS + t * K + j, rq[i]);
+        }
+        if (x < len * v8) {
+          const int t = x / v8, j = (x % v8) * 8;
+          store8_bf16_as_f32(vS + t * V + j, rv[i]);
+        }
+      }
+      if (lane < len) fS[lane] = gate_value(a.gate_kind, gt, al, be, nullptr);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&full[s]);
+    };
+
+    const int pre = min(kStages, nchunks);
+    for (int ch = 0; ch < pre; ++ch) fill(ch);
+    for (int ch = 0; ch < nchunks; ++ch) {
+      const int s = ch % kStages, t0 = ch * TC, len = min(TC, T - t0);
+      if (!mbar_wait(&done[s], (ch / kStages) & 1)) { report_timeout(a.dev_status); return; }
+      if (want_y) {
+        // y[t][col] = sum over compute warps of their partials (+ w_r (.) v), 8 columns per lane
+        const float *vS = stages + (size_t)s * stage_floats + 2 * TC * K;
+        const float *yp = vS + TC * V + TC;
+        const int v8 = V / 8;
+        for (int x = lane; x < len * v8; x += 32) {
+          const int t = x / v8, j = (x % v8) * 8;
+          float acc[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+          for (int w = 0; w < NW; ++w) {
+            const float4 p0 = *reinterpret_cast<const float4 *>(yp + ((size_t)t * NW + w) * V + j);
+            const float4 p1 = *reinterpret_cast<const float4 *>(yp + ((size_t)t * NW + w) * V + j + 4);
+            acc[0] += p0.x; acc[1] += p0.y; acc[2] += p0.z; acc[3] += p0.w;
+            acc[4] += p1.x; acc[5] += p1.y; acc[6] += p1.z; acc[7] += p1.w;
+          }
+          if (wr && rs == 0) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = fmaf(__bfloat162float(wr[(size_t)n * V + j + e]), vS[t * V + j + e], acc[e]);
+          }
+          const size_t yo = (((size_t)b * T + t0 + t) * N + n) * V + j;
+          if (a.y_part) {   // this slab's share of y, fp32; the slabs are added by a second kernel
+            float *yp = a.y_part + (size_t)rs * a.B * T * N * V + yo;
+            *reinterpret_cast<float4 *>(yp) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+            *reinterpret_cast<float4 *>(yp + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
+          } else {
+            uint4 o;
+            o.x = pack_bf16(acc[0], acc[1]); o.y = pack_bf16(acc[2], acc[3]);
+            o.z = pack_bf16(acc[4], acc[5]); o.w = pack_bf16(acc[6], acc[7]);
+            *reinterpret_cast<uint4 *>(yg + yo) = o;
+          }
+        }
+        __syncwarp();
+      }
+      if (ch + kStages < nchunks) fill(ch + kStages);
+    }
+    return;
+  }
+
+  // -------------------------------------------------------------------- chain warps
+  const int g = lane >> 2, c = lane & 3;
+  const int slab = warp >> 1, hf = warp & 1;
+  const int r0 = 16 * slab + g;          // slab rows r0 and r0+8  <->  MMA rows g, g+8
+  const int col0 = hf * VH + SEGH * c;   // first of this thread's SEGH adjacent memory columns
+  const size_t KV = (size_t)Kf * V;
+
+  // B fragments of this warp's half of W: all KT k-tiles x NTH column tiles, kept in the order the
+  // warp uses them (its own k-tiles first, then the partner's) so that every index is static
+  uint32_t Wr[KT][NTH][2];
+  {
+    const uint16_t *w = reinterpret_cast<const uint16_t *>(Wn);
+#pragma unroll
+    for (int kt = 0; kt < KT; ++kt) {
+      const int hk = (kt / KTH) ^ hf, kth = kt % KTH;   // the k-tile's half (own half first) and its index inside it
+      const int l0 = hk * VH + half_col<V>(16 * kth + 2 * c), l1 = hk * VH + half_col<V>(16 * kth + 2 * c + 1);
+      const int l2 = hk * VH + half_col<V>(16 * kth + 8 + 2 * c), l3 = hk * VH + half_col<V>(16 * kth + 8 + 2 * c + 1);
+#pragma unroll
+      for (int nt = 0; nt < NTH; ++nt) {
+        const int j = hf * VH + half_col<V>(8 * nt + g);
+        Wr[kt][nt][0] = (uint32_t)w[l0 * V + j] | ((uint32_t)w[l1 * V + j] << 16);
+        Wr[kt][nt][1] = (uint32_t)w[l2 * V + j] | ((uint32_t)w[l3 * V + j] << 16);
+      }
+    }
+  }
+
+  // H[nt] = {row r0: cols 2nt, 2nt+1 of the thread's segment | row r0+8: same}
+  float H[NTH][4];
+  if (a.h0) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const float *src = a.h0 + bn * KV + (size_t)(rbase + r0 + 8 * h) * V + col0;
+#pragma unroll
+      for (int x = 0; x < SEGH / 4; ++x) {
+        const float4 t4 = *reinterpret_cast<const float4 *>(src + 4 * x);
+        H[2 * x][2 * h] = t4.x; H[2 * x][2 * h + 1] = t4.y; H[2 * x + 1][2 * h] = t4.z; H[2 * x + 1][2 * h + 1] = t4.w;
+      }
+    }
+  } else {
+#pragma unroll
+    for (int nt = 0; nt < NTH; ++nt) H[nt][0] = H[nt][1] = H[nt][2] = H[nt][3] = 0.f;
+  }
+  auto store_state = [&](float *dst) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      float *p = dst + (size_t)(rbase + r0 + 8 * h) * V + col0;
+#pragma unroll
+      for (int x = 0; x < SEGH / 4; ++x)
+        *reinterpret_cast<float4 *>(p + 4 * x) =
+            make_float4(H[2 * x][2 * h], H[2 * x][2 * h + 1], H[2 * x + 1][2 * h], H[2 * x + 1][2 * h + 1]);
+    }
+  };
+
+  // A fragments of the thread's own columns: k-tile kth of the half = accumulator tiles 2kth, 2kth+1
+  auto pack_own = [&](uint32_t (&A)[KTH][4]) {
+#pragma unroll
+    for (int kth = 0; kth < KTH; ++kth) {
+      A[kth][0] = pack_bf16(H[2 * kth][0], H[2 * kth][1]);
+      A[kth][1] = pack_bf16(H[2 * kth][2], H[2 * kth][3]);
+      A[kth][2] = pack_bf16(H[2 * kth + 1][0], H[2 * kth + 1][1]);
+      A[kth][3] = pack_bf16(H[2 * kth + 1][2], H[2 * kth + 1][3]);
+    }
+  };
+  // exchange slot of (parity, slab, half): KTH rows of 32 lanes x 16 bytes
+  auto xslot = [&](int par, int h) { return xchg_sa + (uint32_t)((((par * NW + slab) * 2 + h) * KTH) * 32 + lane) * 16u; };
+  auto xstore = [&](int par, const uint32_t (&A)[KTH][4]) {
+#pragma unroll
+    for (int kth = 0; kth < KTH; ++kth)
+      asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(xslot(par, hf) + 512u * kth), "r"(A[kth][0]), "r"(A[kth][1]),
+                   "r"(A[kth][2]), "r"(A[kth][3]) : "memory");
+  };
+  auto xload = [&](int par, uint32_t (&A)[KTH][4]) {
+#pragma unroll
+    for (int kth = 0; kth < KTH; ++kth)
+      asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(A[kth][0]), "=r"(A[kth][1]), "=r"(A[kth][2]), "=r"(A[kth][3])
+                   : "r"(xslot(par, hf ^ 1) + 512u * kth) : "memory");
+  };
+  auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + slab) : "memory"); };
+
+  // P[0] <- k v^T + (own k-tiles);  P[1] <- partner's k-tiles.  Summed where they are used.
+  auto seed = [&](float (&P)[2][NTH][4], uint32_t krow, uint32_t vrow) {
+    const float k0 = lds32(krow + 4u * r0), k1 = lds32(krow + 4u * (r0 + 8));
+#pragma unroll
+    for (int x = 0; x < SEGH / 4; ++x) {
+      const float4 v4 = lds128(vrow + 4u * (col0 + 4 * x));
+      P[0][2 * x][0] = k0 * v4.x; P[0][2 * x][1] = k0 * v4.y; P[0][2 * x][2] = k1 * v4.x; P[0][2 * x][3] = k1 * v4.y;
+      P[0][2 * x + 1][0] = k0 * v4.z; P[0][2 * x + 1][1] = k0 * v4.w; P[0][2 * x + 1][2] = k1 * v4.z; P[0][2 * x + 1][3] = k1 * v4.w;
+    }
+  };
+  auto mma_own = [&](float (&P)[2][NTH][4], const uint32_t (&A)[KTH][4]) {
+#pragma unroll
+    for (int kth = 0; kth < KTH; ++kth)
+#pragma unroll
+      for (int nt = 0; nt < NTH; ++nt) mma_bf16_16816(P[0][nt], A[kth], Wr[kth][nt][0], Wr[kth][nt][1]);
+  };
+  auto mma_partner = [&](float (&P)[2][NTH][4], const uint32_t (&A)[KTH][4]) {
+#pragma unroll
+    for (int kth = 0; kth < KTH; ++kth)
+#pragma unroll
+      for (int nt = 0; nt < NTH; ++nt) {
+        const int kt = KTH + kth;
+        if (kth == 0) mma_bf16_16816_zero(P[1][nt], A[kth], Wr[kt][nt][0], Wr[kt][nt][1]);
+        else mma_bf16_16816(P[1][nt], A[kth], Wr[kt][nt][0], Wr[kt][nt][1]);
+      }
+  };
+
+  // One step.  Pc: H_{t-1} W + k_t v_t^T (two partial sums), complete or in flight on entry.
+  // Pn receives the same for step t+1 (after the last step: fed a valid but meaningless row).
+  auto step = [&](float (&Pc)[2][NTH][4], float (&Pn)[2][NTH][4], float f, uint32_t qrow, uint32_t ydst,
+                  uint32_t krow_n, uint32_t vrow_n, int par) {
+    seed(Pn, krow_n, vrow_n);
+    const float q0 = lds32(qrow + 4u * r0), q1 = lds32(qrow + 4u * (r0 + 8));
+    float part[SEGH];
+#pragma unroll
+    for (int nt = 0; nt < NTH; ++nt) {
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const float z = tanh_approx(Pc[0][nt][r] + Pc[1][nt][r]);   // Eq. 1
+        H[nt][r] = fmaf(f, H[nt][r] - z, z);                        // Eq. 2
+      }
+      part[2 * nt] = fmaf(q1, H[nt][2], q0 * H[nt][0]);             // Eq. 3, this thread's two rows
+      part[2 * nt + 1] = fmaf(q1, H[nt][3], q0 * H[nt][1]);
+    }
+    uint32_t Aown[KTH][4], Apar[KTH][4];
+    pack_own(Aown);
+    xstore(par, Aown);
+    mma_own(Pn, Aown);
+    pair_sync();
+    xload(par, Apar);
+    mma_partner(Pn, Apar);
+    reduce_over_rows<SEGH>(part, lane);
+    // after the reduction lane (g,c) holds CNT sums starting at segment index (g >> (3-R)) * CNT
+    constexpr int R = SEGH >= 8 ? 3 : (SEGH >= 4 ? 2 : 1), CNT = SEGH >> R;
+    if (((g) & ((1 << (3 - R)) - 1)) == 0) {
+      const uint32_t dst = ydst + 4u * (col0 + (g >> (3 - R)) * CNT);
+      if constexpr (CNT == 2) sts64(dst, make_float2(part[0], part[1]));
+      else sts32(dst, part[0]);
+    }
+  };
+
+  float P0[2][NTH][4], P1[2][NTH][4];
+  int ck_left = 0, ck_idx = 0;
+  auto maybe_checkpoint = [&](int steps) {
+    if constexpr (CKPT) {
+      if (ck_left == 0) {
+        store_state(a.ckpt + ((size_t)bn * a.nchunks + ck_idx) * KV);
+        ++ck_idx;
+        ck_left = a.C;
+      }
+      ck_left -= steps;
+    }
+  };
+  const uint32_t stages_sa = smem_u32(stages);
+  auto stage_sa = [&](int s) { return stages_sa + 4u * (uint32_t)(s * stage_floats); };
+  const uint32_t oK = 4u * TC * K, oV = 2 * oK, oF = oV + 4u * TC * V, oY = oF + 4u * TC;
+
+  if (T > 0) {
+    if (!mbar_wait(&full[0], 0)) { report_timeout(a.dev_status); return; }
+    // prologue: the first step's product from the initial state (exchange parity 1 is free until step 1)
+    seed(P0, stages_sa + oK, stages_sa + oV);
+    uint32_t Aown[KTH][4], Apar[KTH][4];
+    pack_own(Aown);
+    xstore(1, Aown);
+    mma_own(P0, Aown);
+    pair_sync();
+    xload(1, Apar);
+    mma_partner(P0, Apar);
+    pair_sync();   // the partner has read slot 1 before step 1 overwrites it
+  }
+  auto pair = [&](uint32_t st, int tl, uint32_t k2, uint32_t v2) {
+    const uint32_t yp = st + oY + 4u * ((tl * NW + slab) * V);
+    step(P0, P1, lds32(st + oF + 4u * tl), st + 4u * (tl * K), yp, st + oK + 4u * ((tl + 1) * K), st + oV + 4u * ((tl + 1) * V), 0);
+    step(P1, P0, lds32(st + oF + 4u * (tl + 1)), st + 4u * ((tl + 1) * K), yp + 4u * (NW * V), k2, v2, 1);
+  };
+  for (int ch = 0, s = 0; ch < nchunks; ++ch) {
+    const int sn = s + 1 == kStages ? 0 : s + 1;
+    const uint32_t st = stage_sa(s);
+    const int len = min(TC, T - ch * TC);
+    uint32_t kN = st + oK, vN = st + oV;
+    if (ch + 1 < nchunks) {
+      if (!mbar_wait(&full[sn], ((ch + 1) / kStages) & 1)) { report_timeout(a.dev_status); return; }
+      kN = stage_sa(sn) + oK;
+      vN = stage_sa(sn) + oV;
+    }
+    if (len == TC) {
+#pragma unroll 1
+      for (int tl = 0; tl < TC - 2; tl += 2) {
+        maybe_checkpoint(2);
+        pair(st, tl, st + oK + 4u * ((tl + 2) * K), st + oV + 4u * ((tl + 2) * V));
+      }
+      maybe_checkpoint(2);
+      pair(st, TC - 2, kN, vN);
+    } else {   // ragged last stage
+      int tl = 0;
+      for (; tl + 1 < len; tl += 2) {
+        maybe_checkpoint(2);
+        const int nx = tl + 2 < len ? tl + 2 : tl + 1;
+        pair(st, tl, st + oK + 4u * (nx * K), st + oV + 4u * (nx * V));
+      }
+      if (len & 1) {
+        maybe_checkpoint(1);
+        step(P0, P1, lds32(st + oF + 4u * tl), st + 4u * (tl * K), st + oY + 4u * ((tl * NW + slab) * V),
+             st + oK + 4u * (tl * K), st + oV + 4u * (tl * V), 0);
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&done[s]);
+    s = sn;
+  }
+  if (a.hT) store_state(a.hT + bn * KV);
+}
+
+template <int V, int MAXS, bool CKPT, int OCC>
+cudaError_t launch_cs(const ScanArgs &a, cudaStream_t s) {
+  const size_t smem = CsSmem<V>::bytes(a.KCf);
+  cudaError_t e = cudaFuncSetAttribute(fwd_bf16_cs_kernel<V, MAXS, CKPT, OCC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  fwd_bf16_cs_kernel<V, MAXS, CKPT, OCC><<<a.B * a.N * (a.K / a.KCf), (2 * (a.KCf / 16) + 1) * 32, smem, s>>>(a);
+  return cudaGetLastError();
+}
+
+template <int V, int MAXS>
+cudaError_t launch_cs_v(const ScanArgs &a, cudaStream_t s) {
+  return a.ckpt ? launch_cs<V, MAXS, true, 1>(a, s) : launch_cs<V, MAXS, false, 1>(a, s);
+}
+
+}  // namespace
+
+// slabs per CTA this variant supports for a V: the register file holds (2 * slabs + 1) warps
+bool fwd_cs_supported(const ScanArgs &a) {
+  if (a.V == 128) return a.KCf <= 32;
+  return (a.V == 32 || a.V == 64) && a.KCf <= 64;
+}
+
+cudaError_t launch_fwd_bf16_cs(const ScanArgs &a, cudaStream_t s) {
+  switch (a.V) {
+    case 32: return launch_cs_v<32, 4>(a, s);
+    case 64: return launch_cs_v<64, 4>(a, s);
+    case 128: return launch_cs_v<128, 2>(a, s);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+}  // namespace m2rnn
