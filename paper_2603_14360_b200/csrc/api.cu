@@ -40,7 +40,7 @@ int plan_fwd_rows(int B, int N, int K, int V, int io_dtype) {
   // at 64 rows or fewer for the sake of registers.
   constexpr int kSMs = 148;
   const long units = (long)(B > 0 ? B : 1) * N;
-  const int cap = V > 64 ? 64 : 128;
+  const int cap = V > 64 ? 32 : 128;
   int best = 0;
   for (int kc = 16; kc <= K && kc <= cap; kc += 16) {
     if (K % kc) continue;
