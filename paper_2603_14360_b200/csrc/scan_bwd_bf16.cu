@@ -16,8 +16,8 @@
 //   dW warps        (V/16) accumulate dW += H_{t-1}^T dX on tensor cores from the two tiles
 //                          (ldmatrix.trans operands), one 16-row slab of dW per warp, off the chain,
 //                          and take dv = dX^T k along as one more row of the same product;
-//   service warp    (1)    stages q, k, v, dy and the gate for coming chunks, and reduces and writes
-//                          dq, dk, dv, dgate of finished ones.
+//   loader warp     (1)    stages q, k, v, dy and the gate of coming chunks;
+//   writer warp     (1)    reduces and writes dq, dk, dv, dgate of finished ones.
 //
 // While the reverse warps sweep chunk c the recompute warps already work on chunk c-1 (two state
 // buffers).  Hand-over is by mbarriers; every wait is bounded and reports through dev_status.
@@ -118,7 +118,7 @@ __host__ __device__ inline BwdLayout bwd_layout(int KC, int C, bool w_in_smem) {
 template <int V, int NWC>
 __host__ __device__ constexpr bool bwd_rebalance() { return (NWC == 4 && V == 64) || (NWC == 2 && V == 128); }
 template <int V, int NWC>
-__host__ __device__ constexpr int bwd_threads() { return bwd_rebalance<V, NWC>() ? 512 : (2 * NWC + V / 16 + 1) * 32; }
+__host__ __device__ constexpr int bwd_threads() { return bwd_rebalance<V, NWC>() ? 512 : (2 * NWC + V / 16 + 2) * 32; }
 
 template <int V, int NWC>
 __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(ScanArgs a) {
@@ -148,8 +148,9 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
   uint64_t *st_free = st_ready + 2;           // [2]
   uint64_t *dx_full = st_free + 2;            // [2]
   uint64_t *dx_free = dx_full + 2;            // [2]
+  uint64_t *slot_free = dx_free + 2;          // [kRing] chunk slot written out, free for the loader
   if (tid == 0) {
-    for (int s = 0; s < kRing; ++s) { mbar_init(&in_full[s], 1); mbar_init(&out_full[s], NWC + NDW); }
+    for (int s = 0; s < kRing; ++s) { mbar_init(&in_full[s], 1); mbar_init(&out_full[s], NWC + NDW); mbar_init(&slot_free[s], 1); }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&st_ready[s], NWC); mbar_init(&st_free[s], NWC + NDW);
       mbar_init(&dx_full[s], NWC); mbar_init(&dx_free[s], NDW);
@@ -511,9 +512,10 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
     return;
   }
 
-  // =================================================================== service warp
+  // =================================================================== loader and writer warps
   if constexpr (kRebalance) reg_dec<56>();
-  if (warp > 2 * NWC + NDW) return;   // spare warps of a padded CTA
+  if (warp > 2 * NWC + NDW + 1) return;   // spare warps of a padded CTA
+  const bool is_loader = warp == 2 * NWC + NDW;
   {
     const int hq = n / (N / a.Nq), hk = n / (N / a.Nk);
     const float al = a.alpha ? a.alpha[n] : 1.f, be = a.beta ? a.beta[n] : 0.f;
@@ -528,25 +530,40 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
       const int kc8 = KC / 8, v8 = V / 8;
       uint4 *kb = reinterpret_cast<uint4 *>(sf + L.oKB), *vb = reinterpret_cast<uint4 *>(sf + L.oVB);
       uint4 *dyb = reinterpret_cast<uint4 *>(sf + L.oDYB);
-      for (int x = lane; x < len * kc8; x += 32) {
-        const int t = x / kc8, i = (x % kc8) * 8;
-        const uint4 kr = *reinterpret_cast<const uint4 *>(kg + ((bt0 + t) * a.Nk + hk) * K + rbase + i);
-        store8_bf16_as_f32(sf + L.oQ + t * KC + i, *reinterpret_cast<const uint4 *>(qg + ((bt0 + t) * a.Nq + hq) * K + rbase + i));
-        store8_bf16_as_f32(sf + L.oK + t * KC + i, kr);
-        kb[x] = kr;
-      }
-      for (int x = lane; x < len * v8; x += 32) {
-        const int t = x / v8, i = (x % v8) * 8;
-        const uint4 vr = *reinterpret_cast<const uint4 *>(vg + ((bt0 + t) * N + n) * V + i);
-        const uint4 dr = *reinterpret_cast<const uint4 *>(dyg + ((bt0 + t) * N + n) * V + i);
-        store8_bf16_as_f32(sf + L.oV + t * V + i, vr);
-        store8_bf16_as_f32(sf + L.oDY + t * V + i, dr);
-        vb[x] = vr;
-        dyb[x] = dr;
+      float gt = 0.f;
+      if (lane < len) gt = a.gate[(bt0 + lane) * N + n];
+      // 32 rows of 16 bytes of each tensor per pass, every load of a pass issued before its first use
+      const int nk = len * kc8, nv = len * v8;
+      for (int x0 = 0; x0 < max(nk, nv); x0 += 32) {
+        const int x = x0 + lane;
+        uint4 qr, kr, vr, dr;
+        if (x < nk) {
+          const int t = x / kc8, i = (x % kc8) * 8;
+          qr = *reinterpret_cast<const uint4 *>(qg + ((bt0 + t) * a.Nq + hq) * K + rbase + i);
+          kr = *reinterpret_cast<const uint4 *>(kg + ((bt0 + t) * a.Nk + hk) * K + rbase + i);
+        }
+        if (x < nv) {
+          const int t = x / v8, i = (x % v8) * 8;
+          vr = *reinterpret_cast<const uint4 *>(vg + ((bt0 + t) * N + n) * V + i);
+          dr = *reinterpret_cast<const uint4 *>(dyg + ((bt0 + t) * N + n) * V + i);
+        }
+        if (x < nk) {
+          const int t = x / kc8, i = (x % kc8) * 8;
+          store8_bf16_as_f32(sf + L.oQ + t * KC + i, qr);
+          store8_bf16_as_f32(sf + L.oK + t * KC + i, kr);
+          kb[x] = kr;
+        }
+        if (x < nv) {
+          const int t = x / v8, i = (x % v8) * 8;
+          store8_bf16_as_f32(sf + L.oV + t * V + i, vr);
+          store8_bf16_as_f32(sf + L.oDY + t * V + i, dr);
+          vb[x] = vr;
+          dyb[x] = dr;
+        }
       }
       if (lane < len) {
         float dfdx;
-        sf[L.oF + lane] = gate_value(a.gate_kind, a.gate[(bt0 + lane) * N + n], al, be, &dfdx);
+        sf[L.oF + lane] = gate_value(a.gate_kind, gt, al, be, &dfdx);
         sf[L.oDF + lane] = dfdx;
       }
       __syncwarp();
@@ -593,12 +610,18 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
         }
       }
     };
-    for (int j = 0; j < min(2, nch); ++j) fill(j);
-    for (int j = 0; j < nch; ++j) {
-      if (j + 2 < nch) fill(j + 2);
-      if (!mbar_wait(&out_full[j & (kRing - 1)], (j / kRing) & 1)) { report_timeout(a.dev_status); return; }
-      flush(j);
-      __syncwarp();
+    if (is_loader) {
+      for (int j = 0; j < nch; ++j) {   // runs up to kRing chunks ahead of the writer
+        if (j >= kRing && !mbar_wait(&slot_free[j & (kRing - 1)], ((j / kRing) - 1) & 1)) { report_timeout(a.dev_status); return; }
+        fill(j);
+      }
+    } else {
+      for (int j = 0; j < nch; ++j) {
+        if (!mbar_wait(&out_full[j & (kRing - 1)], (j / kRing) & 1)) { report_timeout(a.dev_status); return; }
+        flush(j);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&slot_free[j & (kRing - 1)]);
+      }
     }
   }
 }
