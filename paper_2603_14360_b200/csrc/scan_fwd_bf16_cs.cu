@@ -47,6 +47,9 @@ __global__ void __launch_bounds__((2 * MAXS + 1) * 32, OCC) fwd_bf16_cs_kernel(S
   constexpr int KTH = KT / 2;        // k-tiles a warp produces itself
   constexpr int SEGH = V / 8;        // adjacent memory columns per thread
   constexpr int TC = CsSmem<V>::tc();
+  // packed fp32x2 arithmetic (sm_100) halves the FMA-pipe instructions of the epilogue; at V = 128
+  // the register pairs it needs cost more in spills than the instructions save
+  constexpr bool kPacked = V <= 64;
   extern __shared__ __align__(16) unsigned char smem_raw[];
 
   const int Kf = a.K, K = a.KCf, N = a.N, T = a.T;   // rows of the whole state / of this CTA's slab group
@@ -257,8 +260,16 @@ __global__ void __launch_bounds__((2 * MAXS + 1) * 32, OCC) fwd_bf16_cs_kernel(S
 #pragma unroll
     for (int x = 0; x < SEGH / 4; ++x) {
       const float4 v4 = lds128(vrow + 4u * (col0 + 4 * x));
-      P[0][2 * x][0] = k0 * v4.x; P[0][2 * x][1] = k0 * v4.y; P[0][2 * x][2] = k1 * v4.x; P[0][2 * x][3] = k1 * v4.y;
-      P[0][2 * x + 1][0] = k0 * v4.z; P[0][2 * x + 1][1] = k0 * v4.w; P[0][2 * x + 1][2] = k1 * v4.z; P[0][2 * x + 1][3] = k1 * v4.w;
+      if constexpr (!kPacked) {
+        P[0][2 * x][0] = k0 * v4.x; P[0][2 * x][1] = k0 * v4.y; P[0][2 * x][2] = k1 * v4.x; P[0][2 * x][3] = k1 * v4.y;
+        P[0][2 * x + 1][0] = k0 * v4.z; P[0][2 * x + 1][1] = k0 * v4.w; P[0][2 * x + 1][2] = k1 * v4.z; P[0][2 * x + 1][3] = k1 * v4.w;
+        continue;
+      }
+      // packed fp32 pairs (one instruction per two products on sm_100)
+      const float2 a0 = __fmul2_rn(make_float2(k0, k0), make_float2(v4.x, v4.y)), a1 = __fmul2_rn(make_float2(k1, k1), make_float2(v4.x, v4.y));
+      const float2 b0 = __fmul2_rn(make_float2(k0, k0), make_float2(v4.z, v4.w)), b1 = __fmul2_rn(make_float2(k1, k1), make_float2(v4.z, v4.w));
+      P[0][2 * x][0] = a0.x; P[0][2 * x][1] = a0.y; P[0][2 * x][2] = a1.x; P[0][2 * x][3] = a1.y;
+      P[0][2 * x + 1][0] = b0.x; P[0][2 * x + 1][1] = b0.y; P[0][2 * x + 1][2] = b1.x; P[0][2 * x + 1][3] = b1.y;
     }
   };
   auto mma_own = [&](float (&P)[2][NTH][4], const uint32_t (&A)[KTH][4]) {
@@ -285,15 +296,30 @@ __global__ void __launch_bounds__((2 * MAXS + 1) * 32, OCC) fwd_bf16_cs_kernel(S
     seed(Pn, krow_n, vrow_n);
     const float q0 = lds32(qrow + 4u * r0), q1 = lds32(qrow + 4u * (r0 + 8));
     float part[SEGH];
+    const float2 f2 = make_float2(f, f), m1 = make_float2(-1.f, -1.f), q02 = make_float2(q0, q0), q12 = make_float2(q1, q1);
 #pragma unroll
     for (int nt = 0; nt < NTH; ++nt) {
+      if constexpr (!kPacked) {
 #pragma unroll
-      for (int r = 0; r < 4; ++r) {
-        const float z = tanh_approx(Pc[0][nt][r] + Pc[1][nt][r]);   // Eq. 1
-        H[nt][r] = fmaf(f, H[nt][r] - z, z);                        // Eq. 2
+        for (int r = 0; r < 4; ++r) {
+          const float z = tanh_approx(Pc[0][nt][r] + Pc[1][nt][r]);   // Eq. 1
+          H[nt][r] = fmaf(f, H[nt][r] - z, z);                        // Eq. 2
+        }
+        part[2 * nt] = fmaf(q1, H[nt][2], q0 * H[nt][0]);             // Eq. 3, this thread's two rows
+        part[2 * nt + 1] = fmaf(q1, H[nt][3], q0 * H[nt][1]);
+        continue;
       }
-      part[2 * nt] = fmaf(q1, H[nt][2], q0 * H[nt][0]);             // Eq. 3, this thread's two rows
-      part[2 * nt + 1] = fmaf(q1, H[nt][3], q0 * H[nt][1]);
+      float2 hh[2];
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {   // the two rows' column pairs, as packed fp32 pairs
+        const float2 x = __fadd2_rn(make_float2(Pc[0][nt][2 * h], Pc[0][nt][2 * h + 1]), make_float2(Pc[1][nt][2 * h], Pc[1][nt][2 * h + 1]));
+        const float2 z = make_float2(tanh_approx(x.x), tanh_approx(x.y));                       // Eq. 1
+        const float2 d = __ffma2_rn(z, m1, make_float2(H[nt][2 * h], H[nt][2 * h + 1]));        // H - Z
+        hh[h] = __ffma2_rn(f2, d, z);                                                           // Eq. 2
+        H[nt][2 * h] = hh[h].x; H[nt][2 * h + 1] = hh[h].y;
+      }
+      const float2 pr = __ffma2_rn(q12, hh[1], __fmul2_rn(q02, hh[0]));   // Eq. 3, this thread's two rows
+      part[2 * nt] = pr.x; part[2 * nt + 1] = pr.y;
     }
     uint32_t Aown[KTH][4], Apar[KTH][4];
     pack_own(Aown);
