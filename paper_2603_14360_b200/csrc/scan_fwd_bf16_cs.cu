@@ -28,28 +28,26 @@ struct CsSmem {
   // Per stage (floats): q [TC][K], k [TC][K], v [TC][V], f [TC], ypart [TC][K/16][V]
   __host__ __device__ static int stage_floats(int K, int TC) { return TC * (2 * K + V + 1 + (K / 16) * V); }
   __host__ __device__ static constexpr int tc() { return V >= 128 ? 8 : 16; }
-  // fragment exchange: [2 parities][K/16 slabs][2 halves][V/32 k-tiles][32 lanes] x 16 bytes
-  __host__ __device__ static int xchg_bytes(int K) { return 2 * (K / 16) * 2 * (V / 32) * 32 * 16; }
+  // fragment exchange: [2 parities][K/16 slabs][V/16 k-tiles (part-major)][32 lanes] x 16 bytes
+  __host__ __device__ static int xchg_bytes(int K) { return 2 * (K / 16) * (V / 16) * 32 * 16; }
   __host__ static size_t bytes(int K) {
     return sizeof(float) * (size_t)kStages * stage_floats(K, tc()) + xchg_bytes(K) + kBarrierBytes;
   }
 };
 
-// memory column (inside a half) of MMA column m of that half
-template <int V>
-__host__ __device__ constexpr int half_col(int m) { return (V / 8) * ((m & 7) >> 1) + 2 * (m >> 3) + (m & 1); }
+// memory column (inside a part of VP columns) of MMA column m of that part
+template <int VP>
+__host__ __device__ constexpr int part_col(int m) { return (VP / 4) * ((m & 7) >> 1) + 2 * (m >> 3) + (m & 1); }
 
-template <int V, int MAXS, bool CKPT, int OCC>
-__global__ void __launch_bounds__((2 * MAXS + 1) * 32, OCC) fwd_bf16_cs_kernel(ScanArgs a) {
-  constexpr int VH = V / 2;          // columns of a half
+template <int V, int SP, int MAXS, bool CKPT, int OCC>
+__global__ void __launch_bounds__((SP * MAXS + 1) * 32, OCC) fwd_bf16_cs_kernel(ScanArgs a) {
+  constexpr int VH = V / SP;         // columns of a part
   constexpr int NTH = VH / 8;        // accumulator tiles of a warp
   constexpr int KT = V / 16;         // k-tiles of the product
-  constexpr int KTH = KT / 2;        // k-tiles a warp produces itself
-  constexpr int SEGH = V / 8;        // adjacent memory columns per thread
+  constexpr int KTH = KT / SP;       // k-tiles a warp produces itself
+  constexpr int KTP = KT - KTH;      // k-tiles it receives
+  constexpr int SEGH = VH / 4;       // adjacent memory columns per thread
   constexpr int TC = CsSmem<V>::tc();
-  // packed fp32x2 arithmetic (sm_100) halves the FMA-pipe instructions of the epilogue; at V = 128
-  // the register pairs it needs cost more in spills than the instructions save
-  constexpr bool kPacked = V <= 64;
   extern __shared__ __align__(16) unsigned char smem_raw[];
 
   const int Kf = a.K, K = a.KCf, N = a.N, T = a.T;   // rows of the whole state / of this CTA's slab group
@@ -68,7 +66,7 @@ __global__ void __launch_bounds__((2 * MAXS + 1) * 32, OCC) fwd_bf16_cs_kernel(S
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&full[s], 1);
-      mbar_init(&done[s], 2 * NW);
+      mbar_init(&done[s], SP * NW);
     }
     fence_mbar_init();
   }
@@ -78,7 +76,7 @@ __global__ void __launch_bounds__((2 * MAXS + 1) * 32, OCC) fwd_bf16_cs_kernel(S
   const int nchunks = (T + TC - 1) / TC;
   const bool want_y = a.y != nullptr;
 
-  if (warp == 2 * NW) {
+  if (warp == SP * NW) {
     // ------------------------------------------------------------------ service warp
     const int hq = n / (N / a.Nq), hk = n / (N / a.Nk);
     const float al = a.alpha ? a.alpha[n] : 1.f, be = a.beta ? a.beta[n] : 0.f;
@@ -177,7 +175,7 @@ __global__ void __launch_bounds__((2 * MAXS + 1) * 32, OCC) fwd_bf16_cs_kernel(S
 
   // -------------------------------------------------------------------- chain warps
   const int g = lane >> 2, c = lane & 3;
-  const int slab = warp >> 1, hf = warp & 1;
+  const int slab = warp / SP, hf = warp % SP;
   const int r0 = 16 * slab + g;          // slab rows r0 and r0+8  <->  MMA rows g, g+8
   const int col0 = hf * VH + SEGH * c;   // first of this thread's SEGH adjacent memory columns
   const size_t KV = (size_t)Kf * V;
@@ -189,12 +187,12 @@ __global__ void __launch_bounds__((2 * MAXS + 1) * 32, OCC) fwd_bf16_cs_kernel(S
     const uint16_t *w = reinterpret_cast<const uint16_t *>(Wn);
 #pragma unroll
     for (int kt = 0; kt < KT; ++kt) {
-      const int hk = (kt / KTH) ^ hf, kth = kt % KTH;   // the k-tile's half (own half first) and its index inside it
-      const int l0 = hk * VH + half_col<V>(16 * kth + 2 * c), l1 = hk * VH + half_col<V>(16 * kth + 2 * c + 1);
-      const int l2 = hk * VH + half_col<V>(16 * kth + 8 + 2 * c), l3 = hk * VH + half_col<V>(16 * kth + 8 + 2 * c + 1);
+      const int hk = (hf + kt / KTH) % SP, kth = kt % KTH;   // the k-tile's part (own part first, then round the ring) and its index inside it
+      const int l0 = hk * VH + part_col<VH>(16 * kth + 2 * c), l1 = hk * VH + part_col<VH>(16 * kth + 2 * c + 1);
+      const int l2 = hk * VH + part_col<VH>(16 * kth + 8 + 2 * c), l3 = hk * VH + part_col<VH>(16 * kth + 8 + 2 * c + 1);
 #pragma unroll
       for (int nt = 0; nt < NTH; ++nt) {
-        const int j = hf * VH + half_col<V>(8 * nt + g);
+        const int j = hf * VH + part_col<VH>(8 * nt + g);
         Wr[kt][nt][0] = (uint32_t)w[l0 * V + j] | ((uint32_t)w[l1 * V + j] << 16);
         Wr[kt][nt][1] = (uint32_t)w[l2 * V + j] | ((uint32_t)w[l3 * V + j] << 16);
       }
@@ -239,92 +237,97 @@ __global__ void __launch_bounds__((2 * MAXS + 1) * 32, OCC) fwd_bf16_cs_kernel(S
     }
   };
   // exchange slot of (parity, slab, half): KTH rows of 32 lanes x 16 bytes
-  auto xslot = [&](int par, int h) { return xchg_sa + (uint32_t)((((par * NW + slab) * 2 + h) * KTH) * 32 + lane) * 16u; };
+  auto xslot = [&](int par, int h) { return xchg_sa + (uint32_t)((((par * NW + slab) * SP + h) * KTH) * 32 + lane) * 16u; };
   auto xstore = [&](int par, const uint32_t (&A)[KTH][4]) {
 #pragma unroll
     for (int kth = 0; kth < KTH; ++kth)
       asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(xslot(par, hf) + 512u * kth), "r"(A[kth][0]), "r"(A[kth][1]),
                    "r"(A[kth][2]), "r"(A[kth][3]) : "memory");
   };
-  auto xload = [&](int par, uint32_t (&A)[KTH][4]) {
+  auto xload = [&](int par, uint32_t (&A)[KTP][4]) {
 #pragma unroll
-    for (int kth = 0; kth < KTH; ++kth)
-      asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(A[kth][0]), "=r"(A[kth][1]), "=r"(A[kth][2]), "=r"(A[kth][3])
-                   : "r"(xslot(par, hf ^ 1) + 512u * kth) : "memory");
+    for (int i = 0; i < KTP; ++i) {
+      const int h = (hf + 1 + i / KTH) % SP, kth = i % KTH;   // same ring order as Wr
+      asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(A[i][0]), "=r"(A[i][1]), "=r"(A[i][2]), "=r"(A[i][3])
+                   : "r"(xslot(par, h) + 512u * kth) : "memory");
+    }
   };
-  auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + slab) : "memory"); };
+  auto pair_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(1 + slab), "n"(32 * SP) : "memory"); };
 
-  // P[0] <- k v^T + (own k-tiles);  P[1] <- partner's k-tiles.  Summed where they are used.
-  auto seed = [&](float (&P)[2][NTH][4], uint32_t krow, uint32_t vrow) {
+  // P <- k v^T, then the own k-tiles, then the received ones
+  auto seed = [&](float (&P)[NTH][4], uint32_t krow, uint32_t vrow) {
     const float k0 = lds32(krow + 4u * r0), k1 = lds32(krow + 4u * (r0 + 8));
 #pragma unroll
     for (int x = 0; x < SEGH / 4; ++x) {
       const float4 v4 = lds128(vrow + 4u * (col0 + 4 * x));
-      if constexpr (!kPacked) {
-        P[0][2 * x][0] = k0 * v4.x; P[0][2 * x][1] = k0 * v4.y; P[0][2 * x][2] = k1 * v4.x; P[0][2 * x][3] = k1 * v4.y;
-        P[0][2 * x + 1][0] = k0 * v4.z; P[0][2 * x + 1][1] = k0 * v4.w; P[0][2 * x + 1][2] = k1 * v4.z; P[0][2 * x + 1][3] = k1 * v4.w;
-        continue;
-      }
       // packed fp32 pairs (one instruction per two products on sm_100)
       const float2 a0 = __fmul2_rn(make_float2(k0, k0), make_float2(v4.x, v4.y)), a1 = __fmul2_rn(make_float2(k1, k1), make_float2(v4.x, v4.y));
       const float2 b0 = __fmul2_rn(make_float2(k0, k0), make_float2(v4.z, v4.w)), b1 = __fmul2_rn(make_float2(k1, k1), make_float2(v4.z, v4.w));
-      P[0][2 * x][0] = a0.x; P[0][2 * x][1] = a0.y; P[0][2 * x][2] = a1.x; P[0][2 * x][3] = a1.y;
-      P[0][2 * x + 1][0] = b0.x; P[0][2 * x + 1][1] = b0.y; P[0][2 * x + 1][2] = b1.x; P[0][2 * x + 1][3] = b1.y;
+      P[2 * x][0] = a0.x; P[2 * x][1] = a0.y; P[2 * x][2] = a1.x; P[2 * x][3] = a1.y;
+      P[2 * x + 1][0] = b0.x; P[2 * x + 1][1] = b0.y; P[2 * x + 1][2] = b1.x; P[2 * x + 1][3] = b1.y;
     }
   };
-  auto mma_own = [&](float (&P)[2][NTH][4], const uint32_t (&A)[KTH][4]) {
+  auto mma_own = [&](float (&P)[NTH][4], const uint32_t (&A)[KTH][4]) {
 #pragma unroll
     for (int kth = 0; kth < KTH; ++kth)
 #pragma unroll
-      for (int nt = 0; nt < NTH; ++nt) mma_bf16_16816(P[0][nt], A[kth], Wr[kth][nt][0], Wr[kth][nt][1]);
+      for (int nt = 0; nt < NTH; ++nt) mma_bf16_16816(P[nt], A[kth], Wr[kth][nt][0], Wr[kth][nt][1]);
   };
-  auto mma_partner = [&](float (&P)[2][NTH][4], const uint32_t (&A)[KTH][4]) {
+  auto mma_partner = [&](float (&P)[NTH][4], const uint32_t (&A)[KTP][4]) {
 #pragma unroll
-    for (int kth = 0; kth < KTH; ++kth)
+    for (int i = 0; i < KTP; ++i)
 #pragma unroll
-      for (int nt = 0; nt < NTH; ++nt) {
-        const int kt = KTH + kth;
-        if (kth == 0) mma_bf16_16816_zero(P[1][nt], A[kth], Wr[kt][nt][0], Wr[kt][nt][1]);
-        else mma_bf16_16816(P[1][nt], A[kth], Wr[kt][nt][0], Wr[kt][nt][1]);
-      }
+      for (int nt = 0; nt < NTH; ++nt) mma_bf16_16816(P[nt], A[i], Wr[KTH + i][nt][0], Wr[KTH + i][nt][1]);
   };
 
   // One step.  Pc: H_{t-1} W + k_t v_t^T (two partial sums), complete or in flight on entry.
   // Pn receives the same for step t+1 (after the last step: fed a valid but meaningless row).
-  auto step = [&](float (&Pc)[2][NTH][4], float (&Pn)[2][NTH][4], float f, uint32_t qrow, uint32_t ydst,
+  auto step = [&](float (&Pc)[NTH][4], float (&Pn)[NTH][4], float f, uint32_t qrow, uint32_t ydst,
                   uint32_t krow_n, uint32_t vrow_n, int par) {
     seed(Pn, krow_n, vrow_n);
     const float q0 = lds32(qrow + 4u * r0), q1 = lds32(qrow + 4u * (r0 + 8));
     float part[SEGH];
     const float2 f2 = make_float2(f, f), m1 = make_float2(-1.f, -1.f), q02 = make_float2(q0, q0), q12 = make_float2(q1, q1);
+    // Unit u = (accumulator tile u/2, row half u%2): Eq. 1 and 2 for two elements, and after the
+    // tile's second unit its share of Eq. 3.
+    auto unit = [&](int u) {
+      const int nt = u >> 1, h = u & 1;
+      const float2 z = make_float2(tanh_approx(Pc[nt][2 * h]), tanh_approx(Pc[nt][2 * h + 1]));   // Eq. 1
+      const float2 d = __ffma2_rn(z, m1, make_float2(H[nt][2 * h], H[nt][2 * h + 1]));            // H - Z
+      const float2 hh = __ffma2_rn(f2, d, z);                                                     // Eq. 2
+      H[nt][2 * h] = hh.x; H[nt][2 * h + 1] = hh.y;
+      if (h == 1) {
+        const float2 pr = __ffma2_rn(q12, hh, __fmul2_rn(q02, make_float2(H[nt][0], H[nt][1])));  // Eq. 3, this thread's two rows
+        part[2 * nt] = pr.x; part[2 * nt + 1] = pr.y;
+      }
+    };
+    uint32_t Aown[KTH][4], Apar[KTP][4];
+    auto pack_store = [&](int kth) {
+      Aown[kth][0] = pack_bf16(H[2 * kth][0], H[2 * kth][1]);
+      Aown[kth][1] = pack_bf16(H[2 * kth][2], H[2 * kth][3]);
+      Aown[kth][2] = pack_bf16(H[2 * kth + 1][0], H[2 * kth + 1][1]);
+      Aown[kth][3] = pack_bf16(H[2 * kth + 1][2], H[2 * kth + 1][3]);
+      asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(xslot(par, hf) + 512u * kth), "r"(Aown[kth][0]), "r"(Aown[kth][1]),
+                   "r"(Aown[kth][2]), "r"(Aown[kth][3]) : "memory");
+    };
+    // The MMAs of own k-tile kth are issued between the units of the next k-tile's two
+    // accumulator tiles, so that the tensor pipe and the tanh unit work at the same time
+    // inside one in-order warp.
 #pragma unroll
-    for (int nt = 0; nt < NTH; ++nt) {
-      if constexpr (!kPacked) {
+    for (int u = 0; u < 4; ++u) unit(u);
+    pack_store(0);
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
-          const float z = tanh_approx(Pc[0][nt][r] + Pc[1][nt][r]);   // Eq. 1
-          H[nt][r] = fmaf(f, H[nt][r] - z, z);                        // Eq. 2
+    for (int kth = 0; kth < KTH; ++kth) {
+#pragma unroll
+      for (int nt = 0; nt < NTH; ++nt) {
+        mma_bf16_16816(Pn[nt], Aown[kth], Wr[kth][nt][0], Wr[kth][nt][1]);
+        if (kth + 1 < KTH) {
+#pragma unroll
+          for (int u = 4 * nt / NTH; u < 4 * (nt + 1) / NTH; ++u) unit(4 * (kth + 1) + u);
         }
-        part[2 * nt] = fmaf(q1, H[nt][2], q0 * H[nt][0]);             // Eq. 3, this thread's two rows
-        part[2 * nt + 1] = fmaf(q1, H[nt][3], q0 * H[nt][1]);
-        continue;
       }
-      float2 hh[2];
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {   // the two rows' column pairs, as packed fp32 pairs
-        const float2 x = __fadd2_rn(make_float2(Pc[0][nt][2 * h], Pc[0][nt][2 * h + 1]), make_float2(Pc[1][nt][2 * h], Pc[1][nt][2 * h + 1]));
-        const float2 z = make_float2(tanh_approx(x.x), tanh_approx(x.y));                       // Eq. 1
-        const float2 d = __ffma2_rn(z, m1, make_float2(H[nt][2 * h], H[nt][2 * h + 1]));        // H - Z
-        hh[h] = __ffma2_rn(f2, d, z);                                                           // Eq. 2
-        H[nt][2 * h] = hh[h].x; H[nt][2 * h + 1] = hh[h].y;
-      }
-      const float2 pr = __ffma2_rn(q12, hh[1], __fmul2_rn(q02, hh[0]));   // Eq. 3, this thread's two rows
-      part[2 * nt] = pr.x; part[2 * nt + 1] = pr.y;
+      if (kth + 1 < KTH) pack_store(kth + 1);
     }
-    uint32_t Aown[KTH][4], Apar[KTH][4];
-    pack_own(Aown);
-    xstore(par, Aown);
-    mma_own(Pn, Aown);
     pair_sync();
     xload(par, Apar);
     mma_partner(Pn, Apar);
@@ -338,7 +341,7 @@ __global__ void __launch_bounds__((2 * MAXS + 1) * 32, OCC) fwd_bf16_cs_kernel(S
     }
   };
 
-  float P0[2][NTH][4], P1[2][NTH][4];
+  float P0[NTH][4], P1[NTH][4];
   int ck_left = 0, ck_idx = 0;
   auto maybe_checkpoint = [&](int steps) {
     if constexpr (CKPT) {
@@ -358,7 +361,7 @@ __global__ void __launch_bounds__((2 * MAXS + 1) * 32, OCC) fwd_bf16_cs_kernel(S
     if (!mbar_wait(&full[0], 0)) { report_timeout(a.dev_status); return; }
     // prologue: the first step's product from the initial state (exchange parity 1 is free until step 1)
     seed(P0, stages_sa + oK, stages_sa + oV);
-    uint32_t Aown[KTH][4], Apar[KTH][4];
+    uint32_t Aown[KTH][4], Apar[KTP][4];
     pack_own(Aown);
     xstore(1, Aown);
     mma_own(P0, Aown);
@@ -410,18 +413,18 @@ __global__ void __launch_bounds__((2 * MAXS + 1) * 32, OCC) fwd_bf16_cs_kernel(S
   if (a.hT) store_state(a.hT + bn * KV);
 }
 
-template <int V, int MAXS, bool CKPT, int OCC>
+template <int V, int SP, int MAXS, bool CKPT, int OCC>
 cudaError_t launch_cs(const ScanArgs &a, cudaStream_t s) {
   const size_t smem = CsSmem<V>::bytes(a.KCf);
-  cudaError_t e = cudaFuncSetAttribute(fwd_bf16_cs_kernel<V, MAXS, CKPT, OCC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(fwd_bf16_cs_kernel<V, SP, MAXS, CKPT, OCC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  fwd_bf16_cs_kernel<V, MAXS, CKPT, OCC><<<a.B * a.N * (a.K / a.KCf), (2 * (a.KCf / 16) + 1) * 32, smem, s>>>(a);
+  fwd_bf16_cs_kernel<V, SP, MAXS, CKPT, OCC><<<a.B * a.N * (a.K / a.KCf), (SP * (a.KCf / 16) + 1) * 32, smem, s>>>(a);
   return cudaGetLastError();
 }
 
-template <int V, int MAXS>
+template <int V, int SP, int MAXS>
 cudaError_t launch_cs_v(const ScanArgs &a, cudaStream_t s) {
-  return a.ckpt ? launch_cs<V, MAXS, true, 1>(a, s) : launch_cs<V, MAXS, false, 1>(a, s);
+  return a.ckpt ? launch_cs<V, SP, MAXS, true, 1>(a, s) : launch_cs<V, SP, MAXS, false, 1>(a, s);
 }
 
 }  // namespace
@@ -434,9 +437,9 @@ bool fwd_cs_supported(const ScanArgs &a) {
 
 cudaError_t launch_fwd_bf16_cs(const ScanArgs &a, cudaStream_t s) {
   switch (a.V) {
-    case 32: return launch_cs_v<32, 4>(a, s);
-    case 64: return launch_cs_v<64, 4>(a, s);
-    case 128: return launch_cs_v<128, 2>(a, s);
+    case 32: return launch_cs_v<32, 2, 4>(a, s);
+    case 64: return a.KCf <= 16 ? launch_cs_v<64, 4, 1>(a, s) : launch_cs_v<64, 2, 4>(a, s);
+    case 128: return launch_cs_v<128, 4, 2>(a, s);
     default: return cudaErrorInvalidValue;
   }
 }
