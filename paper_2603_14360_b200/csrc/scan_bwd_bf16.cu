@@ -128,6 +128,8 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
   constexpr bool kWInSmem = V > 64;
   // roles coincide with warpgroups only in this shape (4 + 4 + 4 + 1 warps), the one that needs it
   constexpr bool kRebalance = bwd_rebalance<V, NWC>();
+  // packed fp32x2 element-wise arithmetic where it measured faster (elsewhere its register pairs spill)
+  constexpr bool kPacked = V <= 32 || (V == 64 && NWC == 4);
   constexpr int NSET = V == 128 ? 1 : (KT >= 2 ? 2 : 1);   // accumulator sets of the state x W product, as in the forward kernel
   extern __shared__ __align__(128) unsigned char smem[];
 
@@ -235,8 +237,16 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
 #pragma unroll
         for (int x = 0; x < SEG / 4; ++x) {
           const float4 v4 = lds128(sl + 4u * (L.oV + s * V + SEG * c + 4 * x));
-          P[0][2 * x][0] = k0 * v4.x; P[0][2 * x][1] = k0 * v4.y; P[0][2 * x][2] = k1 * v4.x; P[0][2 * x][3] = k1 * v4.y;
-          P[0][2 * x + 1][0] = k0 * v4.z; P[0][2 * x + 1][1] = k0 * v4.w; P[0][2 * x + 1][2] = k1 * v4.z; P[0][2 * x + 1][3] = k1 * v4.w;
+          if constexpr (kPacked) {   // packed fp32 pairs: one instruction per two products
+            const float2 k02 = make_float2(k0, k0), k12 = make_float2(k1, k1);
+            const float2 a0 = __fmul2_rn(k02, make_float2(v4.x, v4.y)), a1 = __fmul2_rn(k12, make_float2(v4.x, v4.y));
+            const float2 b0 = __fmul2_rn(k02, make_float2(v4.z, v4.w)), b1 = __fmul2_rn(k12, make_float2(v4.z, v4.w));
+            P[0][2 * x][0] = a0.x; P[0][2 * x][1] = a0.y; P[0][2 * x][2] = a1.x; P[0][2 * x][3] = a1.y;
+            P[0][2 * x + 1][0] = b0.x; P[0][2 * x + 1][1] = b0.y; P[0][2 * x + 1][2] = b1.x; P[0][2 * x + 1][3] = b1.y;
+          } else {
+            P[0][2 * x][0] = k0 * v4.x; P[0][2 * x][1] = k0 * v4.y; P[0][2 * x][2] = k1 * v4.x; P[0][2 * x][3] = k1 * v4.y;
+            P[0][2 * x + 1][0] = k0 * v4.z; P[0][2 * x + 1][1] = k0 * v4.w; P[0][2 * x + 1][2] = k1 * v4.z; P[0][2 * x + 1][3] = k1 * v4.w;
+          }
         }
 #pragma unroll
         for (int kt = 0; kt < KT; ++kt) {
@@ -260,12 +270,25 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
           for (int u = 0; u < 2; ++u) {
             const int nt = 2 * x + u;
             float z[4];
+            if constexpr (kPacked) {
 #pragma unroll
-            for (int r = 0; r < 4; ++r) {
-              float xin = P[0][nt][r];
-              if constexpr (NSET == 2) xin += P[1][nt][r];
-              z[r] = tanh_approx(xin);
-              H[nt][r] = fmaf(f, H[nt][r] - z[r], z[r]);
+              for (int h = 0; h < 2; ++h) {
+                float2 xin = make_float2(P[0][nt][2 * h], P[0][nt][2 * h + 1]);
+                if constexpr (NSET == 2) xin = __fadd2_rn(xin, make_float2(P[1][nt][2 * h], P[1][nt][2 * h + 1]));
+                const float2 z2 = make_float2(tanh_approx(xin.x), tanh_approx(xin.y));
+                const float2 d2 = __ffma2_rn(z2, make_float2(-1.f, -1.f), make_float2(H[nt][2 * h], H[nt][2 * h + 1]));
+                const float2 h2 = __ffma2_rn(make_float2(f, f), d2, z2);
+                z[2 * h] = z2.x; z[2 * h + 1] = z2.y;
+                H[nt][2 * h] = h2.x; H[nt][2 * h + 1] = h2.y;
+              }
+            } else {
+#pragma unroll
+              for (int r = 0; r < 4; ++r) {
+                float xin = P[0][nt][r];
+                if constexpr (NSET == 2) xin += P[1][nt][r];
+                z[r] = tanh_approx(xin);
+                H[nt][r] = fmaf(f, H[nt][r] - z[r], z[r]);
+              }
             }
             zw[2 * u] = pack_f16(z[0], z[1]);
             zw[2 * u + 1] = pack_f16(z[2], z[3]);
@@ -361,6 +384,7 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
           matvec(hn, dyp, dqd);
         }
         float df = 0.f;
+        float2 df2 = make_float2(0.f, 0.f);   // packed path: even and odd elements summed apart
         uint32_t xp[NT][2];   // dX as bf16 pairs: the A operand of dX W^T and the tile of the dW warps
 #pragma unroll
         for (int x = 0; x < SEG / 4; ++x) {
@@ -375,19 +399,35 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
             const float2 ha = unpack_bf16(hp[nt][0]), hb = unpack_bf16(hp[nt][1]);
             const float z[4] = {za.x, za.y, zb.x, zb.y}, hprev[4] = {ha.x, ha.y, hb.x, hb.y};
             float dX[4];
+            if constexpr (kPacked) {
+              const float2 dy2 = make_float2(dyv[2 * u], dyv[2 * u + 1]);
 #pragma unroll
-            for (int r = 0; r < 4; ++r) {
-              const float dyc = dyv[2 * u + (r & 1)];
-              const float qr = (r & 2) ? q1 : q0;
-              const float Gv = fmaf(qr, dyc, Cg[nt][r]);        // G = C + q dy^T
-              df = fmaf(Gv, hprev[r] - z[r], df);               // df = sum G (.) (H_{t-1} - Z)
-              dX[r] = omf * Gv * fmaf(-z[r], z[r], 1.f);        // through the gate and tanh
-              Cg[nt][r] = f * Gv;                               // gated path into H_{t-1}
+              for (int h = 0; h < 2; ++h) {
+                const float2 z2 = make_float2(z[2 * h], z[2 * h + 1]), hp2 = make_float2(hprev[2 * h], hprev[2 * h + 1]);
+                const float qh = h ? q1 : q0;
+                const float2 G2 = __ffma2_rn(make_float2(qh, qh), dy2, make_float2(Cg[nt][2 * h], Cg[nt][2 * h + 1]));   // G = C + q dy^T
+                df2 = __ffma2_rn(G2, __ffma2_rn(z2, make_float2(-1.f, -1.f), hp2), df2);                                    // df = sum G (.) (H_{t-1} - Z)
+                const float2 x2 = __fmul2_rn(__fmul2_rn(make_float2(-omf, -omf), G2), __ffma2_rn(z2, z2, make_float2(-1.f, -1.f)));   // (1-f) G (1 - Z^2)
+                const float2 c2 = __fmul2_rn(make_float2(f, f), G2);                                                        // gated path into H_{t-1}
+                dX[2 * h] = x2.x; dX[2 * h + 1] = x2.y;
+                Cg[nt][2 * h] = c2.x; Cg[nt][2 * h + 1] = c2.y;
+              }
+            } else {
+#pragma unroll
+              for (int r = 0; r < 4; ++r) {
+                const float dyc = dyv[2 * u + (r & 1)];
+                const float qr = (r & 2) ? q1 : q0;
+                const float Gv = fmaf(qr, dyc, Cg[nt][r]);        // G = C + q dy^T
+                df = fmaf(Gv, hprev[r] - z[r], df);               // df = sum G (.) (H_{t-1} - Z)
+                dX[r] = omf * Gv * fmaf(-z[r], z[r], 1.f);        // through the gate and tanh
+                Cg[nt][r] = f * Gv;                               // gated path into H_{t-1}
+              }
             }
             xp[nt][0] = pack_bf16(dX[0], dX[1]);
             xp[nt][1] = pack_bf16(dX[2], dX[3]);
           }
         }
+        if constexpr (kPacked) df = df2.x + df2.y;
         // hand dX to the dW warps
         const int xb = nstep & 1;
         if (nstep >= 2 && !mbar_wait(&dx_free[xb], ((nstep >> 1) - 1) & 1)) { report_timeout(a.dev_status); return; }
