@@ -130,7 +130,7 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
   constexpr bool kRebalance = bwd_rebalance<V, NWC>();
   // packed fp32x2 element-wise arithmetic where it measured faster (elsewhere its register pairs spill)
   constexpr bool kPacked = V <= 32 || (V == 64 && NWC == 4);
-  constexpr int NSET = V == 128 ? 1 : (KT >= 2 ? 2 : 1);   // accumulator sets of the state x W product, as in the forward kernel
+  constexpr int NSET = 1;   // accumulator sets of the state x W product, as in the forward kernel
   extern __shared__ __align__(128) unsigned char smem[];
 
   const int K = a.K, N = a.N, T = a.T, C = a.C, nch = a.nchunks;
