@@ -26,7 +26,7 @@ constexpr int kBarrierBytes = 64;
 template <int V>
 struct CsSmem {
   // Per stage (floats): q [TC][K], k [TC][K], v [TC][V], f [TC], ypart [TC][K/16][V]
-  __host__ __device__ static int stage_floats(int K, int TC) { return TC * (2 * K + V + 1 + (K / 16) * V); }
+  __host__ __device__ static constexpr int stage_floats(int K, int TC) { return TC * (2 * K + V + 1 + (K / 16) * V); }
   __host__ __device__ static constexpr int tc() { return V >= 128 ? 8 : 16; }
   // fragment exchange: [2 parities][K/16 slabs][V/16 k-tiles (part-major)][32 lanes] x 16 bytes
   __host__ __device__ static int xchg_bytes(int K) { return 2 * (K / 16) * (V / 16) * 32 * 16; }
@@ -39,8 +39,8 @@ struct CsSmem {
 template <int VP>
 __host__ __device__ constexpr int part_col(int m) { return (VP / 4) * ((m & 7) >> 1) + 2 * (m >> 3) + (m & 1); }
 
-template <int V, int SP, int MAXS, bool CKPT, int OCC>
-__global__ void __launch_bounds__((SP * MAXS + 1) * 32, OCC) fwd_bf16_cs_kernel(ScanArgs a) {
+template <int V, int SP, int NW, bool CKPT, int OCC>
+__global__ void __launch_bounds__((SP * NW + 1) * 32, OCC) fwd_bf16_cs_kernel(ScanArgs a) {
   constexpr int VH = V / SP;         // columns of a part
   constexpr int NTH = VH / 8;        // accumulator tiles of a warp
   constexpr int KT = V / 16;         // k-tiles of the product
@@ -48,15 +48,16 @@ __global__ void __launch_bounds__((SP * MAXS + 1) * 32, OCC) fwd_bf16_cs_kernel(
   constexpr int KTP = KT - KTH;      // k-tiles it receives
   constexpr int SEGH = VH / 4;       // adjacent memory columns per thread
   constexpr int TC = CsSmem<V>::tc();
+  constexpr int kUnroll = 4;         // steps per iteration of the stage loop
   extern __shared__ __align__(16) unsigned char smem_raw[];
 
-  const int Kf = a.K, K = a.KCf, N = a.N, T = a.T;   // rows of the whole state / of this CTA's slab group
+  constexpr int K = 16 * NW;              // rows of this CTA's slab group (NW slabs of 16 rows): a.KCf
+  const int Kf = a.K, N = a.N, T = a.T;   // rows of the whole state
   const int RS = Kf / K;
-  const int NW = K >> 4;                               // 16-row slabs of this CTA
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int bn = blockIdx.x / RS, rs = blockIdx.x % RS, b = bn / N, n = bn % N;
   const int rbase = rs * K;
-  const int stage_floats = CsSmem<V>::stage_floats(K, TC);
+  constexpr int stage_floats = CsSmem<V>::stage_floats(K, TC);
 
   uint64_t *full = reinterpret_cast<uint64_t *>(smem_raw);  // [kStages]
   uint64_t *done = full + kStages;                          // [kStages]
@@ -355,7 +356,7 @@ __global__ void __launch_bounds__((SP * MAXS + 1) * 32, OCC) fwd_bf16_cs_kernel(
   };
   const uint32_t stages_sa = smem_u32(stages);
   auto stage_sa = [&](int s) { return stages_sa + 4u * (uint32_t)(s * stage_floats); };
-  const uint32_t oK = 4u * TC * K, oV = 2 * oK, oF = oV + 4u * TC * V, oY = oF + 4u * TC;
+  constexpr uint32_t oK = 4u * TC * K, oV = 2 * oK, oF = oV + 4u * TC * V, oY = oF + 4u * TC;
 
   if (T > 0) {
     if (!mbar_wait(&full[0], 0)) { report_timeout(a.dev_status); return; }
@@ -386,13 +387,25 @@ __global__ void __launch_bounds__((SP * MAXS + 1) * 32, OCC) fwd_bf16_cs_kernel(
       vN = stage_sa(sn) + oV;
     }
     if (len == TC) {
+      // groups of kUnroll steps with compile-time offsets from one base address
 #pragma unroll 1
-      for (int tl = 0; tl < TC - 2; tl += 2) {
-        maybe_checkpoint(2);
-        pair(st, tl, st + oK + 4u * ((tl + 2) * K), st + oV + 4u * ((tl + 2) * V));
+      for (int t0 = 0; t0 < TC - kUnroll; t0 += kUnroll) {
+        const uint32_t sg = st + 4u * (uint32_t)t0;   // unused: offsets below take t0 into account through tl
+        (void)sg;
+#pragma unroll
+        for (int u = 0; u < kUnroll; u += 2) {
+          const int tl = t0 + u;
+          maybe_checkpoint(2);
+          pair(st, tl, st + oK + 4u * ((tl + 2) * K), st + oV + 4u * ((tl + 2) * V));
+        }
       }
-      maybe_checkpoint(2);
-      pair(st, TC - 2, kN, vN);
+#pragma unroll
+      for (int u = 0; u < kUnroll; u += 2) {
+        const int tl = TC - kUnroll + u;
+        maybe_checkpoint(2);
+        if (u + 2 < kUnroll) pair(st, tl, st + oK + 4u * ((tl + 2) * K), st + oV + 4u * ((tl + 2) * V));
+        else pair(st, tl, kN, vN);
+      }
     } else {   // ragged last stage
       int tl = 0;
       for (; tl + 1 < len; tl += 2) {
@@ -413,35 +426,58 @@ __global__ void __launch_bounds__((SP * MAXS + 1) * 32, OCC) fwd_bf16_cs_kernel(
   if (a.hT) store_state(a.hT + bn * KV);
 }
 
-template <int V, int SP, int MAXS, bool CKPT, int OCC>
+template <int V, int SP, int NW, bool CKPT, int OCC>
 cudaError_t launch_cs(const ScanArgs &a, cudaStream_t s) {
-  const size_t smem = CsSmem<V>::bytes(a.KCf);
-  cudaError_t e = cudaFuncSetAttribute(fwd_bf16_cs_kernel<V, SP, MAXS, CKPT, OCC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const size_t smem = CsSmem<V>::bytes(16 * NW);
+  cudaError_t e = cudaFuncSetAttribute(fwd_bf16_cs_kernel<V, SP, NW, CKPT, OCC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  fwd_bf16_cs_kernel<V, SP, MAXS, CKPT, OCC><<<a.B * a.N * (a.K / a.KCf), (SP * (a.KCf / 16) + 1) * 32, smem, s>>>(a);
+  fwd_bf16_cs_kernel<V, SP, NW, CKPT, OCC><<<a.B * a.N * (a.K / (16 * NW)), (SP * NW + 1) * 32, smem, s>>>(a);
   return cudaGetLastError();
 }
 
-template <int V, int SP, int MAXS>
+template <int V, int SP, int NW>
 cudaError_t launch_cs_v(const ScanArgs &a, cudaStream_t s) {
-  return a.ckpt ? launch_cs<V, SP, MAXS, true, 1>(a, s) : launch_cs<V, SP, MAXS, false, 1>(a, s);
+  return a.ckpt ? launch_cs<V, SP, NW, true, 1>(a, s) : launch_cs<V, SP, NW, false, 1>(a, s);
 }
 
 }  // namespace
 
-// slabs per CTA this variant supports for a V: the register file holds (2 * slabs + 1) warps
+// slabs per CTA this variant supports for a V: the register file holds (parts * slabs + 1) warps
 bool fwd_cs_supported(const ScanArgs &a) {
   if (a.V == 128) return a.KCf <= 32;
   return (a.V == 32 || a.V == 64) && a.KCf <= 64;
 }
 
+// The slab count is a template parameter so that every shared-memory offset of a step is a
+// compile-time constant.  Four warps per slab where the CTA would otherwise leave schedulers idle
+// (one slab) and at V = 128 (a quarter of W per warp fits in registers), two elsewhere.
 cudaError_t launch_fwd_bf16_cs(const ScanArgs &a, cudaStream_t s) {
+  const int nw = a.KCf / 16;
   switch (a.V) {
-    case 32: return launch_cs_v<32, 2, 4>(a, s);
-    case 64: return a.KCf <= 16 ? launch_cs_v<64, 4, 1>(a, s) : launch_cs_v<64, 2, 4>(a, s);
-    case 128: return launch_cs_v<128, 4, 2>(a, s);
-    default: return cudaErrorInvalidValue;
+    case 32:
+      switch (nw) {
+        case 1: return launch_cs_v<32, 2, 1>(a, s);
+        case 2: return launch_cs_v<32, 2, 2>(a, s);
+        case 3: return launch_cs_v<32, 2, 3>(a, s);
+        case 4: return launch_cs_v<32, 2, 4>(a, s);
+      }
+      break;
+    case 64:
+      switch (nw) {
+        case 1: return launch_cs_v<64, 4, 1>(a, s);
+        case 2: return launch_cs_v<64, 2, 2>(a, s);
+        case 3: return launch_cs_v<64, 2, 3>(a, s);
+        case 4: return launch_cs_v<64, 2, 4>(a, s);
+      }
+      break;
+    case 128:
+      switch (nw) {
+        case 1: return launch_cs_v<128, 4, 1>(a, s);
+        case 2: return launch_cs_v<128, 4, 2>(a, s);
+      }
+      break;
   }
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace m2rnn
