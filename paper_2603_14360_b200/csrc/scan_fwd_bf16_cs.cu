@@ -39,8 +39,13 @@ struct CsSmem {
 template <int VP>
 __host__ __device__ constexpr int part_col(int m) { return (VP / 4) * ((m & 7) >> 1) + 2 * (m >> 3) + (m & 1); }
 
+// service warps of a CTA: one per scheduler that also hosts chain warps, so that staging does not
+// weigh on a single scheduler (the chain warps of a slab advance in lockstep with the slowest)
+__host__ __device__ constexpr int cs_service_warps(int chain_warps) { return chain_warps < 4 ? chain_warps : 4; }
+
 template <int V, int SP, int NW, bool CKPT, int OCC>
-__global__ void __launch_bounds__((SP * NW + 1) * 32, OCC) fwd_bf16_cs_kernel(ScanArgs a) {
+__global__ void __launch_bounds__((SP * NW + cs_service_warps(SP * NW)) * 32, OCC) fwd_bf16_cs_kernel(ScanArgs a) {
+  constexpr int kSvc = cs_service_warps(SP * NW);
   constexpr int VH = V / SP;         // columns of a part
   constexpr int NTH = VH / 8;        // accumulator tiles of a warp
   constexpr int KT = V / 16;         // k-tiles of the product
@@ -66,7 +71,7 @@ __global__ void __launch_bounds__((SP * NW + 1) * 32, OCC) fwd_bf16_cs_kernel(Sc
 
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(&full[s], 1);
+      mbar_init(&full[s], kSvc);
       mbar_init(&done[s], SP * NW);
     }
     fence_mbar_init();
@@ -77,8 +82,9 @@ __global__ void __launch_bounds__((SP * NW + 1) * 32, OCC) fwd_bf16_cs_kernel(Sc
   const int nchunks = (T + TC - 1) / TC;
   const bool want_y = a.y != nullptr;
 
-  if (warp == SP * NW) {
-    // ------------------------------------------------------------------ service warp
+  if (warp >= SP * NW) {
+    // ------------------------------------------------------------------ service warps
+    const int sw = warp - SP * NW;   // each takes every kSvc-th group of 32 rows of a stage
     const int hq = n / (N / a.Nq), hk = n / (N / a.Nk);
     const float al = a.alpha ? a.alpha[n] : 1.f, be = a.beta ? a.beta[n] : 0.f;
     const __nv_bfloat16 *qg = static_cast<const __nv_bfloat16 *>(a.q);
@@ -100,6 +106,7 @@ __global__ void __launch_bounds__((SP * NW + 1) * 32, OCC) fwd_bf16_cs_kernel(Sc
       float gt = 0.f;
 #pragma unroll
       for (int i = 0; i < kPerLane; ++i) {
+        if (i % kSvc != sw) continue;
         const int x = lane + 32 * i;
         if (x < len * kq8) {
           const int t = x / kq8, j = (x % kq8) * 8;
@@ -111,9 +118,10 @@ __global__ void __launch_bounds__((SP * NW + 1) * 32, OCC) fwd_bf16_cs_kernel(Sc
           rv[i] = *reinterpret_cast<const uint4 *>(vg + ((bt0 + t) * N + n) * V + j);
         }
       }
-      if (lane < len) gt = a.gate[(bt0 + lane) * N + n];
+      if (sw == kSvc - 1 && lane < len) gt = a.gate[(bt0 + lane) * N + n];
 #pragma unroll
       for (int i = 0; i < kPerLane; ++i) {
+        if (i % kSvc != sw) continue;
         const int x = lane + 32 * i;
         if (x < len * kq8) {
           const int t = x / kq8, j = (x % kq8) * 8;
@@ -125,7 +133,7 @@ __global__ void __launch_bounds__((SP * NW + 1) * 32, OCC) fwd_bf16_cs_kernel(Sc
           store8_bf16_as_f32(vS + t * V + j, rv[i]);
         }
       }
-      if (lane < len) fS[lane] = gate_value(a.gate_kind, gt, al, be, nullptr);
+      if (sw == kSvc - 1 && lane < len) fS[lane] = gate_value(a.gate_kind, gt, al, be, nullptr);
       __syncwarp();
       if (lane == 0) mbar_arrive(&full[s]);
     };
@@ -140,7 +148,7 @@ __global__ void __launch_bounds__((SP * NW + 1) * 32, OCC) fwd_bf16_cs_kernel(Sc
         const float *vS = stages + (size_t)s * stage_floats + 2 * TC * K;
         const float *yp = vS + TC * V + TC;
         const int v8 = V / 8;
-        for (int x = lane; x < len * v8; x += 32) {
+        for (int x = lane + 32 * sw; x < len * v8; x += 32 * kSvc) {
           const int t = x / v8, j = (x % v8) * 8;
           float acc[8];
 #pragma unroll
@@ -169,6 +177,8 @@ __global__ void __launch_bounds__((SP * NW + 1) * 32, OCC) fwd_bf16_cs_kernel(Sc
         }
         __syncwarp();
       }
+      // (a service warp reads, for the residual term, only the rows of v that it refills itself:
+      // the two loops split a stage's rows among the service warps in the same way)
       if (ch + kStages < nchunks) fill(ch + kStages);
     }
     return;
@@ -431,7 +441,7 @@ cudaError_t launch_cs(const ScanArgs &a, cudaStream_t s) {
   const size_t smem = CsSmem<V>::bytes(16 * NW);
   cudaError_t e = cudaFuncSetAttribute(fwd_bf16_cs_kernel<V, SP, NW, CKPT, OCC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  fwd_bf16_cs_kernel<V, SP, NW, CKPT, OCC><<<a.B * a.N * (a.K / (16 * NW)), (SP * NW + 1) * 32, smem, s>>>(a);
+  fwd_bf16_cs_kernel<V, SP, NW, CKPT, OCC><<<a.B * a.N * (a.K / (16 * NW)), (SP * NW + cs_service_warps(SP * NW)) * 32, smem, s>>>(a);
   return cudaGetLastError();
 }
 
