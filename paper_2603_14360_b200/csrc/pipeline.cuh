@@ -33,13 +33,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
 }
 
 // Warp-collective bounded wait for the phase with the given parity.  Returns false for the
-// whole warp if the limit runs out (roughly a second), never spins for ever.
-constexpr uint32_t kWaitLimit = 1u << 22;
+// whole warp if the limit runs out (about a second of SM clocks), never spins for ever.
+// kSleepNs > 0: for waits that are expected to be long and whose end nobody is waiting for (a
+// staging warp far ahead of its consumers): the polls of a tight loop would take issue slots
+// from the warps that do the work.
+constexpr long long kWaitCycles = 1ll << 31;
+template <uint32_t kSleepNs = 0>
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
   bool ok = mbar_try_wait(bar, parity);
-  for (uint32_t it = 0; !ok && it < kWaitLimit; ++it) {
-    if (it > 64) __nanosleep(it > 4096 ? 256 : 32);
-    ok = mbar_try_wait(bar, parity);
+  if (!ok) {
+    const long long t0 = clock64();
+    uint32_t it = 0;
+    do {
+      if constexpr (kSleepNs > 0) __nanosleep(kSleepNs);
+      else if (++it > 64) __nanosleep(32);
+      ok = mbar_try_wait(bar, parity);
+    } while (!ok && clock64() - t0 < kWaitCycles);
   }
   return __all_sync(0xffffffffu, ok);
 }

@@ -652,12 +652,12 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
     };
     if (is_loader) {
       for (int j = 0; j < nch; ++j) {   // runs up to kRing chunks ahead of the writer
-        if (j >= kRing && !mbar_wait(&slot_free[j & (kRing - 1)], ((j / kRing) - 1) & 1)) { report_timeout(a.dev_status); return; }
+        if (j >= kRing && !mbar_wait<1000>(&slot_free[j & (kRing - 1)], ((j / kRing) - 1) & 1)) { report_timeout(a.dev_status); return; }
         fill(j);
       }
     } else {
       for (int j = 0; j < nch; ++j) {
-        if (!mbar_wait(&out_full[j & (kRing - 1)], (j / kRing) & 1)) { report_timeout(a.dev_status); return; }
+        if (!mbar_wait<1000>(&out_full[j & (kRing - 1)], (j / kRing) & 1)) { report_timeout(a.dev_status); return; }
         flush(j);
         __syncwarp();
         if (lane == 0) mbar_arrive(&slot_free[j & (kRing - 1)]);

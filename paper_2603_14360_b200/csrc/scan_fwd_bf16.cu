@@ -150,7 +150,7 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
     for (int ch = 0; ch < pre; ++ch) fill(ch);
     for (int ch = 0; ch < nchunks; ++ch) {
       const int s = ch % kStages, t0 = ch * TC, len = min(TC, T - t0);
-      if (!mbar_wait(&done[s], (ch / kStages) & 1)) { report_timeout(a.dev_status); return; }
+      if (!mbar_wait<1000>(&done[s], (ch / kStages) & 1)) { report_timeout(a.dev_status); return; }
       if (want_y) {
         // y[t][col] = sum over compute warps of their partials (+ w_r (.) v), 8 columns per lane
         const float *vS = stages + (size_t)s * stage_floats + 2 * TC * K;
