@@ -2,12 +2,14 @@
 //
 // At decode time the K rows of every (b,n) state are independent rows of one product per head:
 // [B*K, V] x [V, V].  A CTA stacks the states of 128/K units of one head into an M = 128 tile and
-// runs H W as tcgen05.mma (kind::f16, bf16 operands from shared memory, fp32 accumulator in tensor
+// runs H W as tcgen05.mma (kind::tf32, operands from shared memory, fp32 accumulator in tensor
 // memory), which leaves the SM's issue slots and register file to the streaming part of the step:
 //   - the states of the next task arrive by TMA (cp.async.bulk.tensor, 32-column boxes landing in
 //     128-byte-swizzled rows, completion on an mbarrier) while the current task is computed;
-//   - all warps convert the staged fp32 rows to the bf16, 128-byte-swizzled K-major A tile;
-//   - one thread issues the V/16 MMAs and commits them to an mbarrier;
+//   - the staged fp32 tile is already the canonical K-major 128-byte-swizzled layout of a 32-bit
+//     operand, so it is the A operand as it stands (the tensor core reads it as tf32, which keeps
+//     three more mantissa bits of the state than a bf16 copy would, and no conversion pass runs);
+//   - one thread issues the V/8 MMAs and commits them to an mbarrier;
 //   - every thread then owns one state row and half of its columns: tcgen05.ld, + k_i v^T, tanh,
 //     gate against the staged fp32 row, write H_t back in place (global) and into the stage;
 //   - the readout y = H_t^T q is a column sum over the stage.
@@ -42,9 +44,9 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int x, int 
                ::"l"(map), "r"(x), "r"(y), "r"(src_sa) : "memory");
 }
 
-// Shared-memory matrix descriptor of a K-major bf16 operand in the 128-byte-swizzled canonical
-// layout: rows of 64 elements (128 bytes), groups of 8 rows 1024 bytes apart, 16-byte chunks of a
-// row XOR-ed with the row index modulo 8.
+// Shared-memory matrix descriptor of a K-major operand in the 128-byte-swizzled canonical
+// layout: rows of 128 bytes (32 tf32 elements), groups of 8 rows 1024 bytes apart, 16-byte chunks
+// of a row XOR-ed with the row index modulo 8.
 //   bits  0-13 start address >> 4     bits 32-45 stride between 8-row groups >> 4
 //   bits 16-29 leading offset >> 4 (not used by swizzled K-major layouts)
 //   bits 46-47 descriptor version 1   bits 61-63 swizzle mode (2 = 128 bytes)
@@ -52,14 +54,15 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t sa) {
   return (uint64_t)((sa & 0x3ffffu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
          ((uint64_t)2 << 61);
 }
-// Instruction descriptor of kind::f16: fp32 accumulator (bits 4-5 = 1), bf16 A and B (bits 7-9 and
-// 10-12 = 1), both K-major (bits 15, 16 = 0), N >> 3 in bits 17-22, M >> 4 in bits 24-28.
-__host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+// Instruction descriptor of kind::tf32: fp32 accumulator (bits 4-5 = 1), tf32 A and B (bits 7-9 and
+// 10-12 = 2), both K-major (bits 15, 16 = 0), N >> 3 in bits 17-22, M >> 4 in bits 24-28.
+__host__ __device__ constexpr uint32_t umma_idesc_tf32(int M, int N) {
+  return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+// D[128 x N] (+)= A[128 x 8] B[N x 8]^T, both operands tf32
+__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint64_t *bar) {
@@ -88,11 +91,10 @@ __device__ __forceinline__ uint32_t stage_off(int i, int j) {
 
 template <int V>
 struct TcSmem {
-  static constexpr uint32_t a_bytes = kM * V * 2;             // A tile: V/64 blocks of [128 rows][128 bytes]
-  static constexpr uint32_t b_bytes = V * V * 2;              // B tile (W^T): V/64 blocks of [V rows][128 bytes]
-  static constexpr uint32_t stage_bytes = kM * V * 4;
+  static constexpr uint32_t b_bytes = V * V * 4;              // B tile (W^T as fp32): V/32 blocks of [V rows][128 bytes]
+  static constexpr uint32_t stage_bytes = kM * V * 4;         // a stage = the A tile: V/32 blocks of [128 rows][128 bytes]
   // offsets from the 1024-byte aligned base
-  static constexpr uint32_t oA = 0, oB = oA + a_bytes, oStage = oB + b_bytes, oVec = oStage + 2 * stage_bytes;
+  static constexpr uint32_t oB = 0, oStage = oB + b_bytes, oVec = oStage + 2 * stage_bytes;
   // vectors (two buffers, the next task's are fetched a task ahead): k [128], q [128], f [128] per
   // row, v [128/K <= 8][V]; then the warps' readout partials [8][V]
   static constexpr uint32_t vec_floats = 3 * kM + 8 * V;
@@ -114,8 +116,9 @@ __global__ void __launch_bounds__(256, 1) decode_tc_kernel(ScanArgs a, int GPI, 
   float *vecs = reinterpret_cast<float *>(base + S::oVec);
   float *ypart = vecs + 2 * S::vec_floats;                  // [8 warps][V]
   uint64_t *full = reinterpret_cast<uint64_t *>(base + S::oBar);   // [2]
-  uint64_t *mma_done = full + 2;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(mma_done + 1);
+  uint64_t *mma_done = full + 2;                                    // [2], one per accumulator
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(mma_done + 2);
+  volatile uint32_t *early_flag = tmem_slot + 1;   // the next task's MMAs are already in flight
 
   const int K = a.K, N = a.N, B = a.B;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -128,12 +131,14 @@ __global__ void __launch_bounds__(256, 1) decode_tc_kernel(ScanArgs a, int GPI, 
   if (tid == 0) {
     mbar_init(&full[0], 1);
     mbar_init(&full[1], 1);
-    mbar_init(mma_done, 1);
+    mbar_init(&mma_done[0], 1);
+    mbar_init(&mma_done[1], 1);
+    *early_flag = 0u;
     fence_mbar_init();
   }
-  if (warp == 0) {   // V columns of tensor memory for the accumulator
+  if (warp == 0) {   // 2 x V columns of tensor memory: two accumulators, used by alternate tasks
     __syncwarp();
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(V) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(2 * V) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -205,57 +210,28 @@ __global__ void __launch_bounds__(256, 1) decode_tc_kernel(ScanArgs a, int GPI, 
     park_vecs(0, first);
   }
 
-  constexpr uint32_t idesc = umma_idesc_bf16(kM, V);
+  constexpr uint32_t idesc = umma_idesc_tf32(kM, V);
+  // the V/8 MMAs of the task whose states sit in stage st, into accumulator st (one thread)
+  auto issue_mmas = [&](int st) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t a_sa = base_sa + S::oStage + (uint32_t)st * S::stage_bytes;
+#pragma unroll
+    for (int ks = 0; ks < V / 8; ++ks) {
+      // 8 elements (32 bytes) per step inside a 128-byte block, then the next block
+      const uint32_t koff = (uint32_t)(ks / 4) * 128u * kM + (uint32_t)(ks % 4) * 32u;
+      const uint32_t koffb = (uint32_t)(ks / 4) * 128u * V + (uint32_t)(ks % 4) * 32u;
+      umma_tf32(tmem_base + (uint32_t)st * V, umma_desc_sw128(a_sa + koff), umma_desc_sw128(base_sa + S::oB + koffb), idesc, ks > 0);
+    }
+    umma_commit(&mma_done[st]);
+  };
   int cur_head = -1, it = 0;
   bool failed = false;
+  bool early = false;   // this task's MMAs were issued during the previous one
   for (long task = t_begin; task < t_end; ++task, ++it) {
     const int n = (int)(task / tasks_per_head), b0 = (int)(task % tasks_per_head) * GPI;
     const int rows = min(GPI, B - b0) * K;     // live rows of the tile
     VecRegs next;
     if (task + 1 < t_end) fetch_vecs(task + 1, next);   // lands while this task is computed
-    if (n != cur_head) {
-      // B tile = W_n^T, K-major: row j holds W[:, j]; element (j, l) sits in block l/64 at
-      // row j, 16-byte chunk ((l%64)/8) ^ (j%8), like the A tile
-      const uint16_t *w = reinterpret_cast<const uint16_t *>(a.W) + (size_t)n * V * V;
-      for (int x = tid; x < V * V / 8; x += blockDim.x) {
-        const int j = x % V, l0 = (x / V) * 8;
-        uint32_t p[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) p[e] = (uint32_t)w[(l0 + 2 * e) * V + j] | ((uint32_t)w[(l0 + 2 * e + 1) * V + j] << 16);
-        const uint32_t off = S::oB + (uint32_t)(l0 / 64) * (V * 128) + (uint32_t)j * 128 + ((((l0 % 64) / 8) ^ (j & 7)) << 4);
-        *reinterpret_cast<uint4 *>(base + off) = make_uint4(p[0], p[1], p[2], p[3]);
-      }
-      cur_head = n;
-    }
-    const float *kvec = vecs + (size_t)(it & 1) * S::vec_floats, *qvec = kvec + kM, *fvec = qvec + kM, *vvec = fvec + kM;
-    if (!__syncthreads_and(mbar_wait(&full[it & 1], (it >> 1) & 1))) { failed = true; break; }
-    float *sg = stage + (size_t)(it & 1) * (kM * V);
-
-    // fp32 rows -> bf16 A tile (rows past the live ones are zero: their results are never used)
-    for (int x = tid; x < kM * V / 8; x += blockDim.x) {
-      const int i = x / (V / 8), ch = x % (V / 8);
-      uint4 o = make_uint4(0u, 0u, 0u, 0u);
-      if (i < rows) {
-        const float4 lo = *reinterpret_cast<const float4 *>(sg + stage_off<V>(i, 8 * ch));
-        const float4 hi = *reinterpret_cast<const float4 *>(sg + stage_off<V>(i, 8 * ch + 4));
-        o = make_uint4(pack_bf16(lo.x, lo.y), pack_bf16(lo.z, lo.w), pack_bf16(hi.x, hi.y), pack_bf16(hi.z, hi.w));
-      }
-      const uint32_t off = S::oA + (uint32_t)(ch / 8) * (kM * 128) + (uint32_t)i * 128 + (((ch & 7) ^ (i & 7)) << 4);
-      *reinterpret_cast<uint4 *>(base + off) = o;
-    }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the tensor core
-    __syncthreads();
-    if (tid == 0) {
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-#pragma unroll
-      for (int ks = 0; ks < V / 16; ++ks) {
-        // 16 elements (32 bytes) per step inside a 128-byte block, then the next block
-        const uint32_t koff = (uint32_t)(ks / 4) * 128u * kM + (uint32_t)(ks % 4) * 32u;
-        const uint32_t koffb = (uint32_t)(ks / 4) * 128u * V + (uint32_t)(ks % 4) * 32u;
-        umma_bf16(tmem_base, umma_desc_sw128(base_sa + S::oA + koff), umma_desc_sw128(base_sa + S::oB + koffb), idesc, ks > 0);
-      }
-      umma_commit(mma_done);
-    }
     if (warp == 7 && task + 1 < t_end) {
       // the other stage: its rows were stored by the last task (wait until that store has read
       // them) and written through the generic proxy before; the loads write through the async proxy
@@ -263,7 +239,27 @@ __global__ void __launch_bounds__(256, 1) decode_tc_kernel(ScanArgs a, int GPI, 
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       prefetch(task + 1, (it + 1) & 1);
     }
-    if (!__syncthreads_and(mbar_wait(mma_done, it & 1))) { failed = true; break; }
+    if (n != cur_head) {
+      // B tile = W_n^T widened to fp32, K-major: row j holds W[:, j]; element (j, l) sits in block
+      // l/32 at row j, 16-byte chunk ((l%32)/4) ^ (j%8), like the rows of a stage
+      const uint16_t *w = reinterpret_cast<const uint16_t *>(a.W) + (size_t)n * V * V;
+      for (int x = tid; x < V * V / 4; x += blockDim.x) {
+        const int j = x % V, l0 = (x / V) * 4;
+        uint32_t p[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) p[e] = (uint32_t)w[(l0 + e) * V + j] << 16;
+        const uint32_t off = S::oB + (uint32_t)(l0 / 32) * (V * 128) + (uint32_t)j * 128 + ((((l0 % 32) / 4) ^ (j & 7)) << 4);
+        *reinterpret_cast<uint4 *>(base + off) = make_uint4(p[0], p[1], p[2], p[3]);
+      }
+      cur_head = n;
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the tensor core
+    }
+    const float *kvec = vecs + (size_t)(it & 1) * S::vec_floats, *qvec = kvec + kM, *fvec = qvec + kM, *vvec = fvec + kM;
+    // the task's states have landed (this barrier also orders the B tile's writes before the MMAs)
+    if (!__syncthreads_and(mbar_wait(&full[it & 1], (it >> 1) & 1))) { failed = true; break; }
+    float *sg = stage + (size_t)(it & 1) * (kM * V);
+    if (tid == 0 && !early) issue_mmas(it & 1);
+    if (!__syncthreads_and(mbar_wait(&mma_done[it & 1], (it >> 1) & 1))) { failed = true; break; }
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 
     // epilogue: thread = (row i, column half)
@@ -276,7 +272,7 @@ __global__ void __launch_bounds__(256, 1) decode_tc_kernel(ScanArgs a, int GPI, 
 #pragma unroll
       for (int cb = 0; cb < HC / 32; ++cb) {
         float P[32];
-        tmem_ld32(tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(half * HC + 32 * cb), P);
+        tmem_ld32(tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)((it & 1) * V + half * HC + 32 * cb), P);
         if (live) {
 #pragma unroll
           for (int x = 0; x < 8; ++x) {
@@ -298,6 +294,16 @@ __global__ void __launch_bounds__(256, 1) decode_tc_kernel(ScanArgs a, int GPI, 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // H_t in the stage -> visible to the TMA store
     __syncthreads();
+    if (warp == 0) {
+      // The next task's product does not depend on this one: start it now, into the other
+      // accumulator, so that the tensor core works while the readout runs (unless the head
+      // changes, which rebuilds the B tile first).  The outcome reaches every thread through
+      // shared memory at the next barrier.
+      bool go = task + 1 < t_end && (int)((task + 1) / tasks_per_head) == n;
+      if (go) go = mbar_wait(&full[(it + 1) & 1], ((it + 1) >> 1) & 1);
+      if (go && lane == 0) issue_mmas((it + 1) & 1);
+      if (lane == 0) *early_flag = go ? 1u : 0u;
+    }
     if (warp == 7) {   // H_t back to global memory, in place, one box per unit and 32-column block
       const int units = rows / K;
       const uint32_t src0 = base_sa + S::oStage + (uint32_t)(it & 1) * S::stage_bytes;
@@ -311,18 +317,22 @@ __global__ void __launch_bounds__(256, 1) decode_tc_kernel(ScanArgs a, int GPI, 
     // (all of one unit, K >= 16), a lane takes the columns lane, lane+32, ...; then the warps of a
     // unit are added.
     {
-      float acc[V / 32];
+      // lane = (row group, 32-column block, 16-byte chunk): one 128-byte row of a block per 8 lanes
+      constexpr int NB = V / 32, RG = 4 / NB;
+      const int c8 = lane & 7, m = (lane >> 3) % NB, rg = lane / (8 * NB);
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-      for (int m = 0; m < V / 32; ++m) acc[m] = 0.f;
-#pragma unroll
-      for (int rr = 0; rr < 16; ++rr) {
-        const int i = 16 * warp + rr;
+      for (int rr = 0; rr < 16 / RG; ++rr) {
+        const int i = 16 * warp + rg * (16 / RG) + rr;
         const float qi = qvec[i];
-#pragma unroll
-        for (int m = 0; m < V / 32; ++m) acc[m] = fmaf(qi, sg[stage_off<V>(i, lane + 32 * m)], acc[m]);
+        const float4 h4 = *reinterpret_cast<const float4 *>(sg + (uint32_t)m * (kM * 32) + (uint32_t)i * 32 + (uint32_t)((c8 ^ (i & 7)) << 2));
+        acc.x = fmaf(qi, h4.x, acc.x); acc.y = fmaf(qi, h4.y, acc.y); acc.z = fmaf(qi, h4.z, acc.z); acc.w = fmaf(qi, h4.w, acc.w);
       }
-#pragma unroll
-      for (int m = 0; m < V / 32; ++m) ypart[warp * V + lane + 32 * m] = acc[m];
+      if constexpr (RG == 2) {
+        acc.x += __shfl_xor_sync(0xffffffffu, acc.x, 16); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, 16);
+        acc.z += __shfl_xor_sync(0xffffffffu, acc.z, 16); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, 16);
+      }
+      if (rg == 0) *reinterpret_cast<float4 *>(ypart + warp * V + 32 * m + 4 * c8) = acc;
     }
     __syncthreads();
     for (int x = tid; x < GPI * V; x += blockDim.x) {
@@ -335,6 +345,7 @@ __global__ void __launch_bounds__(256, 1) decode_tc_kernel(ScanArgs a, int GPI, 
       }
     }
     if (task + 1 < t_end) park_vecs((it + 1) & 1, next);
+    early = *early_flag != 0u;   // written before the barrier in front of the final sum
     __syncthreads();   // stage, vectors and tiles are free again
   }
   if (warp == 7) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // the last stores
@@ -343,7 +354,7 @@ __global__ void __launch_bounds__(256, 1) decode_tc_kernel(ScanArgs a, int GPI, 
   __syncthreads();
   if (warp == 0) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(V) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * V) : "memory");
   }
 }
 
