@@ -38,7 +38,7 @@ SM_COUNT, SM_HZ = 148, 1.965e9
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (bptt_bf16: captured at T=512, scaled by 8 -- traffic is per
 # token-head).  None for workloads without a capture of the current kernel.
-NCU_TRAFFIC_BYTES = {"fwd_bf16": 119.4e6, "bptt_bf16": 8 * 658.5e6, "decode": 2.108e9}
+NCU_TRAFFIC_BYTES = {"fwd_bf16": 117.4e6, "bptt_bf16": 8 * 658.5e6, "decode": 2.108e9}
 
 
 def workload_pass(name: str) -> str:
