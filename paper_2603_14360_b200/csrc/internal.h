@@ -59,7 +59,7 @@ cudaError_t launch_bwd_f32(const ScanArgs &a, cudaStream_t s);
 // bf16 tensor-core path
 cudaError_t launch_fwd_bf16(const ScanArgs &a, cudaStream_t s);     // scan_fwd_bf16.cu: picks a variant
 bool fwd_cs_supported(const ScanArgs &a);                            // scan_fwd_bf16_cs.cu
-cudaError_t launch_fwd_bf16_cs(const ScanArgs &a, cudaStream_t s);  // scan_fwd_bf16_cs.cu: two warps per 16-row slab
+cudaError_t launch_fwd_bf16_cs(const ScanArgs &a, cudaStream_t s);  // scan_fwd_bf16_cs.cu: two or four warps per 16-row slab
 cudaError_t launch_bwd_bf16(const ScanArgs &a, cudaStream_t s);     // scan_bwd_bf16.cu
 cudaError_t launch_decode_bf16(const ScanArgs &a, cudaStream_t s);  // decode_bf16.cu: picks a kernel
 bool decode_tc_supported(const ScanArgs &a);                         // decode_tc_bf16.cu

@@ -1,17 +1,19 @@
 // bf16 tensor-core forward scan (Algorithm 1), column-split variant, for sm_100a.
 //
-// Same CTA layout, staging and service warp as scan_fwd_bf16.cu, but every 16-row slab of the state
-// is shared by TWO chain warps, each owning half of the V columns.  A warp's step needs the whole
-// slab as the A operand of H W, so the two exchange their freshly packed bf16 fragments through
-// shared memory once per step (one named barrier for the pair).  The exchange hides behind the
-// MMAs a warp can already issue from its own fragments, and the scheduler now holds two chain warps
-// whose stalls interleave -- a single in-order warp per scheduler spends more than half of the step
-// waiting on its own dependency chain.  Each warp also holds only its half of W (V x V/2) in
-// registers, which keeps W out of shared memory up to V = 128.
+// Same CTA layout and staging as scan_fwd_bf16.cu, but every 16-row slab of the state is shared by
+// SP = 2 or 4 chain warps, each owning V/SP of the columns.  A warp's step needs the whole slab as
+// the A operand of H W, so the warps of a slab exchange their freshly packed bf16 fragments
+// through shared memory once per step (one named barrier per slab).  The exchange hides behind
+// the MMAs a warp can already issue from its own fragments.  Each warp holds only its part of W
+// (V x V/SP) in registers, which keeps W out of shared memory up to V = 128 (SP = 4 there).  The
+// slab count NW is a template parameter and four steps form one loop iteration, so that every
+// shared-memory offset of a step is an immediate: the chain warps are bound by the number of
+// instructions they issue per step.  Up to four service warps stage q, k, v and the gate and write
+// y, one per scheduler, so that no scheduler's chain warps fall behind the others.
 //
-// Accumulator element map of warp (slab s, half hf), lane (g = lane/4, c = lane%4):
-//   rows 16s+g and 16s+g+8; MMA column m of the half  <->  memory column hf*V/2 + (V/8)*c' + 2*(m>>3) + (m&1)
-//   with c' = (m&7)>>1, i.e. a thread holds V/8 adjacent columns of two rows.
+// Accumulator element map of warp (slab s, part hf), lane (g = lane/4, c = lane%4):
+//   rows 16s+g and 16s+g+8; MMA column m of the part  <->  memory column hf*V/SP + SEG*c' + 2*(m>>3) + (m&1)
+//   with SEG = V/(4 SP) and c' = (m&7)>>1, i.e. a thread holds SEG adjacent columns of two rows.
 #include "device_common.cuh"
 #include "internal.h"
 #include "mma_tile.cuh"
@@ -291,7 +293,7 @@ __global__ void __launch_bounds__((SP * NW + cs_service_warps(SP * NW)) * 32, OC
       for (int nt = 0; nt < NTH; ++nt) mma_bf16_16816(P[nt], A[i], Wr[KTH + i][nt][0], Wr[KTH + i][nt][1]);
   };
 
-  // One step.  Pc: H_{t-1} W + k_t v_t^T (two partial sums), complete or in flight on entry.
+  // One step.  Pc: H_{t-1} W + k_t v_t^T, complete or in flight on entry.
   // Pn receives the same for step t+1 (after the last step: fed a valid but meaningless row).
   auto step = [&](float (&Pc)[NTH][4], float (&Pn)[NTH][4], float f, uint32_t qrow, uint32_t ydst,
                   uint32_t krow_n, uint32_t vrow_n, int par) {
