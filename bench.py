@@ -285,12 +285,14 @@ def main():
     if pas == "decode":
         state = dev_sets[0]["h0"].clone()
         y1 = torch.empty((B, N, V), dtype=io, device=dev)
+        y_bufs = [y1, torch.empty_like(y1)]
 
-        def step(i, s=None):
+        def step(i, s=None, ob=0):
             s = s or dev_sets[i % ROTATE]
-            binding.m2rnn_decode_step(s["q"], s["k"], s["v"], s["gate"], W, state, gate_kind=cfg.gate_kind, y=y1,
+            binding.m2rnn_decode_step(s["q"], s["k"], s["v"], s["gate"], W, state, gate_kind=cfg.gate_kind, y=y_bufs[ob],
                                       stream=stream)
         out_tensors = [y1]
+        out_sets = [[y_bufs[0]], [y_bufs[1]]]
     else:
         p = binding._params(dev_sets[0]["q"], dev_sets[0]["k"], dev_sets[0]["v"], W, cfg.gate_kind)
         outs = dict(y=torch.empty((B, T, N, V), dtype=io, device=dev),
@@ -311,16 +313,22 @@ def main():
             # fwd, bwd, dW reduce (+ dv and dgate reduces when a state's rows are split over CTAs)
             launches_per_step += 2 + (2 if binding.m2rnn_bwd_row_slab(p) != K else 0)
         ev_mid = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        # a second set of result buffers for the end-to-end leg (results of step i leave the device
+        # while step i+1 computes); the checkpoints never leave and are shared
+        outs_b = [outs, {k: (v if k == "ckpt" else torch.empty_like(v)) for k, v in outs.items()}]
+        gouts_b = [gouts, {k: torch.empty_like(v) for k, v in gouts.items()}] if bwd else [None, None]
+        out_sets = [[t for k, t in outs_b[j].items() if k != "ckpt"] + (list(gouts_b[j].values()) if bwd else [])
+                    for j in range(2)]
 
-        def step(i, s=None, mark=False):
+        def step(i, s=None, mark=False, ob=0):
             s = s or dev_sets[i % ROTATE]
             binding.m2rnn_fwd(s["q"], s["k"], s["v"], s["gate"], W, s["h0"], gate_kind=cfg.gate_kind,
-                              save_ckpt=bwd, out=outs, workspace=fws, stream=stream)
+                              save_ckpt=bwd, out=outs_b[ob], workspace=fws, stream=stream)
             if bwd:
                 if mark:
                     ev_mid[0].record(stream)
                 binding.m2rnn_bwd(s["q"], s["k"], s["v"], s["gate"], W, s["h0"], s["dy"], ckpt=outs["ckpt"],
-                                  gate_kind=cfg.gate_kind, workspace=ws, out=gouts, stream=stream)
+                                  gate_kind=cfg.gate_kind, workspace=ws, out=gouts_b[ob], stream=stream)
                 if mark:
                     ev_mid[1].record(stream)
 
@@ -356,31 +364,60 @@ def main():
     # end to end: host buffers in, host buffers out, every step
     ms_e2e, e2e_steps, h2d, d2h = 0.0, 0, 0, 0
     if not args.no_e2e:
-        host_out = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in out_tensors if t is not outs.get("ckpt")] \
-            if pas != "decode" else [torch.empty(y1.shape, dtype=y1.dtype).pin_memory()]
-        dev_out = [t for t in out_tensors if pas == "decode" or t is not outs.get("ckpt")]
-        stage = {k: torch.empty_like(v) for k, v in dev_sets[0].items()
-                 if isinstance(v, torch.Tensor) and k != "W" and not (pas == "decode" and k == "h0")}
-        h2d = sum(nbytes(t) for t in stage.values())
+        host_out = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in out_sets[0]]
+        # Two device-side input buffers: the copy of step i+1's inputs runs on a stream of its own
+        # while step i computes and its results go back (as an input pipeline of a training or
+        # serving loop would); every timed step still moves its own inputs in and its results out.
+        stages = [{k: torch.empty_like(v) for k, v in dev_sets[0].items()
+                   if isinstance(v, torch.Tensor) and k != "W" and not (pas == "decode" and k == "h0")} for _ in range(2)]
+        h2d = sum(nbytes(t) for t in stages[0].values())
         d2h = sum(nbytes(t) for t in host_out)
+        copy_stream = torch.cuda.Stream(device=dev)
+        back_stream = torch.cuda.Stream(device=dev)
+        landed = [torch.cuda.Event() for _ in range(2)]     # the buffer's inputs are on the device
+        consumed = [torch.cuda.Event() for _ in range(2)]   # the step that read the buffer is done
+        computed = [torch.cuda.Event() for _ in range(2)]   # the step's results are in their buffers
+        copied_back = [torch.cuda.Event() for _ in range(2)]   # ... and have left them
 
-        def e2e_step(i):
-            hs = host_sets[i % ROTATE]
-            for k, t in stage.items():
-                t.copy_(hs[k], non_blocking=True)
-            step(i, s={**stage, "W": W, "h0": stage.get("h0", dev_sets[0].get("h0"))})
-            for h, d_ in zip(host_out, dev_out):
-                h.copy_(d_, non_blocking=True)
+        def issue_h2d(i, first):
+            b = i % 2
+            with torch.cuda.stream(copy_stream):
+                if not first:
+                    copy_stream.wait_event(consumed[b])
+                hs = host_sets[i % ROTATE]
+                for k, t in stages[b].items():
+                    t.copy_(hs[k], non_blocking=True)
+                landed[b].record(copy_stream)
+
+        def e2e_run(n):
+            start = torch.cuda.Event(enable_timing=True)
+            stop = torch.cuda.Event(enable_timing=True)
+            start.record(stream)
+            copy_stream.wait_event(start)
+            issue_h2d(0, True)
+            for i in range(n):
+                b = i % 2
+                if i + 1 < n:
+                    issue_h2d(i + 1, i + 1 < 2)
+                stream.wait_event(landed[b])
+                if i >= 2:
+                    stream.wait_event(copied_back[b])
+                step(i, s={**stages[b], "W": W, "h0": stages[b].get("h0", dev_sets[0].get("h0"))}, ob=b)
+                consumed[b].record(stream)
+                computed[b].record(stream)
+                with torch.cuda.stream(back_stream):
+                    back_stream.wait_event(computed[b])
+                    for h, d_ in zip(host_out, out_sets[b]):
+                        h.copy_(d_, non_blocking=True)
+                    copied_back[b].record(back_stream)
+            stream.wait_stream(back_stream)
+            stop.record(stream)
+            return start, stop
 
         e2e_steps = max(3, min(args.steps, 50))
-        for i in range(3):
-            e2e_step(i)
+        e2e_run(3)
         barrier()
-        ev2 = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
-        ev2[0].record(stream)
-        for i in range(e2e_steps):
-            e2e_step(i)
-        ev2[1].record(stream)
+        ev2 = e2e_run(e2e_steps)
         barrier()
         ms_e2e = ev2[0].elapsed_time(ev2[1])
 
