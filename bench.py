@@ -237,12 +237,16 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--multi-value", action="store_true",
+                    help="run the workload in the multi-value layout (Nq = Nk = 1) instead of multi-head")
     ap.add_argument("--seq-len", type=int, default=0,
                     help="shorten (or lengthen) the workload's T, for profiler captures; the line's workload name says so")
     args = ap.parse_args()
     cfg = CONFIGS[args.workload]
     if args.seq_len and args.workload != "decode":
         cfg = cfg.with_(T=args.seq_len, name=f"{cfg.name}@T={args.seq_len}")
+    if args.multi_value:   # the paper's layout: one q and one k head shared by all N value heads
+        cfg = cfg.with_(Nq=1, Nk=1, name=f"{cfg.name}+multi_value")
     pas = workload_pass(args.workload)
 
     if args.impl == "reference":
@@ -441,7 +445,7 @@ def main():
         alg_bytes = state_bytes + in_bytes + th * V * esz
         achieved = alg_bytes / (ms_step * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if not args.seq_len else None,
+                "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if not (args.seq_len or args.multi_value) else None,
                 "call": "m2rnn_decode_step",
                 "peak_source": f"{peaks['source']} HBM copy", "algorithmic_bytes_per_step": alg_bytes}
     else:
@@ -460,7 +464,7 @@ def main():
         else:
             bound, peak, psrc = "tensor", peaks["tflops_burst"], f"{peaks['source']} cuBLAS bf16 burst"
         roof = {"bound": bound, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if not args.seq_len else None,
+                "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if not (args.seq_len or args.multi_value) else None,
                 "call": "m2rnn_bwd" if bwd else "m2rnn_fwd", "call_ms": call_ms,
                 "peak_source": psrc,
                 "t_tensor_ms": t_tensor * 1e3, "t_hbm_ms": t_hbm * 1e3, "t_mufu_ms": mufu_s * 1e3,
