@@ -22,6 +22,8 @@ SHAPES = [
     (3, 1, 2, 64, 64, 0, 0),      # a single step
     (1, 4, 1, 64, 64, 0, 0),      # exactly one chunk
     (40, 9, 4, 64, 64, 0, 0),     # enough units that a CTA takes all 64 rows
+    (40, 7, 4, 32, 128, 0, 0),    # ... and the 32-row CTAs of V = 128 (W in shared memory)
+    (40, 7, 4, 32, 64, 0, 0),     # two slabs per CTA
 ]
 
 

@@ -36,6 +36,15 @@ def test_shapes_forward(oracle, shape, gate_kind):
     assert max(errs.values()) < 1e-2          # typical error is a few 1e-3: bf16 rounding of H, tanh.approx
 
 
+@pytest.mark.parametrize("K,V", [(32, 32), (48, 32), (64, 32), (32, 64), (48, 64), (64, 64), (32, 128), (96, 64)])
+def test_more_units_than_sms(oracle, K, V):
+    """152 (b, n) units: every CTA keeps a whole state (two to four 16-row slabs per CTA in the
+    column-split kernel, six in the one-warp-per-slab kernel), the launch takes two waves."""
+    cfg = ScanConfig("many", B=38, T=37, N=4, K=K, V=V, gate_mean=1.0, w_scale=0.5, seed=300 + K + V)
+    errs = parity.check_fwd(oracle, cfg)
+    assert max(errs.values()) < 1e-2
+
+
 @pytest.mark.parametrize("K,V", [(16, 16), (64, 64), (128, 128)])
 def test_saturating_inputs(oracle, K, V):
     cfg = ScanConfig("sat", B=2, T=96, N=2, K=K, V=V, dist="saturating", gate_mean=0.0, seed=7)
