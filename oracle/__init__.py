@@ -54,6 +54,10 @@ def load(path: str | None = None) -> ctypes.CDLL:
     lib.m2rnn_ref_bwd.argtypes = [ctypes.POINTER(_Params)] + [_dp] * 17
     lib.m2rnn_ref_decode_step.restype = ctypes.c_int
     lib.m2rnn_ref_decode_step.argtypes = [ctypes.POINTER(_Params)] + [_dp] * 10
+    lib.m2rnn_ref_gated_norm_fwd.restype = ctypes.c_int
+    lib.m2rnn_ref_gated_norm_fwd.argtypes = [ctypes.c_long, ctypes.c_int] + [_dp] * 3 + [ctypes.c_double, ctypes.c_int] + [_dp] * 2
+    lib.m2rnn_ref_gated_norm_bwd.restype = ctypes.c_int
+    lib.m2rnn_ref_gated_norm_bwd.argtypes = [ctypes.c_long, ctypes.c_int] + [_dp] * 3 + [ctypes.c_double, ctypes.c_int] + [_dp] * 4
     return lib
 
 
@@ -159,3 +163,34 @@ def decode_step(q, k, v, gate, W, state, *, gate_kind=GATE_LOGIT, alpha=None, be
     if rc != 0:
         raise RuntimeError(f"m2rnn_ref_decode_step failed: {rc}")
     return y, state
+
+
+def gated_norm_fwd(y, g_in, w, *, eps=0.0, silu=True, lib=None):
+    """out = RMSNorm(y * g) over the last axis flattened with the head axis: y, g_in [..., N, V],
+    w [N*V] -> (out like y, rstd [...])."""
+    lib = lib or _get()
+    y, g_in = _c(y), _c(g_in, y.shape)
+    d = y.shape[-2] * y.shape[-1]
+    w = _c(np.asarray(w).reshape(-1), (d,))
+    tokens = int(np.prod(y.shape[:-2]))
+    out = np.empty(y.shape, np.float64)
+    rstd = np.empty(y.shape[:-2], np.float64)
+    rc = lib.m2rnn_ref_gated_norm_fwd(tokens, d, _p(y), _p(g_in), _p(w), float(eps), int(bool(silu)), _p(out), _p(rstd))
+    if rc != 0:
+        raise RuntimeError(f"m2rnn_ref_gated_norm_fwd failed: {rc}")
+    return out, rstd
+
+
+def gated_norm_bwd(y, g_in, w, dout, *, eps=0.0, silu=True, lib=None):
+    """Backward of gated_norm_fwd -> dict(dy, dg, dw [N*V])."""
+    lib = lib or _get()
+    y, g_in, dout = _c(y), _c(g_in, y.shape), _c(dout, y.shape)
+    d = y.shape[-2] * y.shape[-1]
+    w = _c(np.asarray(w).reshape(-1), (d,))
+    tokens = int(np.prod(y.shape[:-2]))
+    out = dict(dy=np.empty(y.shape), dg=np.empty(y.shape), dw=np.empty((d,)))
+    rc = lib.m2rnn_ref_gated_norm_bwd(tokens, d, _p(y), _p(g_in), _p(w), float(eps), int(bool(silu)), _p(dout),
+                                      _p(out["dy"]), _p(out["dg"]), _p(out["dw"]))
+    if rc != 0:
+        raise RuntimeError(f"m2rnn_ref_gated_norm_bwd failed: {rc}")
+    return out

@@ -252,3 +252,60 @@ int m2rnn_ref_bwd(const m2rnn_ref_params *p, const double *q, const double *k, c
   free(Hs); free(Z); free(G); free(dX); free(C);
   return 0;
 }
+
+/* ---------------------------------------------------------------------------------------------
+ * Output path after the scan: y_gt = RMSNorm(y_t (.) g_t) over the head-concatenated features. */
+static double silu_fn(double x, double *dx) {
+  const double sg = 1.0 / (1.0 + exp(-x));
+  if (dx) *dx = sg * (1.0 + x * (1.0 - sg));
+  return x * sg;
+}
+
+int m2rnn_ref_gated_norm_fwd(long tokens, int d, const double *y, const double *g_in, const double *w,
+                             double eps, int silu, double *out, double *rstd) {
+  if (!y || !g_in || !w || !out || d <= 0 || tokens < 0) return -1;
+  for (long t = 0; t < tokens; ++t) {
+    const double *yt = y + t * d, *gt = g_in + t * d;
+    double ss = 0.0;
+    for (int j = 0; j < d; ++j) {
+      const double g = silu ? silu_fn(gt[j], NULL) : gt[j];
+      const double x = yt[j] * g;
+      ss += x * x;
+    }
+    const double s = 1.0 / sqrt(ss / d + eps);
+    for (int j = 0; j < d; ++j) {
+      const double g = silu ? silu_fn(gt[j], NULL) : gt[j];
+      out[t * d + j] = w[j] * (yt[j] * g) * s;
+    }
+    if (rstd) rstd[t] = s;
+  }
+  return 0;
+}
+
+int m2rnn_ref_gated_norm_bwd(long tokens, int d, const double *y, const double *g_in, const double *w,
+                             double eps, int silu, const double *dout, double *dy, double *dg_in,
+                             double *dw) {
+  if (!y || !g_in || !w || !dout || !dy || !dg_in || !dw || d <= 0 || tokens < 0) return -1;
+  for (int j = 0; j < d; ++j) dw[j] = 0.0;
+  for (long t = 0; t < tokens; ++t) {
+    const double *yt = y + t * d, *gt = g_in + t * d, *dot = dout + t * d;
+    double ss = 0.0, r = 0.0;
+    for (int j = 0; j < d; ++j) {
+      const double g = silu ? silu_fn(gt[j], NULL) : gt[j];
+      const double x = yt[j] * g;
+      ss += x * x;
+      r += w[j] * dot[j] * x;
+    }
+    const double s = 1.0 / sqrt(ss / d + eps);
+    for (int j = 0; j < d; ++j) {
+      double dsilu = 1.0;
+      const double g = silu ? silu_fn(gt[j], &dsilu) : gt[j];
+      const double x = yt[j] * g;
+      const double dx = s * w[j] * dot[j] - r * s * s * s * x / d;
+      dy[t * d + j] = dx * g;
+      dg_in[t * d + j] = dx * yt[j] * dsilu;
+      dw[j] += dot[j] * x * s;
+    }
+  }
+  return 0;
+}

@@ -64,6 +64,21 @@ int m2rnn_ref_decode_step(const m2rnn_ref_params *p, const double *q, const doub
                           const double *alpha, const double *beta, const double *w_r,
                           double *state, double *y);
 
+/* Output path of the layer after the scan ("M2RNN block" equations, y_gt = RMSNorm(y_t (.) g_t), and
+ * the RMSNorm appendix): per token, over the d features of all heads concatenated,
+ *     x = y (.) g,   s = 1 / sqrt(mean_j x_j^2 + eps),   out_i = w_i x_i s,
+ * with g = g_in (silu = 0) or g = SiLU(g_in) = g_in / (1 + exp(-g_in)) (silu != 0).
+ * y, g_in, out [tokens, d]; w [d]; rstd [tokens] receives s (may be NULL). */
+int m2rnn_ref_gated_norm_fwd(long tokens, int d, const double *y, const double *g_in, const double *w,
+                             double eps, int silu, double *out, double *rstd);
+
+/* Its backward (RMSNorm appendix: p = w (.) dout, r = sum_j p_j x_j, dx = s p - r s^3 x / d,
+ * dw_i = sum over tokens of dout_i x_i s), then through the product: dy = dx (.) g,
+ * dg = dx (.) y, and through SiLU when silu != 0.  dw [d] is the sum over tokens. */
+int m2rnn_ref_gated_norm_bwd(long tokens, int d, const double *y, const double *g_in, const double *w,
+                             double eps, int silu, const double *dout, double *dy, double *dg_in,
+                             double *dw);
+
 #ifdef __cplusplus
 }
 #endif

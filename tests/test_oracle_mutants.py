@@ -29,6 +29,14 @@ MUTANTS = [
     ("bwd_dW_wrong_state", "s += Hprev[i * V + l] * dX[i * V + j];", "s += Hcur[i * V + l] * dX[i * V + j];"),
     ("bwd_dq_pre_update", "s += Hcur[i * V + j] * dyt[j];", "s += Hprev[i * V + j] * dyt[j];"),
     ("bwd_dv_residual_dropped", "if (w_r) s += w_r[(size_t)n * V + j] * dyt[j];", ""),
+    ("norm_mean_is_sum", "const double s = 1.0 / sqrt(ss / d + eps);\n    for (int j = 0; j < d; ++j) {\n      const double g = silu ? silu_fn(gt[j], NULL) : gt[j];\n      out",
+     "const double s = 1.0 / sqrt(ss + eps);\n    for (int j = 0; j < d; ++j) {\n      const double g = silu ? silu_fn(gt[j], NULL) : gt[j];\n      out"),
+    ("norm_weight_dropped", "out[t * d + j] = w[j] * (yt[j] * g) * s;", "out[t * d + j] = (yt[j] * g) * s;"),
+    ("norm_silu_is_sigmoid", "return x * sg;", "return sg;"),
+    ("norm_bwd_projection_dropped", "const double dx = s * w[j] * dot[j] - r * s * s * s * x / d;", "const double dx = s * w[j] * dot[j];"),
+    ("norm_bwd_dg_uses_gate", "dg_in[t * d + j] = dx * yt[j] * dsilu;", "dg_in[t * d + j] = dx * g * dsilu;"),
+    ("norm_bwd_dw_without_s", "dw[j] += dot[j] * x * s;", "dw[j] += dot[j] * x;"),
+    ("norm_bwd_silu_derivative", "if (dx) *dx = sg * (1.0 + x * (1.0 - sg));", "if (dx) *dx = sg * (1.0 - sg);"),
     ("bwd_dh0_seed_ignored", "if (d_hT) memcpy(C, d_hT + bn * KV, sizeof(double) * KV);\n      else memset", "memset"),
 ]
 
@@ -38,12 +46,14 @@ PIN_CALLS = [
     pins.test_symmetries, pins.test_multi_value_equals_broadcast, pins.test_chaining,
     pins.test_gate_modes, pins.test_bwd_last_step_matches_algorithm2, pins.test_bwd_matches_autograd,
     functools.partial(pins.test_bwd_matches_finite_differences, gate_kind=2, shared=True),
+    pins.test_gated_norm_by_hand, pins.test_gated_norm_invariants, pins.test_gated_norm_bwd_matches_autograd,
+    functools.partial(pins.test_gated_norm_bwd_matches_finite_differences, silu=True),
 ]
 
 
 def _proxy(oracle, lib):
     ns = types.SimpleNamespace()
-    for name in ("fwd", "bwd", "decode_step", "gate_fn"):
+    for name in ("fwd", "bwd", "decode_step", "gate_fn", "gated_norm_fwd", "gated_norm_bwd"):
         setattr(ns, name, functools.partial(getattr(oracle, name), lib=lib))
     return ns
 

@@ -329,3 +329,76 @@ def test_bwd_state_gradient_clipping(oracle):
     # the last time step sees no clipped quantity yet
     np.testing.assert_array_equal(tight["dv"][:, -1], base["dv"][:, -1])
     assert not np.array_equal(tight["dv"][:, 0], base["dv"][:, 0])
+
+
+# ---------------------------------------------------------------- output path: RMSNorm(y (.) g)
+def test_gated_norm_by_hand(oracle):
+    """x = (3, 4, 0, 0): mean square 25/4, s = 2/5, out = w (.) x (.) s; SiLU(1) from its definition."""
+    y = np.array([[[1.5, 2.0], [0.0, 7.0]]])          # one token, N = 2 heads, V = 2
+    g = np.array([[[2.0, 2.0], [5.0, 0.0]]])
+    w = np.array([1.0, 0.5, 3.0, 3.0])
+    out, rstd = oracle.gated_norm_fwd(y, g, w, eps=0.0, silu=False)
+    np.testing.assert_allclose(rstd, [0.4], rtol=0, atol=1e-15)
+    np.testing.assert_allclose(out.reshape(-1), [1.2, 0.8, 0.0, 0.0], rtol=0, atol=1e-15)
+    out2, rstd2 = oracle.gated_norm_fwd(y, g, w, eps=0.75, silu=False)     # 25/4 + 3/4 = 7
+    np.testing.assert_allclose(rstd2, [7.0 ** -0.5], rtol=1e-15)
+    # SiLU: the gate value is g / (1 + e^-g); with y = 1 the normalised vector is SiLU(g) / rms
+    gin = np.array([[[1.0, -2.0]]])
+    sl = np.array([1.0 / (1.0 + np.e ** -1.0), -2.0 / (1.0 + np.e ** 2.0)])
+    out3, _ = oracle.gated_norm_fwd(np.ones((1, 1, 2)), gin, np.ones(2), eps=0.0, silu=True)
+    np.testing.assert_allclose(out3.reshape(-1), sl / np.sqrt(np.mean(sl ** 2)), rtol=1e-14)
+
+
+def test_gated_norm_invariants(oracle):
+    rng = np.random.default_rng(31)
+    y, g = rng.standard_normal((3, 5, 4, 6)), rng.standard_normal((3, 5, 4, 6))
+    w = rng.uniform(0.5, 2.0, size=24)
+    out, rstd = oracle.gated_norm_fwd(y, g, w, eps=0.0, silu=True)
+    # unit root-mean-square before the weight; scale invariance in y; rstd is what it says
+    np.testing.assert_allclose(np.mean((out.reshape(3, 5, 24) / w) ** 2, axis=-1), 1.0, rtol=1e-13)
+    out_s, rstd_s = oracle.gated_norm_fwd(-3.0 * y, g, w, eps=0.0, silu=True)
+    np.testing.assert_allclose(out_s, -out, rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(rstd_s, rstd / 3.0, rtol=1e-13)
+    # against torch's RMSNorm and SiLU (library routines, fp64)
+    x = torch.from_numpy(y) * torch.nn.functional.silu(torch.from_numpy(g))
+    ref = torch.nn.functional.rms_norm(x.reshape(3, 5, 24), (24,), torch.from_numpy(w), eps=1e-3)
+    out_e, _ = oracle.gated_norm_fwd(y, g, w, eps=1e-3, silu=True)
+    np.testing.assert_allclose(out_e.reshape(3, 5, 24), ref.numpy(), rtol=1e-13, atol=1e-15)
+
+
+@pytest.mark.parametrize("silu", [False, True])
+def test_gated_norm_bwd_matches_finite_differences(oracle, silu):
+    rng = np.random.default_rng(32)
+    y, g = rng.standard_normal((2, 3, 2, 4)), rng.standard_normal((2, 3, 2, 4))
+    w, dout = rng.uniform(0.5, 2.0, size=8), rng.standard_normal((2, 3, 2, 4))
+    eps = 0.05
+    got = oracle.gated_norm_bwd(y, g, w, dout, eps=eps, silu=silu)
+
+    def loss(y_, g_, w_):
+        return float(np.sum(oracle.gated_norm_fwd(y_, g_, w_, eps=eps, silu=silu)[0] * dout))
+
+    h = 1e-6
+    for name, arr, grad in (("dy", y, got["dy"]), ("dg", g, got["dg"]), ("dw", w, got["dw"])):
+        num = np.zeros_like(arr)
+        it = np.nditer(arr, flags=["multi_index"])
+        for _ in it:
+            i = it.multi_index
+            a, b = arr.copy(), arr.copy()
+            a[i] += h; b[i] -= h
+            args = {"dy": (a, g, w), "dg": (y, a, w), "dw": (y, g, a)}[name], {"dy": (b, g, w), "dg": (y, b, w), "dw": (y, g, b)}[name]
+            num[i] = (loss(*args[0]) - loss(*args[1])) / (2 * h)
+        np.testing.assert_allclose(grad, num, rtol=2e-6, atol=2e-8, err_msg=name)
+
+
+def test_gated_norm_bwd_matches_autograd(oracle):
+    rng = np.random.default_rng(33)
+    y, g = rng.standard_normal((4, 2, 3, 8)), rng.standard_normal((4, 2, 3, 8))
+    w, dout = rng.uniform(0.5, 2.0, size=24), rng.standard_normal((4, 2, 3, 8))
+    ty, tg, tw = (torch.tensor(a, requires_grad=True) for a in (y, g, w))
+    x = (ty * torch.nn.functional.silu(tg)).reshape(4, 2, 24)
+    out = torch.nn.functional.rms_norm(x, (24,), tw, eps=1e-2)
+    (out * torch.from_numpy(dout).reshape(4, 2, 24)).sum().backward()
+    got = oracle.gated_norm_bwd(y, g, w, dout, eps=1e-2, silu=True)
+    np.testing.assert_allclose(got["dy"], ty.grad.numpy(), rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(got["dg"], tg.grad.numpy(), rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(got["dw"], tw.grad.numpy(), rtol=1e-12, atol=1e-14)
