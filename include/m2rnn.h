@@ -174,6 +174,35 @@ int m2rnn_decode_step(const m2rnn_params *params, const void *q, const void *k, 
                       const float *gate, const void *W, const float *alpha, const float *beta,
                       const void *w_r, float *state, void *y, int32_t *dev_status, void *stream);
 
+/* ---- Output path after the scan ("M2RNN block" equations: y_gt = RMSNorm(y_t (.) g_t) with
+ * g_t = SiLU of the gate projection; "RMSNormTP Module" appendix for RMSNorm and its backward).
+ * Fuses the product with the gate and the normalisation over the d = N V features of all heads of
+ * a token, so that y (.) g never goes to memory:
+ *     x = y (.) g,   s = 1 / sqrt((1/d) sum_j x_j^2 + eps),   out_i = w_i x_i s
+ * where g = g_in (silu = 0) or g = SiLU(g_in) = g_in / (1 + exp(-g_in)) (silu != 0).  The paper
+ * prints RMSNorm without an epsilon: eps = 0 reproduces it, a positive eps guards all-zero rows.
+ *   in : y, g_in [tokens, d] (the scan's y [B,T,N,V] has tokens = B T, d = N V), w [d], io_dtype
+ *   out: out [tokens, d] io_dtype; rstd [tokens] fp32 = s (NULL: not stored; the backward needs it)
+ * d is a multiple of 8, at most 8192.  tokens = 0 is a valid empty call.  Pointers: device, 16-byte
+ * aligned, caller-owned; asynchronous on `stream`; errors as for the scan calls. */
+int m2rnn_gated_norm_fwd(int64_t tokens, int32_t d, int32_t io_dtype, const void *y, const void *g_in,
+                         const void *w, float eps, int32_t silu, void *out, float *rstd, void *stream);
+
+/* Bytes of workspace m2rnn_gated_norm_bwd needs (per-CTA partial sums of dw). */
+size_t m2rnn_gated_norm_bwd_workspace_bytes(int64_t tokens, int32_t d);
+
+/* Backward of m2rnn_gated_norm_fwd (appendix formulas: p = w (.) dout, r = sum_j p_j x_j,
+ * dx = s p - r s^3 x / d, dw_i = sum over tokens of dout_i x_i s), continued through the product
+ * (dy = dx (.) g, dg = dx (.) y) and through SiLU when silu != 0.
+ *   in : y, g_in, w as in the forward call; rstd [tokens] as the forward call stored it;
+ *        dout [tokens, d]
+ *   out: dy, dg_in [tokens, d] io_dtype; dw [d] fp32 (sum over tokens, fixed order: bitwise
+ *        repeatable); all overwritten
+ *   workspace: 256-byte aligned device memory of at least the queried size. */
+int m2rnn_gated_norm_bwd(int64_t tokens, int32_t d, int32_t io_dtype, const void *y, const void *g_in,
+                         const void *w, const float *rstd, int32_t silu, const void *dout, void *dy,
+                         void *dg_in, float *dw, void *workspace, size_t workspace_bytes, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -59,6 +59,11 @@ EXPORTS = {
     "m2rnn_bwd": (ctypes.c_int, [_pp] + [_vp] * 19 + [ctypes.c_size_t, _vp, _vp]),
     "m2rnn_bwd_static_scratch": (ctypes.c_int, [_pp] + [_vp] * 20),
     "m2rnn_decode_step": (ctypes.c_int, [_pp] + [_vp] * 12),
+    "m2rnn_gated_norm_fwd": (ctypes.c_int, [ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, _vp, _vp, _vp, ctypes.c_float,
+                                            ctypes.c_int32, _vp, _vp, _vp]),
+    "m2rnn_gated_norm_bwd_workspace_bytes": (ctypes.c_size_t, [ctypes.c_int64, ctypes.c_int32]),
+    "m2rnn_gated_norm_bwd": (ctypes.c_int, [ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, _vp, _vp, _vp, _vp, ctypes.c_int32,
+                                            _vp, _vp, _vp, _vp, _vp, ctypes.c_size_t, _vp]),
 }
 
 STATIC_SCRATCH_BYTES = 8 << 20   # M2RNN_STATIC_SCRATCH_BYTES
@@ -283,3 +288,58 @@ def m2rnn_decode_step(q, k, v, gate, W, state, *, gate_kind=GATE_LOGIT, alpha=No
     if rc != 0:
         raise M2RNNError(rc, "m2rnn_decode_step")
     return y
+
+
+def _norm_dims(y):
+    if y.dim() < 2:
+        raise ValueError("y needs at least the two trailing axes [N, V]")
+    d = y.shape[-2] * y.shape[-1]
+    tokens = y.numel() // d if d else 0
+    return tokens, d
+
+
+def m2rnn_gated_norm_fwd(y, g_in, w, *, eps=0.0, silu=True, out=None, rstd=None, stream=None):
+    """out = RMSNorm(y * SiLU(g_in)) over the head-concatenated features: y, g_in [..., N, V],
+    w [N*V] (or [N, V]).  Returns (out like y, rstd [...] fp32)."""
+    tokens, d = _norm_dims(y)
+    io = y.dtype
+    _chk(g_in, "g_in", tuple(y.shape), io); _chk(w, "w", tuple(w.shape), io)
+    if w.numel() != d:
+        raise ValueError(f"w has {w.numel()} entries, the rows have {d}")
+    if out is None:
+        out = torch.empty_like(y)
+    if rstd is None:
+        rstd = torch.empty(tuple(y.shape[:-2]), dtype=torch.float32, device=y.device)
+    _chk(out, "out", tuple(y.shape), io); _chk(rstd, "rstd", tuple(y.shape[:-2]), torch.float32)
+    rc = _lib().m2rnn_gated_norm_fwd(tokens, d, _io_code(io), _ptr(y), _ptr(g_in), _ptr(w), float(eps), int(bool(silu)),
+                                     _ptr(out), _ptr(rstd), _stream(stream))
+    if rc != 0:
+        raise M2RNNError(rc, "m2rnn_gated_norm_fwd")
+    return out, rstd
+
+
+def m2rnn_gated_norm_bwd_workspace_bytes(tokens: int, d: int) -> int:
+    return int(_lib().m2rnn_gated_norm_bwd_workspace_bytes(tokens, d))
+
+
+def m2rnn_gated_norm_bwd(y, g_in, w, rstd, dout, *, silu=True, workspace=None, out=None, stream=None):
+    """Backward of m2rnn_gated_norm_fwd -> dict(dy, dg, dw [N*V] fp32)."""
+    tokens, d = _norm_dims(y)
+    io = y.dtype
+    _chk(g_in, "g_in", tuple(y.shape), io); _chk(dout, "dout", tuple(y.shape), io); _chk(w, "w", tuple(w.shape), io)
+    _chk(rstd, "rstd", tuple(y.shape[:-2]), torch.float32)
+    out = out or {}
+    dy = out.get("dy", None); dg = out.get("dg", None); dw = out.get("dw", None)
+    dy = torch.empty_like(y) if dy is None else dy
+    dg = torch.empty_like(y) if dg is None else dg
+    dw = torch.empty((d,), dtype=torch.float32, device=y.device) if dw is None else dw
+    _chk(dy, "dy", tuple(y.shape), io); _chk(dg, "dg", tuple(y.shape), io); _chk(dw, "dw", (d,), torch.float32)
+    need = m2rnn_gated_norm_bwd_workspace_bytes(tokens, d)
+    if workspace is None:
+        workspace = torch.empty(max(need, 1), dtype=torch.uint8, device=y.device)
+    rc = _lib().m2rnn_gated_norm_bwd(tokens, d, _io_code(io), _ptr(y), _ptr(g_in), _ptr(w), _ptr(rstd), int(bool(silu)),
+                                     _ptr(dout), _ptr(dy), _ptr(dg), _ptr(dw), _ptr(workspace), workspace.numel(),
+                                     _stream(stream))
+    if rc != 0:
+        raise M2RNNError(rc, "m2rnn_gated_norm_bwd")
+    return dict(dy=dy, dg=dg, dw=dw)

@@ -1,0 +1,249 @@
+// Output path of the layer after the scan ("M2RNN block" equations: y_gt = RMSNorm(y_t (.) g_t),
+// g_t = SiLU of the gate projection; RMSNorm appendix for the formulas and their backward), fused
+// into one pass each way: y and g are read once, the normalised product is written once, the
+// product y (.) g never goes to memory.  Per token over the d = N V features of all heads:
+//     x = y (.) g,   s = 1 / sqrt(mean x^2 + eps),   out = w (.) x s            (s is cached)
+//     p = w (.) dout, r = sum p x, dx = s p - r s^3 x / d, dy = dx (.) g, dg = dx (.) y (SiLU'),
+//     dw = sum over tokens of dout (.) x s.
+// One warp per token (tokens are plentiful and a row is 2-16 KB), 16-byte loads and stores, the
+// row's products parked in shared memory between the reduction and the scaling; HBM-bound.
+// dw: per-warp accumulators in shared memory, one partial per CTA, then a fixed-order second stage.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "internal.h"
+#include "m2rnn.h"
+
+namespace m2rnn {
+namespace {
+
+constexpr int kWarps = 4;
+constexpr int kMaxCtas = 592;   // 4 per SM on 148 SMs: also the number of dw partials at most
+constexpr int kMaxD = 8192;
+
+// 8 consecutive elements as floats
+__device__ __forceinline__ void load8(const __nv_bfloat16 *p, float (&f)[8]) {
+  const uint4 r = *reinterpret_cast<const uint4 *>(p);
+  const uint32_t u[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { f[2 * i] = __uint_as_float(u[i] << 16); f[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u); }
+}
+__device__ __forceinline__ void load8(const float *p, float (&f)[8]) {
+  const float4 a = *reinterpret_cast<const float4 *>(p), b = *reinterpret_cast<const float4 *>(p + 4);
+  f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+}
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t *>(&v);
+}
+__device__ __forceinline__ void store8(__nv_bfloat16 *p, const float (&f)[8]) {
+  *reinterpret_cast<uint4 *>(p) = make_uint4(pack2(f[0], f[1]), pack2(f[2], f[3]), pack2(f[4], f[5]), pack2(f[6], f[7]));
+}
+__device__ __forceinline__ void store8(float *p, const float (&f)[8]) {
+  *reinterpret_cast<float4 *>(p) = make_float4(f[0], f[1], f[2], f[3]);
+  *reinterpret_cast<float4 *>(p + 4) = make_float4(f[4], f[5], f[6], f[7]);
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+// SiLU and its derivative
+__device__ __forceinline__ float silu(float x, float *dx) {
+  const float sg = 1.f / (1.f + __expf(-x));
+  if (dx) *dx = sg * (1.f + x * (1.f - sg));
+  return x * sg;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kWarps * 32) gated_norm_fwd_kernel(long tokens, int d, const T *__restrict__ y,
+                                                                       const T *__restrict__ g_in, const T *__restrict__ w,
+                                                                       float eps, int use_silu, T *__restrict__ out,
+                                                                       float *__restrict__ rstd) {
+  extern __shared__ __align__(16) float xs_all[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float *xs = xs_all + (size_t)warp * d;
+  const int chunks = d >> 3;
+  for (long t = (long)blockIdx.x * kWarps + warp; t < tokens; t += (long)gridDim.x * kWarps) {
+    const T *yt = y + t * d, *gt = g_in + t * d;
+    float ss = 0.f;
+    for (int c = lane; c < chunks; c += 32) {
+      float a[8], b[8];
+      load8(yt + 8 * c, a);
+      load8(gt + 8 * c, b);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const float x = a[e] * (use_silu ? silu(b[e], nullptr) : b[e]);
+        a[e] = x;
+        ss = fmaf(x, x, ss);
+      }
+      *reinterpret_cast<float4 *>(xs + 8 * c) = make_float4(a[0], a[1], a[2], a[3]);
+      *reinterpret_cast<float4 *>(xs + 8 * c + 4) = make_float4(a[4], a[5], a[6], a[7]);
+    }
+    ss = warp_sum(ss);
+    const float s = 1.f / sqrtf(ss / (float)d + eps);
+    for (int c = lane; c < chunks; c += 32) {   // each lane re-reads what it wrote itself
+      float wv[8], o[8];
+      load8(w + 8 * c, wv);
+      const float4 x0 = *reinterpret_cast<const float4 *>(xs + 8 * c), x1 = *reinterpret_cast<const float4 *>(xs + 8 * c + 4);
+      const float x[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+#pragma unroll
+      for (int e = 0; e < 8; ++e) o[e] = wv[e] * x[e] * s;
+      store8(out + t * d + 8 * c, o);
+    }
+    if (rstd && lane == 0) rstd[t] = s;
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kWarps * 32) gated_norm_bwd_kernel(long tokens, int d, const T *__restrict__ y,
+                                                                       const T *__restrict__ g_in, const T *__restrict__ w,
+                                                                       const float *__restrict__ rstd, int use_silu,
+                                                                       const T *__restrict__ dout, T *__restrict__ dy,
+                                                                       T *__restrict__ dg_in, float *__restrict__ dw_part) {
+  extern __shared__ __align__(16) float acc_all[];   // [kWarps][d] partial sums of dw
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float *acc = acc_all + (size_t)warp * d;
+  const int chunks = d >> 3;
+  for (int c = lane; c < chunks; c += 32) {
+    *reinterpret_cast<float4 *>(acc + 8 * c) = make_float4(0.f, 0.f, 0.f, 0.f);
+    *reinterpret_cast<float4 *>(acc + 8 * c + 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  for (long t = (long)blockIdx.x * kWarps + warp; t < tokens; t += (long)gridDim.x * kWarps) {
+    const T *yt = y + t * d, *gt = g_in + t * d, *dot = dout + t * d;
+    const float s = rstd[t];
+    // r = sum_j w_j dout_j x_j
+    float r = 0.f;
+    for (int c = lane; c < chunks; c += 32) {
+      float a[8], b[8], wv[8], dv[8];
+      load8(yt + 8 * c, a);
+      load8(gt + 8 * c, b);
+      load8(w + 8 * c, wv);
+      load8(dot + 8 * c, dv);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) r = fmaf(wv[e] * dv[e], a[e] * (use_silu ? silu(b[e], nullptr) : b[e]), r);
+    }
+    r = warp_sum(r);
+    const float k3 = r * s * s * s / (float)d;
+    // second pass over the same row (served by the L1): the gradients
+    for (int c = lane; c < chunks; c += 32) {
+      float a[8], b[8], wv[8], dv[8], o1[8], o2[8];
+      load8(yt + 8 * c, a);
+      load8(gt + 8 * c, b);
+      load8(w + 8 * c, wv);
+      load8(dot + 8 * c, dv);
+      float4 w0 = *reinterpret_cast<const float4 *>(acc + 8 * c), w1 = *reinterpret_cast<const float4 *>(acc + 8 * c + 4);
+      float aw[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        float dsl = 1.f;
+        const float g = use_silu ? silu(b[e], &dsl) : b[e];
+        const float x = a[e] * g;
+        const float dx = s * wv[e] * dv[e] - k3 * x;
+        o1[e] = dx * g;
+        o2[e] = dx * a[e] * dsl;
+        aw[e] = fmaf(dv[e] * x, s, aw[e]);
+      }
+      store8(dy + t * d + 8 * c, o1);
+      store8(dg_in + t * d + 8 * c, o2);
+      *reinterpret_cast<float4 *>(acc + 8 * c) = make_float4(aw[0], aw[1], aw[2], aw[3]);
+      *reinterpret_cast<float4 *>(acc + 8 * c + 4) = make_float4(aw[4], aw[5], aw[6], aw[7]);
+    }
+  }
+  __syncthreads();
+  // this CTA's partial of dw: the warps' sums in a fixed order
+  for (int j = threadIdx.x; j < d; j += blockDim.x) {
+    float v = 0.f;
+#pragma unroll
+    for (int wi = 0; wi < kWarps; ++wi) v += acc_all[(size_t)wi * d + j];
+    dw_part[(size_t)blockIdx.x * d + j] = v;
+  }
+}
+
+int grid_for(long tokens) {
+  const long need = (tokens + kWarps - 1) / kWarps;
+  return (int)(need < kMaxCtas ? need : kMaxCtas);
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check(long tokens, int d, int io_dtype) {
+  if (tokens < 0 || d <= 0) return M2RNN_ERR_SHAPE;
+  if (io_dtype != M2RNN_F32 && io_dtype != M2RNN_BF16) return M2RNN_ERR_UNSUPPORTED;
+  if (d % 8 || d > kMaxD) return M2RNN_ERR_UNSUPPORTED;
+  return M2RNN_OK;
+}
+
+template <typename T>
+cudaError_t launch_fwd(long tokens, int d, const void *y, const void *g, const void *w, float eps, int silu_on, void *out,
+                       float *rstd, cudaStream_t s) {
+  const size_t smem = (size_t)kWarps * d * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(gated_norm_fwd_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  gated_norm_fwd_kernel<T><<<grid_for(tokens), kWarps * 32, smem, s>>>(tokens, d, static_cast<const T *>(y), static_cast<const T *>(g),
+                                                                      static_cast<const T *>(w), eps, silu_on, static_cast<T *>(out), rstd);
+  return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t launch_bwd(long tokens, int d, const void *y, const void *g, const void *w, const float *rstd, int silu_on,
+                       const void *dout, void *dy, void *dg, float *dw_part, cudaStream_t s) {
+  const size_t smem = (size_t)kWarps * d * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(gated_norm_bwd_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  gated_norm_bwd_kernel<T><<<grid_for(tokens), kWarps * 32, smem, s>>>(tokens, d, static_cast<const T *>(y), static_cast<const T *>(g),
+                                                                      static_cast<const T *>(w), rstd, silu_on, static_cast<const T *>(dout),
+                                                                      static_cast<T *>(dy), static_cast<T *>(dg), dw_part);
+  return cudaGetLastError();
+}
+
+}  // namespace
+}  // namespace m2rnn
+
+using namespace m2rnn;
+
+extern "C" {
+
+int m2rnn_gated_norm_fwd(int64_t tokens, int32_t d, int32_t io_dtype, const void *y, const void *g_in, const void *w,
+                         float eps, int32_t silu_on, void *out, float *rstd, void *stream) {
+  const int rc = check((long)tokens, d, io_dtype);
+  if (rc != M2RNN_OK) return rc;
+  if (tokens == 0) return M2RNN_OK;   // nothing to read or write
+  if (!y || !g_in || !w || !out) return M2RNN_ERR_NULL;
+  if (!aligned16(y) || !aligned16(g_in) || !aligned16(w) || !aligned16(out)) return M2RNN_ERR_ALIGN;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const cudaError_t e = io_dtype == M2RNN_BF16 ? launch_fwd<__nv_bfloat16>((long)tokens, d, y, g_in, w, eps, silu_on, out, rstd, s)
+                                               : launch_fwd<float>((long)tokens, d, y, g_in, w, eps, silu_on, out, rstd, s);
+  return e == cudaSuccess ? M2RNN_OK : M2RNN_ERR_CUDA;
+}
+
+size_t m2rnn_gated_norm_bwd_workspace_bytes(int64_t tokens, int32_t d) {
+  if (tokens <= 0 || d <= 0) return 0;
+  return (size_t)grid_for((long)tokens) * (size_t)d * sizeof(float);
+}
+
+int m2rnn_gated_norm_bwd(int64_t tokens, int32_t d, int32_t io_dtype, const void *y, const void *g_in, const void *w,
+                         const float *rstd, int32_t silu_on, const void *dout, void *dy, void *dg_in, float *dw,
+                         void *workspace, size_t workspace_bytes, void *stream) {
+  const int rc = check((long)tokens, d, io_dtype);
+  if (rc != M2RNN_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (tokens == 0) {   // an empty sum
+    if (!dw) return M2RNN_ERR_NULL;
+    return cudaMemsetAsync(dw, 0, (size_t)d * sizeof(float), s) == cudaSuccess ? M2RNN_OK : M2RNN_ERR_CUDA;
+  }
+  if (!y || !g_in || !w || !rstd || !dout || !dy || !dg_in || !dw) return M2RNN_ERR_NULL;
+  if (!aligned16(y) || !aligned16(g_in) || !aligned16(w) || !aligned16(dout) || !aligned16(dy) || !aligned16(dg_in) || !aligned16(dw))
+    return M2RNN_ERR_ALIGN;
+  if (!workspace || workspace_bytes < m2rnn_gated_norm_bwd_workspace_bytes(tokens, d)) return M2RNN_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return M2RNN_ERR_ALIGN;
+  float *part = static_cast<float *>(workspace);
+  cudaError_t e = io_dtype == M2RNN_BF16 ? launch_bwd<__nv_bfloat16>((long)tokens, d, y, g_in, w, rstd, silu_on, dout, dy, dg_in, part, s)
+                                         : launch_bwd<float>((long)tokens, d, y, g_in, w, rstd, silu_on, dout, dy, dg_in, part, s);
+  if (e != cudaSuccess) return M2RNN_ERR_CUDA;
+  e = launch_reduce_slabs(part, dw, M2RNN_F32, grid_for((long)tokens), (size_t)d, s);
+  return e == cudaSuccess ? M2RNN_OK : M2RNN_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -134,6 +134,18 @@ def make_inputs(cfg: ScanConfig, *, backward: bool = False, seed: int | None = N
     return out
 
 
+def make_gated_norm_inputs(B: int, T: int, N: int, V: int, dtype: str = "bf16", seed: int = 0) -> dict:
+    """CPU tensors for the output path after the scan: y, g_in, dout [B,T,N,V] ~ N(0,1) (the scan's
+    readout is of unit scale), w [N*V] ~ U(0.5, 1.5); drawn in fp32 in that order from one PCG64
+    stream, then rounded to the I/O dtype."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    io = torch_dtype(dtype)
+    out = {"y": _normal(rng, (B, T, N, V)).to(io), "g_in": _normal(rng, (B, T, N, V)).to(io)}
+    out["dout"] = _normal(rng, (B, T, N, V)).to(io)
+    out["w"] = torch.from_numpy(rng.uniform(0.5, 1.5, size=(N * V,)).astype(np.float32)).to(io)
+    return out
+
+
 def to_f64(t):
     """Exact widening of a (possibly bf16) tensor to a numpy float64 array; None stays None."""
     return None if t is None else t.detach().to("cpu", torch.float64).numpy()
