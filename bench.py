@@ -228,12 +228,155 @@ def nbytes(t):
     return 0 if t is None else t.numel() * t.element_size()
 
 
+def main_out_norm(args):
+    """`--workload out_norm`: the output path after the scan (y (.) SiLU(g) -> RMSNorm over the
+    concatenated heads), forward + backward, on the y of the fwd_bf16 workload (B=8, T=2048, N=16,
+    V=64, bf16).  HBM-bound: 6d+4 bytes per token forward, 10d+4 backward (d = N V)."""
+    from paper_2603_14360_b200 import binding
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_
+        dist_.init_process_group("nccl", device_id=dev)
+        dist = dist_
+    base = CONFIGS["fwd_bf16"]
+    B, T, N, V = base.B, base.T, base.N, base.V
+    d = N * V
+    tokens = B * T
+    args.steps = args.steps or 200
+    args.warmup = max(args.warmup or 10, 3)
+    R = 8                                              # 8 x 168 MB of inputs and outputs cycled: far above L2
+    host = [{k: v.pin_memory() for k, v in inputs.make_gated_norm_inputs(B, T, N, V, "bf16",
+                                                                         seed=rank_input_seed(7, rank, r)).items()}
+            for r in range(R)]
+    sets = [{k: v.to(dev) for k, v in h.items()} for h in host]
+    outs = [dict(out=torch.empty_like(s["y"]), rstd=torch.empty((B, T), dtype=torch.float32, device=dev),
+                 dy=torch.empty_like(s["y"]), dg=torch.empty_like(s["y"]),
+                 dw=torch.empty((d,), dtype=torch.float32, device=dev)) for s in sets[:2]]
+    ws = torch.empty(max(1, binding.m2rnn_gated_norm_bwd_workspace_bytes(tokens, d)), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def launch(s, o, st):
+        binding.m2rnn_gated_norm_fwd(s["y"], s["g_in"], s["w"], eps=1e-6, out=o["out"], rstd=o["rstd"], stream=st)
+        binding.m2rnn_gated_norm_bwd(s["y"], s["g_in"], s["w"], o["rstd"], s["dout"], workspace=ws, out=o, stream=st)
+
+    # the three launches of a step are short (tens of microseconds): one CUDA graph per input set
+    # replays them without the per-launch host work
+    for s_ in sets:
+        launch(s_, outs[0], stream)
+    torch.cuda.synchronize()
+    graphs = []
+    for s_ in sets:
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr):
+            launch(s_, outs[0], torch.cuda.current_stream())
+        graphs.append(gr)
+
+    def step(i, s=None, ob=0):
+        if s is None:
+            graphs[i % R].replay()
+        else:
+            launch(s, outs[ob], stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    with ClockSampler(local) as clocks:
+        barrier()
+        ev[0].record(stream)
+        for i in range(args.steps):
+            step(i)
+        ev[1].record(stream)
+        barrier()
+    ms_total = ev[0].elapsed_time(ev[1])
+    # end to end: y, g, dout in from pinned host memory, out, dy, dg, dw back, every step (one stream)
+    ms_e2e, e2e_steps, h2d, d2h = 0.0, 0, 0, 0
+    if not args.no_e2e:
+        stage = {k: torch.empty_like(v) for k, v in sets[0].items()}
+        hout = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in outs[0].items() if k != "rstd"}
+        h2d = sum(nbytes(t) for t in stage.values())
+        d2h = sum(nbytes(t) for t in hout.values())
+        e2e_steps = 20
+
+        def e2e_step(i):
+            for k, t in stage.items():
+                t.copy_(host[i % R][k], non_blocking=True)
+            step(i, s=stage)
+            for k, t in hout.items():
+                t.copy_(outs[0][k], non_blocking=True)
+
+        for i in range(3):
+            e2e_step(i)
+        barrier()
+        ev2 = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        ev2[0].record(stream)
+        for i in range(e2e_steps):
+            e2e_step(i)
+        ev2[1].record(stream)
+        barrier()
+        ms_e2e = ev2[0].elapsed_time(ev2[1])
+    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], dist, dev)
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+    ms_step = ms_total / args.steps
+    peaks = measured_peaks()
+    alg_bytes = tokens * ((6 * d + 4) + (10 * d + 4)) + 2 * d * 2 + d * 4
+    achieved = alg_bytes / (ms_step * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": whole_job_tokens_per_s(tokens, world, ms_step), "unit": "tokens/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "out_norm", "pass": "fwd+bwd of RMSNorm(y * SiLU(g))", "B": B, "T": T, "N": N, "V": V, "d": d,
+                   "per_gpu_batch": B, "l2": f"{R} input sets cycled; bytes touched per step {int(alg_bytes / 1e6)} MB vs 126 MB L2"},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"], "traffic": None, "call": "m2rnn_gated_norm_fwd + m2rnn_gated_norm_bwd",
+                     "peak_source": f"{peaks['source']} HBM copy", "algorithmic_bytes_per_step": alg_bytes},
+        "gpu_launches": args.steps * 3,
+        "clocks": clocks.summary(),
+    }
+    if not args.no_e2e:
+        line["e2e"] = {"value": tokens * world / (ms_e2e / e2e_steps * 1e-3), "unit": "tokens/s",
+                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+    if not args.no_cpu_baseline:
+        import oracle
+        f = inputs.to_f64
+        n_tok = 1024                                    # a bounded sample: the first tokens of the first set
+        hs = {k: (v.reshape(tokens, N, V)[:n_tok] if v.dim() == 4 else v) for k, v in host[0].items()}
+        t0 = time.perf_counter()
+        reps = 0
+        while time.perf_counter() - t0 < 10.0:
+            oracle.gated_norm_fwd(f(hs["y"]), f(hs["g_in"]), f(hs["w"]), eps=1e-6)
+            oracle.gated_norm_bwd(f(hs["y"]), f(hs["g_in"]), f(hs["w"]), f(hs["dout"]), eps=1e-6)
+            reps += 1
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": reps * n_tok / dt, "unit": "tokens/s", "cores": 1, "kind": "oracle",
+                                "sample": f"{reps} x the first {n_tok} tokens of one input set, forward + backward", "seconds": dt}
+    print(json.dumps(line), flush=True)
+    if dist:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=0, help="0: a default per workload")
     ap.add_argument("--warmup", type=int, default=0)
-    ap.add_argument("--workload", default="fwd_bf16", choices=sorted(CONFIGS))
+    ap.add_argument("--workload", default="fwd_bf16", choices=sorted(CONFIGS) + ["out_norm"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -242,6 +385,11 @@ def main():
     ap.add_argument("--seq-len", type=int, default=0,
                     help="shorten (or lengthen) the workload's T, for profiler captures; the line's workload name says so")
     args = ap.parse_args()
+    if args.workload == "out_norm" and args.impl == "ours":
+        main_out_norm(args)
+        return
+    if args.workload == "out_norm":
+        raise SystemExit("--impl reference times the scan workloads; the out_norm line carries its own cpu_baseline")
     cfg = CONFIGS[args.workload]
     if args.seq_len and args.workload != "decode":
         cfg = cfg.with_(T=args.seq_len, name=f"{cfg.name}@T={args.seq_len}")

@@ -17,6 +17,10 @@ SHAPES = [
     (1, 131, 32, 128),    # d = 4096: several chunks per lane
     (5, 7, 2, 32),
     (2, 700, 4, 16),      # more tokens than one pass of the grid
+    (3, 41, 4, 64),       # d = 256: eight rows in flight per pass of the staged kernel
+    (1, 67, 8, 64),       # d = 512
+    (2, 29, 16, 128),     # d = 2048: one row per pass
+    (1, 1300, 16, 64),    # d = 1024, more blocks of rows than CTAs (the ring of stages wraps)
 ]
 
 
@@ -44,7 +48,7 @@ def test_gated_norm_bf16(oracle, shape, silu):
     assert errs["rstd"] < 1e-5, errs          # fp32 statistics of exactly representable inputs
 
 
-@pytest.mark.parametrize("shape", SHAPES[:4], ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("shape", SHAPES[:4] + SHAPES[6:9], ids=lambda s: "x".join(map(str, s)))
 @pytest.mark.parametrize("silu", [False, True])
 def test_gated_norm_f32(oracle, shape, silu):
     errs = _run(oracle, shape, "f32", silu, 0.0)
