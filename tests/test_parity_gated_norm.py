@@ -55,6 +55,13 @@ def test_gated_norm_f32(oracle, shape, silu):
     assert max(errs.values()) < 1e-4, errs
 
 
+def test_gated_norm_at_the_bench_size(oracle):
+    """The token count and row length bench.py times (fwd_bf16's y: 16 384 tokens of 1 024 features),
+    every element against the oracle."""
+    errs = _run(oracle, (8, 2048, 16, 64), "bf16", True, 1e-6)
+    assert max(errs.values()) < 2e-2, errs
+
+
 def test_gated_norm_repeatable_and_empty():
     d = parity.to_dev(inputs.make_gated_norm_inputs(2, 300, 16, 64, "bf16", seed=9))
     out, rstd = binding.m2rnn_gated_norm_fwd(d["y"], d["g_in"], d["w"], eps=1e-6)
