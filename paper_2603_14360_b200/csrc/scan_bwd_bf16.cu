@@ -128,6 +128,10 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
   constexpr bool kWInSmem = V > 64;
   // roles coincide with warpgroups only in this shape (4 + 4 + 4 + 1 warps), the one that needs it
   constexpr bool kRebalance = bwd_rebalance<V, NWC>();
+  // running operand addresses and per-lane tile offsets worked out once (an add per step instead of
+  // a multiply per use) where they measured faster; the 32-row V = 64 shape is short of registers
+  // and works them out at every use
+  constexpr bool kWalk = !(V == 64 && NWC == 2);
   // packed fp32x2 element-wise arithmetic where it measured faster (elsewhere its register pairs spill)
   constexpr bool kPacked = V <= 32 || (V == 64 && NWC == 4);
   constexpr int NSET = 1;   // accumulator sets of the state x W product, as in the forward kernel
@@ -184,6 +188,48 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
   // SEG memory columns SEG*c .. SEG*c+SEG-1 (MMA columns 8nt+2c+e <-> memory column SEG*c+2nt+e).
   auto tile_store = [&](uint32_t tile_sa, int w, const uint32_t (&p)[NT][2]) { m2rnn::tile_store<V>(tile_sa, w, lane, p); };
   auto tile_load = [&](uint32_t tile_sa, int w, uint32_t (&p)[NT][2]) { m2rnn::tile_load<V>(tile_sa, w, lane, p); };
+  // The same with the lane's byte offsets inside a tile worked out once per warp (they do not depend
+  // on the step): toff[h][x] for row g + 8h of slab w and the thread's x-th 16-byte chunk.
+  constexpr int CPRT = (SEG * 2 / 16) > 0 ? (SEG * 2 / 16) : 1;
+  auto tile_offsets = [&](int w, uint32_t (&toff)[2][CPRT]) {
+    if constexpr (!kWalk) return;
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+      for (int x = 0; x < CPRT; ++x) {
+        const int row = 16 * w + g + 8 * h;
+        if constexpr (SEG * 2 / 16 == 0) toff[h][x] = tile_off<V>(row, c >> 1) + 8u * (c & 1);
+        else toff[h][x] = tile_off<V>(row, CPRT * c + x);
+      }
+  };
+  auto tile_store_at = [&](uint32_t tile_sa, int w, const uint32_t (&toff)[2][CPRT], const uint32_t (&p)[NT][2]) {
+    if constexpr (!kWalk) { m2rnn::tile_store<V>(tile_sa, w, lane, p); return; }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      if constexpr (SEG * 2 / 16 == 0) {
+        asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(tile_sa + toff[h][0]), "r"(p[0][h]), "r"(p[1][h]) : "memory");
+      } else {
+#pragma unroll
+        for (int x = 0; x < CPRT; ++x)
+          asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(tile_sa + toff[h][x]), "r"(p[4 * x][h]), "r"(p[4 * x + 1][h]),
+                       "r"(p[4 * x + 2][h]), "r"(p[4 * x + 3][h]) : "memory");
+      }
+    }
+  };
+  auto tile_load_at = [&](uint32_t tile_sa, int w, const uint32_t (&toff)[2][CPRT], uint32_t (&p)[NT][2]) {
+    if constexpr (!kWalk) { m2rnn::tile_load<V>(tile_sa, w, lane, p); return; }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      if constexpr (SEG * 2 / 16 == 0) {
+        asm volatile("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(p[0][h]), "=r"(p[1][h]) : "r"(tile_sa + toff[h][0]));
+      } else {
+#pragma unroll
+        for (int x = 0; x < CPRT; ++x)
+          asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];"
+                       : "=r"(p[4 * x][h]), "=r"(p[4 * x + 1][h]), "=r"(p[4 * x + 2][h]), "=r"(p[4 * x + 3][h]) : "r"(tile_sa + toff[h][x]));
+      }
+    }
+  };
   // Z fragments: private to the (warp, lane) pair that wrote them, 2*NT words per thread kept as
   // NT/2 groups of 16 bytes (group x of lane l at word ((w*NT/2 + x)*32 + l)*4)
   constexpr int ZG = NT / 2;
@@ -198,6 +244,9 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
     // ================================================================= recompute warps
     if constexpr (kRebalance && V == 64) reg_inc<168>();
     const int w = warp, r0 = 16 * w + g;
+    uint32_t toff[2][CPRT];
+    tile_offsets(w, toff);
+    const uint32_t zoff = L.ztile + (uint32_t)(w * ZG * 32 + lane) * 16u;   // this lane's Z fragments inside a step's block
     uint32_t Wr[kWInSmem ? 1 : KT][kWInSmem ? 1 : NT][2];
     if constexpr (!kWInSmem) {
 #pragma unroll
@@ -222,21 +271,31 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
       if (!mbar_wait(&in_full[j & (kRing - 1)], (j / kRing) & 1)) { report_timeout(a.dev_status); return; }
       if (j >= 2 && !mbar_wait(&st_free[j & 1], ((j >> 1) - 1) & 1)) { report_timeout(a.dev_status); return; }
       const uint32_t sl = slot_sa(j);
+      // addresses of the step's operands: walked (one add per step) or worked out from s
+      struct Ptrs { uint32_t st, k, f, v; };
+      auto ptrs_at = [&](int s) {
+        return Ptrs{state_sa(j, s), sl + 4u * (L.oK + s * KC + r0), sl + 4u * (L.oF + s), sl + 4u * (L.oV + s * V + SEG * c)};
+      };
+      Ptrs run = ptrs_at(0);
       for (int s = 0; s < len; ++s) {
-        const uint32_t st = state_sa(j, s);
+        // (worked out at the place of use when not walked: short live ranges)
+        const uint32_t st = kWalk ? run.st : state_sa(j, s);
+#define pK (kWalk ? run.k : sl + 4u * (L.oK + s * KC + r0))
+#define pF (kWalk ? run.f : sl + 4u * (L.oF + s))
+#define pV (kWalk ? run.v : sl + 4u * (L.oV + s * V + SEG * c))
         // H_{t-1} as bf16: the A operand of this step and the tile the dW and reverse warps read
         uint32_t hp[NT][2];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) { hp[nt][0] = pack_bf16(H[nt][0], H[nt][1]); hp[nt][1] = pack_bf16(H[nt][2], H[nt][3]); }
-        tile_store(st, w, hp);
+        tile_store_at(st, w, toff, hp);
         // P = k v^T + H W   (Eq. 1 before the non-linearity)
-        const float k0 = lds32(sl + 4u * (L.oK + s * KC + r0)), k1 = lds32(sl + 4u * (L.oK + s * KC + r0 + 8));
-        const float f = lds32(sl + 4u * (L.oF + s));
+        const float k0 = lds32(pK), k1 = lds32(pK + 32u);
+        const float f = lds32(pF);
         // (two accumulator sets, as in the one-warp-per-slab forward kernel)
         float P[NSET][NT][4];
 #pragma unroll
         for (int x = 0; x < SEG / 4; ++x) {
-          const float4 v4 = lds128(sl + 4u * (L.oV + s * V + SEG * c + 4 * x));
+          const float4 v4 = lds128(pV + 16u * x);
           if constexpr (kPacked) {   // packed fp32 pairs: one instruction per two products
             const float2 k02 = make_float2(k0, k0), k12 = make_float2(k1, k1);
             const float2 a0 = __fmul2_rn(k02, make_float2(v4.x, v4.y)), a1 = __fmul2_rn(k12, make_float2(v4.x, v4.y));
@@ -262,7 +321,7 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
           }
         }
         // Z = tanh(P), kept as fp16 for the reverse sweep; H <- f H + (1-f) Z  (Eq. 2)
-        const uint32_t zs = zfrag_sa(st, w);
+        const uint32_t zs = kWalk ? st + zoff : zfrag_sa(st, w);
 #pragma unroll
         for (int x = 0; x < ZG; ++x) {
           uint32_t zw[4];
@@ -295,12 +354,16 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
           }
           asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(zs + 512u * x), "r"(zw[0]), "r"(zw[1]), "r"(zw[2]), "r"(zw[3]) : "memory");
         }
+        if constexpr (kWalk) { run.st += L.state_stride; run.k += 4u * KC; run.f += 4u; run.v += 4u * V; }
       }
+#undef pK
+#undef pF
+#undef pV
       if (j == 0) {   // the state after the last step of the scan: H_t of the first reverse step
         uint32_t hp[NT][2];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) { hp[nt][0] = pack_bf16(H[nt][0], H[nt][1]); hp[nt][1] = pack_bf16(H[nt][2], H[nt][3]); }
-        tile_store(sm0 + L.hfin, w, hp);
+        tile_store_at(sm0 + L.hfin, w, toff, hp);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&st_ready[j & 1]);
@@ -312,6 +375,9 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
     // ================================================================= reverse warps
     if constexpr (kRebalance && V == 64) reg_inc<208>();
     const int w = warp - NWC, r0 = 16 * w + g;
+    uint32_t toff[2][CPRT];
+    tile_offsets(w, toff);
+    const uint32_t zoff = L.ztile + (uint32_t)(w * ZG * 32 + lane) * 16u;
     uint32_t WTr[kWInSmem ? 1 : KT][kWInSmem ? 1 : NT][2];
     if constexpr (!kWInSmem) {
 #pragma unroll
@@ -366,21 +432,37 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
       const int len = chunk_len(j);
       if (!mbar_wait(&in_full[j & (kRing - 1)], (j / kRing) & 1)) { report_timeout(a.dev_status); return; }
       if (!mbar_wait(&st_ready[j & 1], (j >> 1) & 1)) { report_timeout(a.dev_status); return; }
-      if (j == 0) tile_load(sm0 + L.hfin, w, hn);
+      if (j == 0) tile_load_at(sm0 + L.hfin, w, toff, hn);
       const uint32_t sl = slot_sa(j);
+      // addresses of the step's operands: walked backwards (one add per step) or worked out from s
+      struct Ptrs { uint32_t st, f, q, dyb, vb, dy, dfp, dq, dk; };
+      auto ptrs_at = [&](int s) {
+        return Ptrs{state_sa(j, s), sl + 4u * (L.oF + s), sl + 4u * (L.oQ + s * KC + r0), sl + 4u * (L.oDYB + s * (V / 2)),
+                    sl + 4u * (L.oVB + s * (V / 2)), sl + 4u * (L.oDY + s * V + SEG * c),
+                    sl + 4u * (L.oDFP + (s * NWC + w) * 32 + lane), sl + 4u * (L.oDQ + s * KC + r0), sl + 4u * (L.oDK + s * KC + r0)};
+      };
+      Ptrs run = ptrs_at(len - 1);
       for (int s = len - 1; s >= 0; --s, ++nstep) {
-        const uint32_t st = state_sa(j, s);
+        const uint32_t st = kWalk ? run.st : state_sa(j, s);
+#define pF (kWalk ? run.f : sl + 4u * (L.oF + s))
+#define pQ (kWalk ? run.q : sl + 4u * (L.oQ + s * KC + r0))
+#define pDYB (kWalk ? run.dyb : sl + 4u * (L.oDYB + s * (V / 2)))
+#define pVB (kWalk ? run.vb : sl + 4u * (L.oVB + s * (V / 2)))
+#define pDY (kWalk ? run.dy : sl + 4u * (L.oDY + s * V + SEG * c))
+#define pDFP (kWalk ? run.dfp : sl + 4u * (L.oDFP + (s * NWC + w) * 32 + lane))
+#define pDQ (kWalk ? run.dq : sl + 4u * (L.oDQ + s * KC + r0))
+#define pDK (kWalk ? run.dk : sl + 4u * (L.oDK + s * KC + r0))
         uint32_t hp[NT][2];
-        tile_load(st, w, hp);
-        const uint32_t zs = zfrag_sa(st, w);
-        const float f = lds32(sl + 4u * (L.oF + s));
-        const float q0 = lds32(sl + 4u * (L.oQ + s * KC + r0)), q1 = lds32(sl + 4u * (L.oQ + s * KC + r0 + 8));
+        tile_load_at(st, w, toff, hp);
+        const uint32_t zs = kWalk ? st + zoff : zfrag_sa(st, w);
+        const float f = lds32(pF);
+        const float q0 = lds32(pQ), q1 = lds32(pQ + 32u);
         const float omf = 1.f - f;
         // dq = H_t dy on the tensor cores (Algorithm 2, "dq <- H . dy")
         float dqd[2][4], dkd[2][4];
         {
           uint32_t dyp[NT];
-          load_pairs(sl + 4u * (L.oDYB + s * (V / 2)), dyp);
+          load_pairs(pDYB, dyp);
           matvec(hn, dyp, dqd);
         }
         float df = 0.f;
@@ -388,7 +470,7 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
         uint32_t xp[NT][2];   // dX as bf16 pairs: the A operand of dX W^T and the tile of the dW warps
 #pragma unroll
         for (int x = 0; x < SEG / 4; ++x) {
-          const float4 dy4 = lds128(sl + 4u * (L.oDY + s * V + SEG * c + 4 * x));
+          const float4 dy4 = lds128(pDY + 16u * x);
           const float dyv[4] = {dy4.x, dy4.y, dy4.z, dy4.w};
           uint32_t zw[4];
           asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(zw[0]), "=r"(zw[1]), "=r"(zw[2]), "=r"(zw[3]) : "r"(zs + 512u * x));
@@ -431,7 +513,7 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
         // hand dX to the dW warps
         const int xb = nstep & 1;
         if (nstep >= 2 && !mbar_wait(&dx_free[xb], ((nstep >> 1) - 1) & 1)) { report_timeout(a.dev_status); return; }
-        tile_store(sm0 + L.dx + (uint32_t)xb * (KC * V * 2), w, xp);
+        tile_store_at(sm0 + L.dx + (uint32_t)xb * (KC * V * 2), w, toff, xp);
         __syncwarp();
         if (lane == 0) mbar_arrive(&dx_full[xb]);
         // C_{t-1} = f G + dX W^T
@@ -451,7 +533,7 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
         // dk = dX v on the tensor cores (Algorithm 2, "dk <- dX . v")
         {
           uint32_t vp[NT];
-          load_pairs(sl + 4u * (L.oVB + s * (V / 2)), vp);
+          load_pairs(pVB, vp);
           matvec(xp, vp, dkd);
         }
         if (clip > 0.f) {
@@ -460,14 +542,26 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
 #pragma unroll
             for (int r = 0; r < 4; ++r) Cg[nt][r] = fminf(fmaxf(Cg[nt][r], -clip), clip);
         }
-        sts32(sl + 4u * (L.oDFP + (s * NWC + w) * 32 + lane), df);   // summed by the service warp
+        sts32(pDFP, df);   // summed by the service warp
         if (c == 0) {
-          sts32(sl + 4u * (L.oDQ + s * KC + r0), dqd[0][0] + dqd[1][0]); sts32(sl + 4u * (L.oDQ + s * KC + r0 + 8), dqd[0][2] + dqd[1][2]);
-          sts32(sl + 4u * (L.oDK + s * KC + r0), dkd[0][0] + dkd[1][0]); sts32(sl + 4u * (L.oDK + s * KC + r0 + 8), dkd[0][2] + dkd[1][2]);
+          sts32(pDQ, dqd[0][0] + dqd[1][0]); sts32(pDQ + 32u, dqd[0][2] + dqd[1][2]);
+          sts32(pDK, dkd[0][0] + dkd[1][0]); sts32(pDK + 32u, dkd[0][2] + dkd[1][2]);
         }
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) { hn[nt][0] = hp[nt][0]; hn[nt][1] = hp[nt][1]; }
+        if constexpr (kWalk) {
+          run.st -= L.state_stride; run.f -= 4u; run.q -= 4u * KC; run.dyb -= 2u * V; run.vb -= 2u * V;
+          run.dy -= 4u * V; run.dfp -= 4u * NWC * 32; run.dq -= 4u * KC; run.dk -= 4u * KC;
+        }
       }
+#undef pF
+#undef pQ
+#undef pDYB
+#undef pVB
+#undef pDY
+#undef pDFP
+#undef pDQ
+#undef pDK
       __syncwarp();
       if (lane == 0) { mbar_arrive(&st_free[j & 1]); mbar_arrive(&out_full[j & (kRing - 1)]); }
     }
