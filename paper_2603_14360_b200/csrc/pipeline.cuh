@@ -44,11 +44,15 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
   if (!ok) {
     const long long t0 = clock64();
     uint32_t it = 0;
-    do {
+    for (;;) {
       if constexpr (kSleepNs > 0) __nanosleep(kSleepNs);
-      else if (++it > 64) __nanosleep(32);
+      else if (it > 64) __nanosleep(32);
       ok = mbar_try_wait(bar, parity);
-    } while (!ok && clock64() - t0 < kWaitCycles);
+      if (ok) break;
+      // the clock is read every 32nd poll only: a poll is a handful of instructions, and polling
+      // warps share issue slots with the warps that do the work
+      if ((++it & 31u) == 0u && clock64() - t0 > kWaitCycles) break;
+    }
   }
   return __all_sync(0xffffffffu, ok);
 }
