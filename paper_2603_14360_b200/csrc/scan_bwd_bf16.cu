@@ -587,6 +587,17 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
     const int mi = lane >> 3, mr = lane & 7;   // ldmatrix: lane supplies row mr of matrix mi
+    // Per-lane byte offsets of the ldmatrix rows inside a tile, without the slab term (16 rows =
+    // 32 V bytes per kt, added as an immediate): rows of 128 bytes or more keep their chunk swizzle
+    // (row & 7 = mr) when 16 rows are added, so the offsets are worked out once.
+    constexpr bool kPreOff = kWalk && 2 * V >= 128;
+    uint32_t offA = 0, offDv = 0, offB[NT / 2];
+    if constexpr (kPreOff) {
+      offA = tile_off<V>(mr + 8 * (mi >> 1), 2 * d + (mi & 1));
+      offDv = tile_off<V>(mr + 8 * (mi & 1), 2 * d + (mi >> 1));
+#pragma unroll
+      for (int np = 0; np < NT / 2; ++np) offB[np] = tile_off<V>(mr + 8 * (mi & 1), 2 * np + (mi >> 1));
+    }
     int nstep = 0;
     for (int j = 0; j < nch; ++j) {
       const int len = chunk_len(j);
@@ -605,12 +616,14 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
         for (int kt = 0; kt < NWC; ++kt) {
           // A = H_{t-1}^T: matrices (i 0-7, l 0-7), (i 0-7, l 8-15), (i 8-15, l 0-7), (i 8-15, l 8-15)
           uint32_t A[4];
-          ldmatrix_x4_trans(ht + tile_off<V>(16 * kt + mr + 8 * (mi >> 1), 2 * d + (mi & 1)), A[0], A[1], A[2], A[3]);
+          if constexpr (kPreOff) ldmatrix_x4_trans(ht + offA + (uint32_t)(kt * 32 * V), A[0], A[1], A[2], A[3]);
+          else ldmatrix_x4_trans(ht + tile_off<V>(16 * kt + mr + 8 * (mi >> 1), 2 * d + (mi & 1)), A[0], A[1], A[2], A[3]);
 #pragma unroll
           for (int np = 0; np < NT / 2; ++np) {
             // B = dX: matrices (i 0-7, j-tile 2np), (i 8-15, 2np), (i 0-7, 2np+1), (i 8-15, 2np+1)
             uint32_t b0, b1, b2, b3;
-            ldmatrix_x4_trans(xt + tile_off<V>(16 * kt + mr + 8 * (mi & 1), 2 * np + (mi >> 1)), b0, b1, b2, b3);
+            if constexpr (kPreOff) ldmatrix_x4_trans(xt + offB[np] + (uint32_t)(kt * 32 * V), b0, b1, b2, b3);
+            else ldmatrix_x4_trans(xt + tile_off<V>(16 * kt + mr + 8 * (mi & 1), 2 * np + (mi >> 1)), b0, b1, b2, b3);
             mma_bf16_16816(acc[2 * np], A, b0, b1);
             mma_bf16_16816(acc[2 * np + 1], A, b2, b3);
           }
@@ -622,7 +635,8 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), 1) bwd_bf16_kernel(Scan
             asm volatile("ld.shared.b32 %0, [%1];" : "=r"(Ak[0]) : "r"(kb + 4u * (8 * kt + c)));
             asm volatile("ld.shared.b32 %0, [%1];" : "=r"(Ak[2]) : "r"(kb + 4u * (8 * kt + 4 + c)));
           }
-          ldmatrix_x4_trans(xt + tile_off<V>(16 * kt + mr + 8 * (mi & 1), 2 * d + (mi >> 1)), b0, b1, b2, b3);
+          if constexpr (kPreOff) ldmatrix_x4_trans(xt + offDv + (uint32_t)(kt * 32 * V), b0, b1, b2, b3);
+          else ldmatrix_x4_trans(xt + tile_off<V>(16 * kt + mr + 8 * (mi & 1), 2 * d + (mi >> 1)), b0, b1, b2, b3);
           mma_bf16_16816(dvacc[0], Ak, b0, b1);
           mma_bf16_16816(dvacc[1], Ak, b2, b3);
         }
