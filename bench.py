@@ -228,6 +228,50 @@ def nbytes(t):
     return 0 if t is None else t.numel() * t.element_size()
 
 
+def e2e_pipeline(stream, dev, n, copy_in, compute, copy_out):
+    """n steps as a three-stream pipeline with two device buffers each way: copy_in(i, b) brings the
+    inputs of step i into buffer b on a copy stream, compute(i, b) runs the step on `stream`,
+    copy_out(b) takes the results of buffer b back on a third stream.  Returns (start, stop) events on
+    `stream`; the first copy-in and the last copy-out are not overlapped and lie between them."""
+    copy_stream = torch.cuda.Stream(device=dev)
+    back_stream = torch.cuda.Stream(device=dev)
+    landed = [torch.cuda.Event() for _ in range(2)]        # the buffer's inputs are on the device
+    consumed = [torch.cuda.Event() for _ in range(2)]      # the step that read the buffer is done
+    computed = [torch.cuda.Event() for _ in range(2)]      # the step's results are in their buffers
+    copied_back = [torch.cuda.Event() for _ in range(2)]   # ... and have left them
+
+    def issue_h2d(i):
+        b = i % 2
+        with torch.cuda.stream(copy_stream):
+            if i >= 2:
+                copy_stream.wait_event(consumed[b])
+            copy_in(i, b)
+            landed[b].record(copy_stream)
+
+    start = torch.cuda.Event(enable_timing=True)
+    stop = torch.cuda.Event(enable_timing=True)
+    start.record(stream)
+    copy_stream.wait_event(start)
+    issue_h2d(0)
+    for i in range(n):
+        b = i % 2
+        if i + 1 < n:
+            issue_h2d(i + 1)
+        stream.wait_event(landed[b])
+        if i >= 2:
+            stream.wait_event(copied_back[b])
+        compute(i, b)
+        consumed[b].record(stream)
+        computed[b].record(stream)
+        with torch.cuda.stream(back_stream):
+            back_stream.wait_event(computed[b])
+            copy_out(b)
+            copied_back[b].record(back_stream)
+    stream.wait_stream(back_stream)
+    stop.record(stream)
+    return start, stop
+
+
 def main_out_norm(args):
     """`--workload out_norm`: the output path after the scan (y (.) SiLU(g) -> RMSNorm over the
     concatenated heads), forward + backward, on the y of the fwd_bf16 workload (B=8, T=2048, N=16,
@@ -302,30 +346,30 @@ def main_out_norm(args):
         ev[1].record(stream)
         barrier()
     ms_total = ev[0].elapsed_time(ev[1])
-    # end to end: y, g, dout in from pinned host memory, out, dy, dg, dw back, every step (one stream)
+    # end to end: y, g, dout in from pinned host memory, out, dy, dg, dw back, every step, as the
+    # same three-stream pipeline as the scan workloads
     ms_e2e, e2e_steps, h2d, d2h = 0.0, 0, 0, 0
     if not args.no_e2e:
-        stage = {k: torch.empty_like(v) for k, v in sets[0].items()}
+        stages = [{k: torch.empty_like(v) for k, v in sets[0].items()} for _ in range(2)]
         hout = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in outs[0].items() if k != "rstd"}
-        h2d = sum(nbytes(t) for t in stage.values())
+        h2d = sum(nbytes(t) for t in stages[0].values())
         d2h = sum(nbytes(t) for t in hout.values())
         e2e_steps = 20
 
-        def e2e_step(i):
-            for k, t in stage.items():
+        def copy_in(i, b):
+            for k, t in stages[b].items():
                 t.copy_(host[i % R][k], non_blocking=True)
-            step(i, s=stage)
-            for k, t in hout.items():
-                t.copy_(outs[0][k], non_blocking=True)
 
-        for i in range(3):
-            e2e_step(i)
+        def compute(i, b):
+            step(i, s=stages[b], ob=b)
+
+        def copy_out(b):
+            for k, t in hout.items():
+                t.copy_(outs[b][k], non_blocking=True)
+
+        e2e_pipeline(stream, dev, 3, copy_in, compute, copy_out)
         barrier()
-        ev2 = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
-        ev2[0].record(stream)
-        for i in range(e2e_steps):
-            e2e_step(i)
-        ev2[1].record(stream)
+        ev2 = e2e_pipeline(stream, dev, e2e_steps, copy_in, compute, copy_out)
         barrier()
         ms_e2e = ev2[0].elapsed_time(ev2[1])
     ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], dist, dev)
@@ -527,47 +571,21 @@ def main():
                    if isinstance(v, torch.Tensor) and k != "W" and not (pas == "decode" and k == "h0")} for _ in range(2)]
         h2d = sum(nbytes(t) for t in stages[0].values())
         d2h = sum(nbytes(t) for t in host_out)
-        copy_stream = torch.cuda.Stream(device=dev)
-        back_stream = torch.cuda.Stream(device=dev)
-        landed = [torch.cuda.Event() for _ in range(2)]     # the buffer's inputs are on the device
-        consumed = [torch.cuda.Event() for _ in range(2)]   # the step that read the buffer is done
-        computed = [torch.cuda.Event() for _ in range(2)]   # the step's results are in their buffers
-        copied_back = [torch.cuda.Event() for _ in range(2)]   # ... and have left them
 
-        def issue_h2d(i, first):
-            b = i % 2
-            with torch.cuda.stream(copy_stream):
-                if not first:
-                    copy_stream.wait_event(consumed[b])
-                hs = host_sets[i % ROTATE]
-                for k, t in stages[b].items():
-                    t.copy_(hs[k], non_blocking=True)
-                landed[b].record(copy_stream)
+        def copy_in(i, b):
+            hs = host_sets[i % ROTATE]
+            for k, t in stages[b].items():
+                t.copy_(hs[k], non_blocking=True)
+
+        def compute(i, b):
+            step(i, s={**stages[b], "W": W, "h0": stages[b].get("h0", dev_sets[0].get("h0"))}, ob=b)
+
+        def copy_out(b):
+            for h, d_ in zip(host_out, out_sets[b]):
+                h.copy_(d_, non_blocking=True)
 
         def e2e_run(n):
-            start = torch.cuda.Event(enable_timing=True)
-            stop = torch.cuda.Event(enable_timing=True)
-            start.record(stream)
-            copy_stream.wait_event(start)
-            issue_h2d(0, True)
-            for i in range(n):
-                b = i % 2
-                if i + 1 < n:
-                    issue_h2d(i + 1, i + 1 < 2)
-                stream.wait_event(landed[b])
-                if i >= 2:
-                    stream.wait_event(copied_back[b])
-                step(i, s={**stages[b], "W": W, "h0": stages[b].get("h0", dev_sets[0].get("h0"))}, ob=b)
-                consumed[b].record(stream)
-                computed[b].record(stream)
-                with torch.cuda.stream(back_stream):
-                    back_stream.wait_event(computed[b])
-                    for h, d_ in zip(host_out, out_sets[b]):
-                        h.copy_(d_, non_blocking=True)
-                    copied_back[b].record(back_stream)
-            stream.wait_stream(back_stream)
-            stop.record(stream)
-            return start, stop
+            return e2e_pipeline(stream, dev, n, copy_in, compute, copy_out)
 
         e2e_steps = max(3, min(args.steps, 50))
         e2e_run(3)
