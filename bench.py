@@ -5,9 +5,11 @@
 
 One "step" is one pass of the scan over one batch of synthetic input of the named workload:
 a forward scan (`fwd_bf16`, the default: B=8, N=16, K=V=64, T=2048; also `long_ctx`,
-`paper_layer`, `tiny_f32`), a forward + backward scan (`bptt_bf16`, `sweep16..128`) or one decoding
-step (`decode`).  Prints ONE JSON line: tokens/s with inputs resident in HBM (`value`), the same
-through host buffers (`e2e`), the achieved fraction of the roofline of the dominant call
+`paper_layer`, `tiny_f32`), a forward + backward scan (`bptt_bf16`, `sweep16..128`), one decoding
+step (`decode`), or the output path after the scan (`out_norm`: gated RMSNorm forward + backward on
+fwd_bf16's y).  `--multi-value` runs a scan workload in the paper's shared q/k head layout.
+Prints ONE JSON line: tokens/s with inputs resident in HBM (`value`), the same
+through host buffers (`e2e`: copy-in, step and copy-out as a three-stream pipeline), the achieved fraction of the roofline of the dominant call
 (`roofline`), the CPU oracle timed on this host (`cpu_baseline`) and the GPU clocks seen while
 timing.
 

@@ -7,6 +7,8 @@ a missing or stale library raises.
     y, hT, ckpt = m2rnn_fwd(q, k, v, gate, W, h0, save_ckpt=True)
     grads       = m2rnn_bwd(q, k, v, gate, W, h0, dy, ckpt=ckpt)
     y1          = m2rnn_decode_step(q1, k1, v1, gate1, W, state)      # state updated in place
+    out, rstd   = m2rnn_gated_norm_fwd(y, g_in, w)                    # RMSNorm(y * SiLU(g)) over N*V
+    grads       = m2rnn_gated_norm_bwd(y, g_in, w, rstd, dout)        # dy, dg, dw
 
 Tensor layouts are the paper's (Algorithm 1/2): q [B,T,Nq,K], k [B,T,Nk,K], v [B,T,N,V],
 gate [B,T,N] fp32, W [N,V,V], h0 [B,N,K,V] fp32.
