@@ -395,7 +395,13 @@ template <int V, int MAXW, bool CKPT>
 cudaError_t launch_vwc(const ScanArgs &a, cudaStream_t s) {
   // two CTAs per SM where there are units to fill them and the slab count leaves the registers
   if constexpr (MAXW == 4 && V <= 64) {
-    if ((long)a.B * a.N * (a.K / a.KCf) > 148) return launch_vwco<V, MAXW, CKPT, 2>(a, s);
+    const long ctas = (long)a.B * a.N * (a.K / a.KCf);
+    // V = 16: the state is small enough for three CTAs per SM, which takes e.g. the 336 units of
+    // the paper's layer shape (84 heads x batch 4) in one wave instead of two
+    if constexpr (V == 16) {
+      if (ctas > 2 * 148) return launch_vwco<V, MAXW, CKPT, 3>(a, s);
+    }
+    if (ctas > 148) return launch_vwco<V, MAXW, CKPT, 2>(a, s);
   }
   return launch_vwco<V, MAXW, CKPT, 1>(a, s);
 }
