@@ -29,6 +29,10 @@ BwdPlan plan_bwd(int B, int N, int K, int V, int io_dtype) {
   int c = 16;
   while (c > 2 && bwd_bf16_smem_bytes(KC, V, c) > kSmemLimit) c -= 2;
   pl.C_max = c;
+  // V = 16 with more CTAs than SMs (the paper's layer shape: 84 heads): a shorter chunk lets two
+  // CTAs share an SM, which saves a wave
+  if (V == 16 && units * (K / KC) > kSMs)
+    while (c > 2 && bwd_bf16_smem_bytes(KC, V, c) > 110 * 1024) c -= 2;
   pl.C = c;
   return pl;
 }

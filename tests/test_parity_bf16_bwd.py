@@ -24,6 +24,7 @@ SHAPES = [
     (40, 9, 4, 64, 64, 0, 0),     # enough units that a CTA takes all 64 rows
     (40, 7, 4, 32, 128, 0, 0),    # ... and the 32-row CTAs of V = 128 (W in shared memory)
     (40, 7, 4, 32, 64, 0, 0),     # two slabs per CTA
+    (40, 15, 4, 64, 16, 1, 1),    # V = 16 with more units than SMs: shorter chunks, two CTAs per SM
 ]
 
 
