@@ -470,7 +470,9 @@ def main():
     bwd = pas == "fwd+bwd"
     io = inputs.torch_dtype(cfg.dtype)
     B, T, N, K, V = cfg.B, cfg.T, cfg.N, cfg.K, cfg.V
-    # ROTATE seeded input sets per rank, resident in HBM; the same sets pinned on the host for e2e.
+    # seeded input sets per rank, resident in HBM; the same sets pinned on the host for e2e (decode: a
+    # ring of 8 token sets, so that every step of a short ring still sees fresh per-token inputs)
+    ROTATE = 8 if pas == "decode" else globals()["ROTATE"]
     # The decode workload rotates its per-token inputs; its state (2 x 1 GB per step) is far above L2.
     host_sets = []
     for r in range(ROTATE):
