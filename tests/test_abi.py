@@ -131,3 +131,38 @@ def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "missing.so"))
     with pytest.raises(ImportError):
         binding.m2rnn_version()
+
+
+def test_plans_for_small_states_with_many_units(lib):
+    """V = 16 with more CTAs than SMs (the paper's layer shape, 84 heads x batch 4): the backward
+    plan shortens the chunk so that two CTAs share an SM; few units keep the long chunk."""
+    many = _p(B=4, N=84, Nq=1, Nk=1, K=64, V=16, T=64)
+    few = _p(B=1, N=4, Nq=1, Nk=1, K=64, V=16, T=64)
+    c_many, c_few = lib.m2rnn_ckpt_interval(ctypes.byref(many)), lib.m2rnn_ckpt_interval(ctypes.byref(few))
+    assert 2 <= c_many < c_few <= 16 and c_many % 2 == 0
+    assert lib.m2rnn_bwd_row_slab(ctypes.byref(many)) == 64        # a CTA keeps the whole state
+    assert lib.m2rnn_bwd_row_slab(ctypes.byref(few)) == 16         # few units: spread the rows over the SMs
+    # a caller may still ask for a longer chunk, up to what one CTA's shared memory holds
+    assert lib.m2rnn_ckpt_interval(ctypes.byref(_p(B=4, N=84, Nq=1, Nk=1, K=64, V=16, T=64, ckpt_interval=12))) == 12
+    assert lib.m2rnn_ckpt_interval(ctypes.byref(_p(B=4, N=84, Nq=1, Nk=1, K=64, V=16, T=64, ckpt_interval=18))) == -3
+
+
+def test_gated_norm_rejects_bad_arguments(lib):
+    f = lib.m2rnn_gated_norm_fwd
+    assert f(-1, 1024, 1, FAKE, FAKE, FAKE, 0.0, 1, FAKE, None, None) == -2
+    assert f(4, 0, 1, FAKE, FAKE, FAKE, 0.0, 1, FAKE, None, None) == -2
+    assert f(4, 1020, 1, FAKE, FAKE, FAKE, 0.0, 1, FAKE, None, None) == -3          # not a multiple of 8
+    assert f(4, 16384, 1, FAKE, FAKE, FAKE, 0.0, 1, FAKE, None, None) == -3         # longer than 8192
+    assert f(4, 1024, 5, FAKE, FAKE, FAKE, 0.0, 1, FAKE, None, None) == -3
+    assert f(4, 1024, 1, None, FAKE, FAKE, 0.0, 1, FAKE, None, None) == -1
+    assert f(4, 1024, 1, ODD, FAKE, FAKE, 0.0, 1, FAKE, None, None) == -4
+    assert f(0, 1024, 1, None, None, None, 0.0, 1, None, None, None) == 0           # an empty call needs no pointers
+    b = lib.m2rnn_gated_norm_bwd
+    need = lib.m2rnn_gated_norm_bwd_workspace_bytes(4096, 1024)
+    assert need > 0 and lib.m2rnn_gated_norm_bwd_workspace_bytes(0, 1024) == 0
+    args = [FAKE] * 4 + [1] + [FAKE] * 4
+    assert b(4096, 1024, 1, *args, None, 0, None) == -5                              # no workspace
+    assert b(4096, 1024, 1, *args, FAKE, need - 1, None) == -5                       # too small
+    assert b(4096, 1024, 1, *args, ODD, need, None) == -4                            # workspace alignment
+    assert b(4096, 1020, 1, *args, FAKE, need, None) == -3
+    assert b(4096, 1024, 1, FAKE, FAKE, FAKE, None, 1, FAKE, FAKE, FAKE, FAKE, FAKE, need, None) == -1   # rstd missing
