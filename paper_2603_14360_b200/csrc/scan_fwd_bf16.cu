@@ -47,7 +47,9 @@ struct FwdSmem {
 // OCC: CTAs per SM the kernel is compiled for.  With more (b,n) units than SMs, two co-resident
 // CTAs (two chain warps per scheduler) hide each other's latencies; the price is a smaller
 // register budget.
-template <int V, int MAXW, bool CKPT, int OCC>
+// NWT: the slab count when it is known at compile time (0: read from the arguments); with it every
+// shared-memory offset of a step is an immediate.
+template <int V, int MAXW, bool CKPT, int OCC, int NWT = 0>
 __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs a) {
   using G = TileGeom<V>;
   constexpr int NT = G::NT, KT = G::KT, SEG = G::SEG;
@@ -59,9 +61,11 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
   constexpr int NSET = V == 128 ? 1 : (KT >= 2 ? 2 : 1);
   extern __shared__ __align__(16) unsigned char smem_raw[];
 
-  const int Kf = a.K, K = a.KCf, N = a.N, T = a.T;   // rows of the whole state / of this CTA's slab
+  const int Kf = a.K, N = a.N, T = a.T;              // rows of the whole state
+  const int K = NWT ? 16 * NWT : a.KCf;              // rows of this CTA's slab
   const int RS = Kf / K;
-  const int NW = K >> 4;
+  const int NW = NWT ? NWT : (K >> 4);
+  constexpr bool kPacked = V <= 64;                  // packed fp32x2 arithmetic (spills at V = 128)
   constexpr int TC = FwdSmem<V>::tc(MAXW * 16);   // K > 64 <=> MAXW == 8
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int bn = blockIdx.x / RS, rs = blockIdx.x % RS, b = bn / N, n = bn % N;
@@ -237,8 +241,16 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
 #pragma unroll
     for (int x = 0; x < SEG / 4; ++x) {
       const float4 v4 = lds128(vrow + 4 * (SEG * c + 4 * x));
-      P[0][2 * x][0] = kk.x * v4.x; P[0][2 * x][1] = kk.x * v4.y; P[0][2 * x][2] = kk.y * v4.x; P[0][2 * x][3] = kk.y * v4.y;
-      P[0][2 * x + 1][0] = kk.x * v4.z; P[0][2 * x + 1][1] = kk.x * v4.w; P[0][2 * x + 1][2] = kk.y * v4.z; P[0][2 * x + 1][3] = kk.y * v4.w;
+      if constexpr (kPacked) {   // one instruction per two products
+        const float2 k02 = make_float2(kk.x, kk.x), k12 = make_float2(kk.y, kk.y);
+        const float2 a0 = __fmul2_rn(k02, make_float2(v4.x, v4.y)), a1 = __fmul2_rn(k12, make_float2(v4.x, v4.y));
+        const float2 b0 = __fmul2_rn(k02, make_float2(v4.z, v4.w)), b1 = __fmul2_rn(k12, make_float2(v4.z, v4.w));
+        P[0][2 * x][0] = a0.x; P[0][2 * x][1] = a0.y; P[0][2 * x][2] = a1.x; P[0][2 * x][3] = a1.y;
+        P[0][2 * x + 1][0] = b0.x; P[0][2 * x + 1][1] = b0.y; P[0][2 * x + 1][2] = b1.x; P[0][2 * x + 1][3] = b1.y;
+      } else {
+        P[0][2 * x][0] = kk.x * v4.x; P[0][2 * x][1] = kk.x * v4.y; P[0][2 * x][2] = kk.y * v4.x; P[0][2 * x][3] = kk.y * v4.y;
+        P[0][2 * x + 1][0] = kk.x * v4.z; P[0][2 * x + 1][1] = kk.x * v4.w; P[0][2 * x + 1][2] = kk.y * v4.z; P[0][2 * x + 1][3] = kk.y * v4.w;
+      }
     }
   };
   // P += A[kt] * W[kt][:]  : one k tile of H W
@@ -273,15 +285,30 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
     for (int kt = 0; kt < KT; ++kt) {
 #pragma unroll
       for (int nt = 2 * kt; nt < 2 * kt + 2; ++nt) {
+        if constexpr (kPacked) {
+          float2 hh[2];
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
-          float x = Pc[0][nt][r];
-          if constexpr (NSET == 2) x += Pc[1][nt][r];
-          const float z = tanh_approx(x);                  // Eq. 1
-          H[nt][r] = fmaf(f, H[nt][r] - z, z);             // Eq. 2: f H + (1-f) Z
+          for (int h = 0; h < 2; ++h) {   // the two rows' column pairs, as packed fp32 pairs
+            float2 x = make_float2(Pc[0][nt][2 * h], Pc[0][nt][2 * h + 1]);
+            if constexpr (NSET == 2) x = __fadd2_rn(x, make_float2(Pc[1][nt][2 * h], Pc[1][nt][2 * h + 1]));
+            const float2 z = make_float2(tanh_approx(x.x), tanh_approx(x.y));                                      // Eq. 1
+            const float2 dd = __ffma2_rn(z, make_float2(-1.f, -1.f), make_float2(H[nt][2 * h], H[nt][2 * h + 1]));  // H - Z
+            hh[h] = __ffma2_rn(make_float2(f, f), dd, z);                                                          // Eq. 2
+            H[nt][2 * h] = hh[h].x; H[nt][2 * h + 1] = hh[h].y;
+          }
+          const float2 pr = __ffma2_rn(make_float2(qq.y, qq.y), hh[1], __fmul2_rn(make_float2(qq.x, qq.x), hh[0]));   // Eq. 3
+          part[2 * nt] = pr.x; part[2 * nt + 1] = pr.y;
+        } else {
+#pragma unroll
+          for (int r = 0; r < 4; ++r) {
+            float x = Pc[0][nt][r];
+            if constexpr (NSET == 2) x += Pc[1][nt][r];
+            const float z = tanh_approx(x);                  // Eq. 1
+            H[nt][r] = fmaf(f, H[nt][r] - z, z);             // Eq. 2: f H + (1-f) Z
+          }
+          part[2 * nt] = fmaf(qq.y, H[nt][2], qq.x * H[nt][0]);      // Eq. 3, this thread's two rows
+          part[2 * nt + 1] = fmaf(qq.y, H[nt][3], qq.x * H[nt][1]);
         }
-        part[2 * nt] = fmaf(qq.y, H[nt][2], qq.x * H[nt][0]);      // Eq. 3, this thread's two rows
-        part[2 * nt + 1] = fmaf(qq.y, H[nt][3], qq.x * H[nt][1]);
       }
       uint32_t Ak[4];
       Ak[0] = pack_bf16(H[2 * kt][0], H[2 * kt][1]);
@@ -355,13 +382,23 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
       vN = stage_sa(sn) + oV;
     }
     if (len == TC) {
+      constexpr int kUnroll = 4;   // steps per loop iteration (TC is a multiple of 4)
 #pragma unroll 1
-      for (int tl = 0; tl < TC - 2; tl += 2) {
-        maybe_checkpoint(2);
-        pair(st, tl, st + oK + 4u * ((tl + 2) * K), st + oV + 4u * ((tl + 2) * V));
+      for (int t0 = 0; t0 < TC - kUnroll; t0 += kUnroll) {
+#pragma unroll
+        for (int u = 0; u < kUnroll; u += 2) {
+          const int tl = t0 + u;
+          maybe_checkpoint(2);
+          pair(st, tl, st + oK + 4u * ((tl + 2) * K), st + oV + 4u * ((tl + 2) * V));
+        }
       }
-      maybe_checkpoint(2);
-      pair(st, TC - 2, kN, vN);
+#pragma unroll
+      for (int u = 0; u < kUnroll; u += 2) {
+        const int tl = TC - kUnroll + u;
+        maybe_checkpoint(2);
+        if (u + 2 < kUnroll) pair(st, tl, st + oK + 4u * ((tl + 2) * K), st + oV + 4u * ((tl + 2) * V));
+        else pair(st, tl, kN, vN);
+      }
     } else {   // ragged last stage
       int tl = 0;
       for (; tl + 1 < len; tl += 2) {
@@ -385,9 +422,18 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
 template <int V, int MAXW, bool CKPT, int OCC>
 cudaError_t launch_vwco(const ScanArgs &a, cudaStream_t s) {
   const size_t smem = FwdSmem<V>::bytes(a.KCf);
+  const unsigned grid = a.B * a.N * (a.K / a.KCf), threads = (a.KCf / 16 + 1) * 32;
+  if constexpr (V == 16 && MAXW == 4) {
+    if (a.KCf == 64) {   // the paper's layer shape (K = 64, V = 16): slab count known at compile time
+      cudaError_t e = cudaFuncSetAttribute(fwd_bf16_kernel<V, MAXW, CKPT, OCC, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+      fwd_bf16_kernel<V, MAXW, CKPT, OCC, 4><<<grid, threads, smem, s>>>(a);
+      return cudaGetLastError();
+    }
+  }
   cudaError_t e = cudaFuncSetAttribute(fwd_bf16_kernel<V, MAXW, CKPT, OCC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  fwd_bf16_kernel<V, MAXW, CKPT, OCC><<<a.B * a.N * (a.K / a.KCf), (a.KCf / 16 + 1) * 32, smem, s>>>(a);
+  fwd_bf16_kernel<V, MAXW, CKPT, OCC><<<grid, threads, smem, s>>>(a);
   return cudaGetLastError();
 }
 
