@@ -35,12 +35,43 @@ from paper_2603_14360_b200.inputs import CONFIGS  # noqa: E402
 
 METRIC = "m2rnn_scan_tokens_per_s"
 ROTATE = 4  # input sets cycled through so that no step finds its inputs in L2
-PASS_OF = {"fwd_bf16": "fwd", "long_ctx": "fwd", "paper_layer": "fwd", "tiny_f32": "fwd", "decode": "decode"}
+PASS_OF = {"fwd_bf16": "fwd", "long_ctx": "fwd", "paper_layer": "fwd", "tiny_f32": "fwd", "decode": "decode"}   # others: fwd+bwd
 SM_COUNT, SM_HZ = 148, 1.965e9
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
-# captures summarised under profiles/ (bptt_bf16: captured at T=512, scaled by 8 -- traffic is per
-# token-head).  None for workloads without a capture of the current kernel.
-NCU_TRAFFIC_BYTES = {"fwd_bf16": 117.4e6, "bptt_bf16": 8 * 658.5e6, "decode": 2.108e9}
+TRAFFIC_TABLE = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+CSRC = os.path.join(ROOT, "paper_2603_14360_b200", "csrc")
+
+
+def kernel_source_digest(cu_file: str) -> str:
+    """Digest of a kernel's translation unit and the headers of its directory: the table's rows are
+    valid for the sources they were captured from, not after a change."""
+    import hashlib
+    h = hashlib.sha256()
+    names = [cu_file] + sorted(f for f in os.listdir(CSRC) if f.endswith((".cuh", ".h")))
+    for f in names:
+        h.update(open(os.path.join(CSRC, f), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def profiled_traffic(workload: str, units: int):
+    """DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the workload's
+    dominant kernel, from the table that `python -m paper_2603_14360_b200.ncu_traffic` writes out of
+    an ncu capture.  A row captured at another sequence length is scaled by the token-heads of a
+    full launch (traffic is per token-head).  None when there is no row, or when the kernel's
+    sources have changed since the capture."""
+    if not os.path.exists(TRAFFIC_TABLE):
+        return None
+    for ln in open(TRAFFIC_TABLE):
+        f = ln.split()
+        if len(f) < 6 or f[0].startswith("#") or f[0] != workload:
+            continue
+        _, kernel, cu_file, bytes_per_launch, units_captured, digest = f[:6]
+        if digest != kernel_source_digest(cu_file):
+            return None
+        scale = units / float(units_captured)
+        return {"bytes": float(bytes_per_launch) * scale,
+                "source": f"profiles/dram_traffic.txt: {kernel}, captured on {units_captured} token-heads"
+                          + ("" if scale == 1 else f", scaled x{scale:g}")}
+    return None
 
 
 def workload_pass(name: str) -> str:
@@ -181,6 +212,49 @@ def oracle_sample_rate(cfg, pas, seconds_target=12.0):
     full_time = dt * (cfg.B * cfg.N) / units * (cfg.T / T_use)
     what = f"{units} of {cfg.B * cfg.N} (b,n) units x T={T_use}" + ("" if T_use == cfg.T else f" of {cfg.T}")
     return cfg.tokens / full_time, f"{what}, {pas}, fp64, 1 thread, scaled by unit (and step) count", dt
+
+
+def oracle_all_cores_rate(cfg, pas, seconds_target=10.0):
+    """The fp32 build of the oracle's loops on every core of this host: whole (b,n) units of the
+    workload handed to a thread pool (units are independent; the C loops run outside the
+    interpreter lock), scaled by the exact ratio of units (and of steps, when one unit alone
+    exceeds the budget).  Returns (tokens/s, cores, description, seconds)."""
+    import concurrent.futures
+    import oracle
+    oracle.build_f32()
+    cores = os.cpu_count() or 1
+    bwd = pas == "fwd+bwd"
+    nb, nn = min(cfg.B, 4), min(cfg.N, max(1, 64 // min(cfg.B, 4)))
+    small = cfg.with_(B=nb, N=nn, Nq=0, Nk=0)
+    d = inputs.make_inputs(small, backward=bwd)
+    names = ("q", "k", "v", "gate", "W", "h0") + (("dy",) if bwd else ())
+    f32 = {x: (None if d[x] is None else d[x].float().numpy()) for x in names}
+
+    def unit_args(b, n, T):
+        out = [f32[x][b:b + 1, :T, n:n + 1] for x in ("q", "k", "v", "gate")]
+        out += [f32["W"][n:n + 1], None if f32["h0"] is None else f32["h0"][b:b + 1, n:n + 1]]
+        return out + ([f32["dy"][b:b + 1, :T, n:n + 1]] if bwd else [])
+
+    def run(a):
+        oracle.fwd_f32(*a[:6])
+        if bwd:
+            oracle.bwd_f32(*a)
+
+    probe_T = min(cfg.T, 64)
+    t0 = time.perf_counter()
+    run(unit_args(0, 0, probe_T))
+    per_step = (time.perf_counter() - t0) / probe_T
+    T_use = cfg.T if per_step * cfg.T <= seconds_target else max(probe_T, int(seconds_target / per_step))
+    rounds = max(1, int(seconds_target / (per_step * T_use)))
+    units = [(u // nn % nb, u % nn) for u in range(min(nb * nn, cores * rounds))]
+    work = [unit_args(b, n, T_use) for (b, n) in units]
+    t0 = time.perf_counter()
+    with concurrent.futures.ThreadPoolExecutor(max_workers=cores) as ex:
+        list(ex.map(run, work))
+    dt = time.perf_counter() - t0
+    full_time = dt * (cfg.B * cfg.N) / len(units) * (cfg.T / T_use)
+    what = f"{len(units)} of {cfg.B * cfg.N} (b,n) units x T={T_use}" + ("" if T_use == cfg.T else f" of {cfg.T}")
+    return cfg.tokens / full_time, min(cores, len(units)), f"{what}, {pas}, fp32 build of the same loops, one unit per thread, scaled by unit (and step) count", dt
 
 
 def run_reference(args, cfg, pas):
@@ -420,39 +494,48 @@ def main_out_norm(args):
         dist.destroy_process_group()
 
 
+def pick_config(args, workload):
+    cfg = CONFIGS["paper_layer" if workload == "paper_layer_bptt" else workload]
+    if workload == "paper_layer_bptt":
+        cfg = cfg.with_(name="paper_layer_bptt")
+    if args.seq_len and workload != "decode":
+        cfg = cfg.with_(T=args.seq_len, name=f"{cfg.name}@T={args.seq_len}")
+    if args.multi_value:   # the paper's layout: one q and one k head shared by all N value heads
+        cfg = cfg.with_(Nq=1, Nk=1, name=f"{cfg.name}+multi_value")
+    return cfg, workload_pass(workload)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=0, help="0: a default per workload")
     ap.add_argument("--warmup", type=int, default=0)
-    ap.add_argument("--workload", default="fwd_bf16", choices=sorted(CONFIGS) + ["out_norm"])
+    ap.add_argument("--workload", default=None, choices=sorted(CONFIGS) + ["paper_layer_bptt", "out_norm"],
+                    help="default: fwd_bf16 as the line's value, with bptt_bf16 (forward + backward) as the sub-object 'bptt'")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-bptt", action="store_true", help="default run: leave the forward + backward sub-object out")
     ap.add_argument("--multi-value", action="store_true",
                     help="run the workload in the multi-value layout (Nq = Nk = 1) instead of multi-head")
     ap.add_argument("--seq-len", type=int, default=0,
                     help="shorten (or lengthen) the workload's T, for profiler captures; the line's workload name says so")
     args = ap.parse_args()
-    if args.workload == "out_norm" and args.impl == "ours":
+    both_halves = args.workload is None and not args.no_bptt and not args.seq_len
+    workload = args.workload or "fwd_bf16"
+    if workload == "out_norm" and args.impl == "ours":
         main_out_norm(args)
         return
-    if args.workload == "out_norm":
+    if workload == "out_norm":
         raise SystemExit("--impl reference times the scan workloads; the out_norm line carries its own cpu_baseline")
-    cfg = CONFIGS[args.workload]
-    if args.seq_len and args.workload != "decode":
-        cfg = cfg.with_(T=args.seq_len, name=f"{cfg.name}@T={args.seq_len}")
-    if args.multi_value:   # the paper's layout: one q and one k head shared by all N value heads
-        cfg = cfg.with_(Nq=1, Nk=1, name=f"{cfg.name}+multi_value")
-    pas = workload_pass(args.workload)
+    cfg, pas = pick_config(args, workload)
 
     if args.impl == "reference":
         args.steps, args.warmup = min(args.steps or 3, 5), min(args.warmup or 1, 1)
         run_reference(args, cfg, pas)
         return
-    if not args.steps:
-        args.steps = {"fwd_bf16": 300, "decode": 1000, "tiny_f32": 300}.get(args.workload, 20)
-    args.warmup = max(args.warmup or (20 if pas != "fwd+bwd" else 3), 3)
+    steps = args.steps or {"fwd_bf16": 300, "decode": 1000, "tiny_f32": 300}.get(workload, 20)
+    warmup = max(args.warmup or (20 if pas != "fwd+bwd" else 3), 3)
 
     from paper_2603_14360_b200 import binding
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -466,7 +549,26 @@ def main():
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
+    env = dict(binding=binding, world=world, rank=rank, local=local, dev=dev, dist=dist)
 
+    line = run_scan_workload(args, workload, cfg, pas, steps, warmup, env)
+    if both_halves:
+        # the other half of the metric: forward + backward through time on the BPTT configuration,
+        # measured the same way (its own roofline, end-to-end and CPU legs), fewer steps
+        cfg2, pas2 = pick_config(args, "bptt_bf16")
+        sub = run_scan_workload(args, "bptt_bf16", cfg2, pas2, max(3, min(steps, 10)), 3, env)
+        if line is not None:
+            line["bptt"] = {k: sub[k] for k in ("value", "unit", "steps", "warmup", "ms_per_step", "ms_fwd", "ms_bwd", "dtype",
+                                                 "config", "roofline", "gpu_launches", "clocks", "e2e", "cpu_baseline") if k in sub}
+    if line is not None:
+        print(json.dumps(line), flush=True)
+    if dist:
+        dist.destroy_process_group()
+
+
+def run_scan_workload(args, workload, cfg, pas, steps, warmup, env):
+    """Times one scan workload; returns the JSON line as a dict on rank 0, None elsewhere."""
+    binding, world, rank, local, dev, dist = (env[k] for k in ("binding", "world", "rank", "local", "dev", "dist"))
     bwd = pas == "fwd+bwd"
     io = inputs.torch_dtype(cfg.dtype)
     B, T, N, K, V = cfg.B, cfg.T, cfg.N, cfg.K, cfg.V
@@ -541,7 +643,7 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
-    for i in range(args.warmup):
+    for i in range(warmup):
         step(i)
     barrier()
     binding.check_device_status()
@@ -549,7 +651,7 @@ def main():
     with ClockSampler(local) as clocks:
         barrier()
         ev[0].record(stream)
-        for i in range(args.steps):
+        for i in range(steps):
             step(i)
         ev[1].record(stream)
         barrier()
@@ -558,7 +660,7 @@ def main():
     # the backward call alone (its kernels only), for the roofline of the dominant call
     ms_bwd = 0.0
     if bwd:
-        reps = min(args.steps, 10)
+        reps = min(steps, 10)
         for i in range(reps):
             step(i, mark=True)
             torch.cuda.synchronize()
@@ -591,7 +693,7 @@ def main():
         def e2e_run(n):
             return e2e_pipeline(stream, dev, n, copy_in, compute, copy_out)
 
-        e2e_steps = max(3, min(args.steps, 50))
+        e2e_steps = max(3, min(steps, 50))
         e2e_run(3)
         barrier()
         ev2 = e2e_run(e2e_steps)
@@ -600,11 +702,9 @@ def main():
 
     ms_total, ms_e2e, ms_bwd = max_over_ranks([ms_total, ms_e2e, ms_bwd], dist, dev)
     if rank != 0:
-        if dist:
-            dist.destroy_process_group()
-        return
+        return None
 
-    ms_step = ms_total / args.steps
+    ms_step = ms_total / steps
     tokens = (B if pas == "decode" else cfg.tokens) * world
     value = whole_job_tokens_per_s(tokens // world, world, ms_step)
     peaks = measured_peaks()
@@ -613,13 +713,14 @@ def main():
     th = B * Tn * N                                              # token-heads per step
     in_bytes = B * Tn * (cfg.nq + cfg.nk) * K * esz + th * V * esz + th * 4          # q,k | v | gate
     state_bytes = 2 * B * N * K * V * 4                                                # h0 in, hT out
+    traffic = None if (args.seq_len or args.multi_value) else profiled_traffic(workload, B * Tn * N)
     if pas == "decode":
         # HBM-bound: the fp32 state is read and written once per step
         alg_bytes = state_bytes + in_bytes + th * V * esz
         achieved = alg_bytes / (ms_step * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if not (args.seq_len or args.multi_value) else None,
-                "call": "m2rnn_decode_step",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": traffic and traffic["bytes"],
+                "traffic_source": traffic and traffic["source"], "call": "m2rnn_decode_step",
                 "peak_source": f"{peaks['source']} HBM copy", "algorithmic_bytes_per_step": alg_bytes}
     else:
         # the contraction(s): forward 2KV^2 per token-head; backward 6KV^2 (recompute, dX W^T, H^T dX)
@@ -628,24 +729,31 @@ def main():
         alg_bytes = in_bytes + th * V * esz + state_bytes
         if bwd:  # + dy in, dq dk dv dgate out, dh0 out (checkpoints are not algorithmic)
             alg_bytes = 2 * in_bytes + th * V * esz + state_bytes
-        achieved = flops / (call_ms * 1e-3) / 1e12
         t_tensor, t_hbm = flops / (peaks["tflops_burst"] * 1e12), alg_bytes / (peaks["hbm_gbs"] * 1e9)
         passes = 2 if bwd else 1                                 # tanh per state element: recompute counts once more
         mufu_s = th * K * V / (16 * SM_COUNT * SM_HZ)
+        # the roofline that bounds the call: the slower of its contraction at the tensor peak and its
+        # streamed bytes at the HBM bandwidth
         if cfg.dtype == "f32":   # the fp32 path is plain FMA: 148 SMs x 128 FMA lanes x 2 flop x 1.965 GHz
             bound, peak, psrc = "alu", SM_COUNT * 128 * 2 * SM_HZ / 1e12, "derived: 148 SMs x 128 fp32 FMA/clk x 1.965 GHz"
-        else:
+            achieved, unit = flops / (call_ms * 1e-3) / 1e12, "TFLOP/s"
+        elif t_tensor >= t_hbm:
             bound, peak, psrc = "tensor", peaks["tflops_burst"], f"{peaks['source']} cuBLAS bf16 burst"
-        roof = {"bound": bound, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if not (args.seq_len or args.multi_value) else None,
+            achieved, unit = flops / (call_ms * 1e-3) / 1e12, "TFLOP/s"
+        else:
+            bound, peak, psrc = "hbm", peaks["hbm_gbs"], f"{peaks['source']} HBM copy"
+            achieved, unit = alg_bytes / (call_ms * 1e-3) / 1e9, "GB/s"
+        roof = {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
+                "frac": achieved / peak, "traffic": traffic and traffic["bytes"],
+                "traffic_source": traffic and traffic["source"],
                 "call": "m2rnn_bwd" if bwd else "m2rnn_fwd", "call_ms": call_ms,
-                "peak_source": psrc,
+                "peak_source": psrc, "algorithmic_bytes_per_call": alg_bytes, "flops_per_call": flops,
                 "t_tensor_ms": t_tensor * 1e3, "t_hbm_ms": t_hbm * 1e3, "t_mufu_ms": mufu_s * 1e3,
                 "frac_of_mufu_ceiling": mufu_s / (call_ms * 1e-3),
                 "ns_per_scan_step": call_ms * 1e6 / T / passes}
     line = {
-        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": steps,
+        "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
         "config": {"workload": cfg.name, "pass": pas, "B": B, "T": Tn, "N": N, "K": K, "V": V,
                    "Nq": cfg.nq, "Nk": cfg.nk, "gate": "logit", "state": "fp32", "accumulate": "fp32",
@@ -653,7 +761,7 @@ def main():
                    "l2": f"{ROTATE} input sets cycled; bytes touched per step {int((alg_bytes) / 1e6)} MB"
                          f" x {ROTATE} sets vs 126 MB L2"},
         "roofline": roof,
-        "gpu_launches": args.steps * launches_per_step,
+        "gpu_launches": steps * launches_per_step,
         "clocks": clocks.summary(),
     }
     if bwd:
@@ -665,9 +773,11 @@ def main():
         rate, desc, dt = oracle_sample_rate(cfg, pas)
         line["cpu_baseline"] = {"value": rate, "unit": "tokens/s", "cores": 1, "kind": "oracle", "sample": desc,
                                 "seconds": dt}
-    print(json.dumps(line), flush=True)
-    if dist:
-        dist.destroy_process_group()
+        if pas != "decode":
+            rate32, cores, desc32, dt32 = oracle_all_cores_rate(cfg, pas)
+            line["cpu_baseline"]["fp32_all_cores"] = {"value": rate32, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                                                      "sample": desc32, "seconds": dt32}
+    return line
 
 
 if __name__ == "__main__":

@@ -25,9 +25,11 @@
  *   - The library allocates nothing and keeps nothing between calls.  Outputs are
  *     overwritten, never accumulated into.
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = the
- *     default stream) and never synchronise.  The return value is an m2rnn_status:
- *     argument errors are reported before anything is launched, launch errors right
- *     after; nothing is launched when an error is returned.
+ *     default stream) and never synchronise.  The return value is an m2rnn_status.
+ *     Argument errors (every code but M2RNN_ERR_CUDA) are found on the host first: nothing
+ *     has been launched when one is returned.  M2RNN_ERR_CUDA means the runtime refused a
+ *     launch or a copy; a call is several launches, earlier ones may already be on the
+ *     stream, and the outputs are then undefined.
  *   - `dev_status` (device int32, may be NULL): every wait inside a kernel is bounded;
  *     if one runs out the kernel stores M2RNN_ERR_TIMEOUT there and returns early.
  *     The caller zeroes it and reads it back after synchronising.
@@ -146,13 +148,17 @@ int m2rnn_bwd(const m2rnn_params *params, const void *q, const void *k, const vo
  * input and output tensor; only the scratch comes from the library.
  *
  * The scratch is a fixed array of M2RNN_STATIC_SCRATCH_BYTES inside the library's device image:
- * every GPU that loads the library holds that much memory until the process exits, whether or
- * not this function is ever called.  The function itself calls no allocating routine.
+ * every GPU that loads the library's device code holds that much memory until the process exits,
+ * whether or not this function is ever called.  The function itself calls no allocating routine.
+ * The CUDA runtime, however, may load a library's device code lazily (its default), and the
+ * array's memory is claimed at that moment: on a device that is already full the first call can
+ * therefore fail with M2RNN_ERR_CUDA.  So make the first call on each device at start-up, while
+ * memory is still to be had (any small problem will do), or run with CUDA_MODULE_LOADING=EAGER.
  *   - A problem whose m2rnn_bwd_workspace_bytes(params, ckpt != NULL) exceeds
  *     M2RNN_STATIC_SCRATCH_BYTES is refused with M2RNN_ERR_WORKSPACE before anything runs;
  *     passing the checkpoints written by m2rnn_fwd lowers the need.
  *   - The first call on each device looks up the array's device address (the device that is
- *     current at the call); make that first call before starting any stream capture.
+ *     current at the call); that same start-up call must come before any stream capture.
  *   - All calls share the one array, which keeps whatever the last call left in it.  Nothing in
  *     it has to start at zero (each call writes what it later reads), but two calls that overlap
  *     on the GPU -- different streams, or different host threads -- race on it: run them one
@@ -173,6 +179,14 @@ int m2rnn_bwd_static_scratch(const m2rnn_params *params, const void *q, const vo
 int m2rnn_decode_step(const m2rnn_params *params, const void *q, const void *k, const void *v,
                       const float *gate, const void *W, const float *alpha, const float *beta,
                       const void *w_r, float *state, void *y, int32_t *dev_status, void *stream);
+
+/* Self-test of the bounded waits (`dev_status` above).  Launches one warp that waits, with the
+ * library's own wait routine and a limit of `limit_cycles` SM clocks (0 .. 1e8), on a barrier that
+ * nothing ever completes.  The wait gives up, the kernel stores M2RNN_ERR_TIMEOUT in *dev_status
+ * and returns normally; the context stays usable.  `waited_cycles` (device int64, may be NULL)
+ * receives the SM clocks the wait took.  The paper has no counterpart: this exercises the
+ * library's failure reporting without making anything fail. */
+int m2rnn_wait_selftest(int64_t limit_cycles, int32_t *dev_status, int64_t *waited_cycles, void *stream);
 
 /* ---- Output path after the scan ("M2RNN block" equations: y_gt = RMSNorm(y_t (.) g_t) with
  * g_t = SiLU of the gate projection; "RMSNormTP Module" appendix for RMSNorm and its backward).

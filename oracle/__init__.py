@@ -34,6 +34,17 @@ def build(force: bool = False, src: str = _SRC, out: str = _LIB) -> str:
     return out
 
 
+def build_f32(force: bool = False) -> str:
+    """Compile the fp32 build of the same loops (m2rnn_ref_f32.c) for the bench's all-cores leg."""
+    src, out = os.path.join(_HERE, "m2rnn_ref_f32.c"), os.path.join(_HERE, "libm2rnn_ref_f32.so")
+    deps = [src, _SRC, os.path.join(_HERE, "m2rnn_ref.h")]
+    if force or not os.path.exists(out) or os.path.getmtime(out) < max(os.path.getmtime(d) for d in deps):
+        tmp = f"{out}.{os.getpid()}.tmp"
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-I", _HERE, "-o", tmp, src, "-lm"])
+        os.replace(tmp, out)
+    return out
+
+
 class _Params(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int), ("T", ctypes.c_int), ("N", ctypes.c_int),
                 ("Nq", ctypes.c_int), ("Nk", ctypes.c_int), ("K", ctypes.c_int),
@@ -193,4 +204,61 @@ def gated_norm_bwd(y, g_in, w, dout, *, eps=0.0, silu=True, lib=None):
                                       _p(out["dy"]), _p(out["dg"]), _p(out["dw"]))
     if rc != 0:
         raise RuntimeError(f"m2rnn_ref_gated_norm_bwd failed: {rc}")
+    return out
+
+
+# ------------------------------------------------------------------ fp32 build (bench leg only)
+class _Params32(ctypes.Structure):
+    _fields_ = _Params._fields_[:-1] + [("dh_clip", ctypes.c_float)]
+
+
+_fp = ctypes.POINTER(ctypes.c_float)
+_lib32 = None
+
+
+def _get32():
+    global _lib32
+    if _lib32 is None:
+        _lib32 = ctypes.CDLL(build_f32())
+        _lib32.m2rnn_ref_fwd.restype = ctypes.c_int
+        _lib32.m2rnn_ref_fwd.argtypes = [ctypes.POINTER(_Params32)] + [_fp] * 12
+        _lib32.m2rnn_ref_bwd.restype = ctypes.c_int
+        _lib32.m2rnn_ref_bwd.argtypes = [ctypes.POINTER(_Params32)] + [_fp] * 17
+    return _lib32
+
+
+def _c32(a):
+    return None if a is None else np.ascontiguousarray(np.asarray(a, dtype=np.float32))
+
+
+def _p32(a):
+    return None if a is None else a.ctypes.data_as(_fp)
+
+
+def fwd_f32(q, k, v, gate, W, h0=None, *, gate_kind=GATE_LOGIT):
+    """The forward loop in its fp32 build -> (y, hT) as float32."""
+    q, k, v, gate, W, h0 = (_c32(a) for a in (q, k, v, gate, W, h0))
+    B, T, N, Nq, Nk, K, V = _shapes(q, k, v, W)
+    y, hT = np.empty((B, T, N, V), np.float32), np.empty((B, N, K, V), np.float32)
+    p = _Params32(B, T, N, Nq, Nk, K, V, gate_kind, 0.0)
+    rc = _get32().m2rnn_ref_fwd(ctypes.byref(p), _p32(q), _p32(k), _p32(v), _p32(gate), _p32(W), _p32(h0),
+                                None, None, None, _p32(y), _p32(hT), None)
+    if rc != 0:
+        raise RuntimeError(f"m2rnn_ref_fwd (fp32 build) failed: {rc}")
+    return y, hT
+
+
+def bwd_f32(q, k, v, gate, W, h0, dy, *, gate_kind=GATE_LOGIT):
+    """The backward loop in its fp32 build -> dict(dq, dk, dv, dgate, dW, dh0) as float32."""
+    q, k, v, gate, W, h0, dy = (_c32(a) for a in (q, k, v, gate, W, h0, dy))
+    B, T, N, Nq, Nk, K, V = _shapes(q, k, v, W)
+    out = dict(dq=np.empty((B, T, Nq, K), np.float32), dk=np.empty((B, T, Nk, K), np.float32),
+               dv=np.empty((B, T, N, V), np.float32), dgate=np.empty((B, T, N), np.float32),
+               dW=np.empty((N, V, V), np.float32), dh0=np.empty((B, N, K, V), np.float32))
+    p = _Params32(B, T, N, Nq, Nk, K, V, gate_kind, 0.0)
+    rc = _get32().m2rnn_ref_bwd(ctypes.byref(p), _p32(q), _p32(k), _p32(v), _p32(gate), _p32(W), _p32(h0),
+                                None, None, None, _p32(dy), None, _p32(out["dq"]), _p32(out["dk"]),
+                                _p32(out["dv"]), _p32(out["dgate"]), _p32(out["dW"]), _p32(out["dh0"]))
+    if rc != 0:
+        raise RuntimeError(f"m2rnn_ref_bwd (fp32 build) failed: {rc}")
     return out

@@ -136,16 +136,17 @@ int m2rnn_ref_decode_step(const m2rnn_ref_params *p, const double *q, const doub
  *
  * Pass 1 keeps every H_t (the algorithm's H_full).  Pass 2 runs t = T-1 .. 0
  * with C = dL/dH_t carried from the later steps (C starts as d_hT, or 0):
- *     G   = C + q_t dy_t^T                 total gradient reaching H_t; the printed
- *                                          "r" is q dy^T alone, which is only right at
- *                                          the last step -- every use of r below takes G
- *     dq  = H_t dy_t                                        (Alg. 2 "dq <- H . dy")
- *     df  = sum( G (.) (H_{t-1} - Z_t) )                    (Alg. 2 "df")
- *     dZ  = (1-f) G ;  dX = dZ (.) (1 - Z (.) Z)            (Alg. 2 "dZ", "dX")
- *     C   = f G + dX W^T          both paths into H_{t-1}: the gated residual
- *                                 ("dH <- r (.) f") plus the transition ("dX . W^T");
- *                                 the printed second dH line multiplies where the
- *                                 chain rule adds
+ *     G   = C + q_t dy_t^T                 total gradient reaching H_t; Algorithm 2's r is
+ *                                          q dy^T alone, which is only right at the last
+ *                                          step -- every use of r below takes G
+ *     dq  = H_t dy_t                                        (Algorithm 2, query-gradient line)
+ *     df  = sum( G (.) (H_{t-1} - Z_t) )                    (Algorithm 2, gate-gradient line)
+ *     dZ  = (1-f) G ;  dX = dZ (.) (1 - Z (.) Z)            (Algorithm 2, candidate and
+ *                                                            pre-activation gradient lines)
+ *     C   = f G + dX W^T          both paths into H_{t-1}: the gated residual (Algorithm 2's
+ *                                 first state-gradient line) plus the path through the
+ *                                 transition (its second one, which as printed multiplies
+ *                                 the two where the chain rule adds them)
  *     dW += H_{t-1}^T dX ;  dk = dX v ;  dv = dX^T k (+ w_r (.) dy from Eq. 3)
  * dq/dk add over the heads sharing them, dW over batch (the algorithm's atomic adds).
  * dh0 = C after the last reverse step. */

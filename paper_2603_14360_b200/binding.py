@@ -61,6 +61,7 @@ EXPORTS = {
     "m2rnn_bwd": (ctypes.c_int, [_pp] + [_vp] * 19 + [ctypes.c_size_t, _vp, _vp]),
     "m2rnn_bwd_static_scratch": (ctypes.c_int, [_pp] + [_vp] * 20),
     "m2rnn_decode_step": (ctypes.c_int, [_pp] + [_vp] * 12),
+    "m2rnn_wait_selftest": (ctypes.c_int, [ctypes.c_int64, _vp, _vp, _vp]),
     "m2rnn_gated_norm_fwd": (ctypes.c_int, [ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, _vp, _vp, _vp, ctypes.c_float,
                                             ctypes.c_int32, _vp, _vp, _vp]),
     "m2rnn_gated_norm_bwd_workspace_bytes": (ctypes.c_size_t, [ctypes.c_int64, ctypes.c_int32]),
@@ -133,6 +134,20 @@ def check_device_status(device=None) -> None:
     if v != 0:
         w.zero_()
         raise M2RNNError(v, "device status")
+
+
+def m2rnn_wait_selftest(limit_cycles: int, device=None, stream=None):
+    """Launches the library's wait self-test: one warp waits, with a limit of ``limit_cycles`` SM
+    clocks, on a barrier nothing completes.  Returns (status word as the kernel left it, SM clocks
+    the wait took); the status must be M2RNN_ERR_TIMEOUT (-7).  Uses words of its own, not the
+    device status word of the scan calls."""
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    waited = torch.zeros(1, dtype=torch.int64, device=dev)
+    rc = _lib().m2rnn_wait_selftest(int(limit_cycles), _ptr(status), _ptr(waited), _stream(stream))
+    if rc != 0:
+        raise M2RNNError(rc, "m2rnn_wait_selftest")
+    return int(status.item()), int(waited.item())
 
 
 def _params(q, k, v, W, gate_kind, ckpt_interval=0, dh_clip=0.0, decode=False) -> Params:

@@ -7,6 +7,18 @@
 
 namespace m2rnn {
 
+// SMs of the current device (the plans size their grids by it); 148, a B200's count, when no device
+// can be asked -- the size queries of the ABI also run on hosts without a GPU.
+int sm_count() {
+  int dev = -1, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
+    (void)cudaGetLastError();
+    return 148;
+  }
+  return sms;
+}
+
 BwdPlan plan_bwd(int B, int N, int K, int V, int io_dtype) {
   BwdPlan pl{};
   if (io_dtype == M2RNN_F32) {  // recomputed states live in global scratch
@@ -16,7 +28,7 @@ BwdPlan plan_bwd(int B, int N, int K, int V, int io_dtype) {
   // Rows per CTA: the largest slab that still spreads the problem over the SMs (rows are independent
   // recurrences; a smaller slab only shortens the work per step).  V = 128 keeps the slab at 32 rows
   // for the sake of registers.
-  constexpr int kSMs = 148;
+  const int kSMs = sm_count();
   const long units = (long)(B > 0 ? B : 1) * N;
   const int cap = V > 64 ? 32 : 64;
   int KC = 16;
@@ -42,7 +54,7 @@ int plan_fwd_rows(int B, int N, int K, int V, int io_dtype) {
   // The smallest slab (a multiple of 16 rows that divides K) that still gives every CTA an SM of
   // its own; with more units than SMs the whole state stays in one CTA.  V = 128 keeps the slab
   // at 64 rows or fewer for the sake of registers.
-  constexpr int kSMs = 148;
+  const int kSMs = sm_count();
   const long units = (long)(B > 0 ? B : 1) * N;
   const int cap = V > 64 ? 32 : 128;
   int best = 0;
@@ -55,6 +67,13 @@ int plan_fwd_rows(int B, int N, int K, int V, int io_dtype) {
 }
 
 namespace {
+
+// A refused launch, attribute or copy: the runtime's last-error slot is cleared here, so that the
+// caller's own next cudaGetLastError() does not report this library's failure a second time.
+int cuda_failed() {
+  (void)cudaGetLastError();
+  return M2RNN_ERR_CUDA;
+}
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -195,7 +214,7 @@ int m2rnn_fwd(const m2rnn_params *params, const void *q, const void *k, const vo
   if (e == cudaSuccess && a.y_part)
     e = launch_reduce_slabs(a.y_part, y, params->io_dtype, params->K / a.KCf,
                             (size_t)params->B * params->T * params->N * params->V, s);
-  return e == cudaSuccess ? M2RNN_OK : M2RNN_ERR_CUDA;
+  return e == cudaSuccess ? M2RNN_OK : cuda_failed();
 }
 
 size_t m2rnn_bwd_workspace_bytes(const m2rnn_params *params, int have_ckpt) {
@@ -221,7 +240,7 @@ int m2rnn_bwd(const m2rnn_params *params, const void *q, const void *k, const vo
       const size_t bytes = sizeof(float) * (size_t)params->B * params->N * params->K * params->V;
       e = d_hT ? cudaMemcpyAsync(dh0, d_hT, bytes, cudaMemcpyDeviceToDevice, s) : cudaMemsetAsync(dh0, 0, bytes, s);
     }
-    return e == cudaSuccess ? M2RNN_OK : M2RNN_ERR_CUDA;
+    return e == cudaSuccess ? M2RNN_OK : cuda_failed();
   }
   if (!q || !k || !v || !gate || !W || !dy || !dq || !dk || !dv || !dgate) return M2RNN_ERR_NULL;
   if (params->gate_kind == M2RNN_GATE_PSI && (!alpha || !beta)) return M2RNN_ERR_NULL;
@@ -246,7 +265,7 @@ int m2rnn_bwd(const m2rnn_params *params, const void *q, const void *k, const vo
     f.y = nullptr; f.hT = nullptr;
     f.ckpt = reinterpret_cast<float *>(ws + w.ckpt);
     e = f32 ? launch_fwd_f32(f, s) : launch_fwd_bf16(f, s);
-    if (e != cudaSuccess) return M2RNN_ERR_CUDA;
+    if (e != cudaSuccess) return cuda_failed();
     a.ckpt = f.ckpt;
   } else {
     a.ckpt = const_cast<float *>(ckpt);
@@ -260,23 +279,23 @@ int m2rnn_bwd(const m2rnn_params *params, const void *q, const void *k, const vo
   a.dv_part = RS > 1 ? reinterpret_cast<float *>(ws + w.dv_part) : nullptr;
   a.dgate_part = RS > 1 ? reinterpret_cast<float *>(ws + w.dgate_part) : nullptr;
   e = f32 ? launch_bwd_f32(a, s) : launch_bwd_bf16(a, s);
-  if (e != cudaSuccess) return M2RNN_ERR_CUDA;
+  if (e != cudaSuccess) return cuda_failed();
   e = launch_reduce_dW(a.dW_part, dW, params->B * RS, params->N, params->V, s);
-  if (e != cudaSuccess) return M2RNN_ERR_CUDA;
+  if (e != cudaSuccess) return cuda_failed();
   const size_t BT = (size_t)params->B * params->T;
   if (RS > 1) {
     e = launch_reduce_slabs(a.dv_part, dv, params->io_dtype, RS, BT * params->N * params->V, s);
-    if (e != cudaSuccess) return M2RNN_ERR_CUDA;
+    if (e != cudaSuccess) return cuda_failed();
     e = launch_reduce_slabs(a.dgate_part, dgate, M2RNN_F32, RS, BT * params->N, s);
-    if (e != cudaSuccess) return M2RNN_ERR_CUDA;
+    if (e != cudaSuccess) return cuda_failed();
   }
   if (a.dq_part) {
     e = launch_reduce_heads(a.dq_part, dq, params->io_dtype, BT, params->N, params->Nq, params->K, s);
-    if (e != cudaSuccess) return M2RNN_ERR_CUDA;
+    if (e != cudaSuccess) return cuda_failed();
   }
   if (a.dk_part) {
     e = launch_reduce_heads(a.dk_part, dk, params->io_dtype, BT, params->N, params->Nk, params->K, s);
-    if (e != cudaSuccess) return M2RNN_ERR_CUDA;
+    if (e != cudaSuccess) return cuda_failed();
   }
   return M2RNN_OK;
 }
@@ -302,7 +321,7 @@ int m2rnn_decode_step(const m2rnn_params *params, const void *q, const void *k, 
   // one step of Eq. 1-3: a T=1 scan whose initial and final state share storage (each CTA reads
   // its own slice of the state completely before it writes it back)
   cudaError_t e = params->io_dtype == M2RNN_F32 ? launch_fwd_f32(a, s) : launch_decode_bf16(a, s);
-  return e == cudaSuccess ? M2RNN_OK : M2RNN_ERR_CUDA;
+  return e == cudaSuccess ? M2RNN_OK : cuda_failed();
 }
 
 }  // extern "C"

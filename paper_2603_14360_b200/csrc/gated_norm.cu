@@ -406,6 +406,7 @@ int m2rnn_gated_norm_fwd(int64_t tokens, int32_t d, int32_t io_dtype, const void
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const cudaError_t e = io_dtype == M2RNN_BF16 ? launch_fwd<__nv_bfloat16>((long)tokens, d, y, g_in, w, eps, silu_on, out, rstd, s)
                                                : launch_fwd<float>((long)tokens, d, y, g_in, w, eps, silu_on, out, rstd, s);
+  if (e != cudaSuccess) (void)cudaGetLastError();   // leave the runtime's last-error slot clear
   return e == cudaSuccess ? M2RNN_OK : M2RNN_ERR_CUDA;
 }
 
@@ -432,7 +433,7 @@ int m2rnn_gated_norm_bwd(int64_t tokens, int32_t d, int32_t io_dtype, const void
   float *part = static_cast<float *>(workspace);
   cudaError_t e = io_dtype == M2RNN_BF16 ? launch_bwd<__nv_bfloat16>((long)tokens, d, y, g_in, w, rstd, silu_on, dout, dy, dg_in, part, s)
                                          : launch_bwd<float>((long)tokens, d, y, g_in, w, rstd, silu_on, dout, dy, dg_in, part, s);
-  if (e != cudaSuccess) return M2RNN_ERR_CUDA;
+  if (e != cudaSuccess) { (void)cudaGetLastError(); return M2RNN_ERR_CUDA; }
   const int partials = (d == 256 || d == 512 || d == 1024) ? reg_grid((long)tokens, d / 256) : grid_for((long)tokens, bwd_warps(d));
   reduce_partials_kernel<<<(d + 31) / 32, 256, 0, s>>>(part, dw, partials, d);
   return cudaGetLastError() == cudaSuccess ? M2RNN_OK : M2RNN_ERR_CUDA;

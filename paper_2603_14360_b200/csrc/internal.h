@@ -48,6 +48,7 @@ struct BwdPlan {
   int C;      // default checkpoint interval
   int C_max;  // largest supported checkpoint interval
 };
+int sm_count();   // SMs of the current device (148 when there is none to ask)
 BwdPlan plan_bwd(int B, int N, int K, int V, int io_dtype);
 int plan_fwd_rows(int B, int N, int K, int V, int io_dtype);   // state rows per CTA of the forward kernel
 size_t bwd_bf16_smem_bytes(int KC, int V, int C);  // scan_bwd_bf16.cu

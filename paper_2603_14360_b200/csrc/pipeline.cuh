@@ -37,9 +37,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
 // kSleepNs > 0: for waits that are expected to be long and whose end nobody is waiting for (a
 // staging warp far ahead of its consumers): the polls of a tight loop would take issue slots
 // from the warps that do the work.
+// `limit` is in SM clocks; the kernels pass the default, the library's self-test a few thousand.
 constexpr long long kWaitCycles = 1ll << 31;
 template <uint32_t kSleepNs = 0>
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, long long limit = kWaitCycles) {
   bool ok = mbar_try_wait(bar, parity);
   if (!ok) {
     const long long t0 = clock64();
@@ -51,7 +52,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
       if (ok) break;
       // the clock is read every 32nd poll only: a poll is a handful of instructions, and polling
       // warps share issue slots with the warps that do the work
-      if ((++it & 31u) == 0u && clock64() - t0 > kWaitCycles) break;
+      if ((++it & 31u) == 0u && clock64() - t0 > limit) break;
     }
   }
   return __all_sync(0xffffffffu, ok);

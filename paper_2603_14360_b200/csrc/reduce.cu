@@ -6,7 +6,7 @@
 namespace m2rnn {
 namespace {
 
-// dW[n] = sum_b dW_part[b][n]   (Algorithm 2: "accumulate dW across batch")
+// dW[n] = sum_b dW_part[b][n]   (Algorithm 2 sums dW over the batch with an atomic add)
 __global__ void reduce_dW_kernel(const float *__restrict__ part, float *__restrict__ dW, int B, size_t NVV) {
   const size_t x = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (x >= NVV) return;
@@ -16,7 +16,7 @@ __global__ void reduce_dW_kernel(const float *__restrict__ part, float *__restri
 }
 
 // out[bt][g][:] = sum over the heads n of group g of part[bt][n][:]
-// (Algorithm 2: "accumulate across shared heads" for dq and dk)
+// (Algorithm 2 sums dq and dk over the heads that share them with atomic adds)
 template <typename TIO>
 __global__ void reduce_heads_kernel(const float *__restrict__ part, TIO *__restrict__ out, size_t BT,
                                     int N, int Ng, int K) {

@@ -445,9 +445,9 @@ cudaError_t launch_vwc(const ScanArgs &a, cudaStream_t s) {
     // V = 16: the state is small enough for three CTAs per SM, which takes e.g. the 336 units of
     // the paper's layer shape (84 heads x batch 4) in one wave instead of two
     if constexpr (V == 16) {
-      if (ctas > 2 * 148) return launch_vwco<V, MAXW, CKPT, 3>(a, s);
+      if (ctas > 2 * sm_count()) return launch_vwco<V, MAXW, CKPT, 3>(a, s);
     }
-    if (ctas > 148) return launch_vwco<V, MAXW, CKPT, 2>(a, s);
+    if (ctas > sm_count()) return launch_vwco<V, MAXW, CKPT, 2>(a, s);
   }
   return launch_vwco<V, MAXW, CKPT, 1>(a, s);
 }

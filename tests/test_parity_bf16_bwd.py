@@ -32,14 +32,16 @@ SHAPES = [
 @pytest.mark.parametrize("gate_kind", [GATE_VALUE, GATE_LOGIT, GATE_PSI])
 def test_shapes_backward(oracle, shape, gate_kind):
     B, T, N, K, V, Nq, Nk = shape
+    # W ~ N(0, 1/V) as in the benchmark configurations for the value and logit gates, half that
+    # scale for the psi gate (short memory: chaotic at full scale, see test_parity_bf16_fwd.W_SCALE)
     cfg = ScanConfig("case", B=B, T=T, N=N, K=K, V=V, Nq=Nq, Nk=Nk, gate_kind=gate_kind, gate_mean=1.0,
-                     w_scale=0.5, seed=300 + T)
+                     w_scale=0.5 if gate_kind == GATE_PSI else 1.0, seed=300 + T)
     errs = parity.check_bwd(oracle, cfg, residual=True, d_hT=True)
-    assert max(errs.values()) < 1e-2, errs
+    assert max(errs.values()) < 1.5e-2, errs
 
 
 def test_checkpoints_recomputed_when_not_passed(oracle):
-    cfg = ScanConfig("nock", B=2, T=29, N=2, K=32, V=64, gate_mean=1.0, w_scale=0.5, seed=21)
+    cfg = ScanConfig("nock", B=2, T=29, N=2, K=32, V=64, gate_mean=1.0, seed=21)
     parity.check_bwd(oracle, cfg, use_fwd_ckpt=False)
 
 
@@ -64,7 +66,7 @@ def test_state_gradient_clipping(oracle):
 
 
 def test_explicit_checkpoint_interval(oracle):
-    cfg = ScanConfig("ck2", B=1, T=23, N=2, K=32, V=32, gate_mean=1.0, w_scale=0.5, seed=13)
+    cfg = ScanConfig("ck2", B=1, T=23, N=2, K=32, V=32, gate_mean=1.0, seed=13)
     d = inputs.make_inputs(cfg, backward=True)
     ref = parity.oracle_bwd(oracle, cfg, d)
     g = parity.to_dev(d)

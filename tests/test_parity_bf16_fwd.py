@@ -9,6 +9,14 @@ from paper_2603_14360_b200.inputs import CONFIGS, GATE_LOGIT, GATE_PSI, GATE_VAL
 
 pytestmark = pytest.mark.gpu
 
+# W ~ N(0, w_scale^2 / V).  The gate tensor and the logits keep the benchmark configurations' scale
+# (w_scale 1: f ~ 0.7, a long memory).  With the psi gate at the same gate mean f ~ 0.2: the state
+# is nearly Z_t alone, and Eq. 1 with W ~ N(0, 1/V) is then a chaotic map for some seeds (the
+# oracle's own amplification of a 1e-6 nudge of h0 reaches 136 within 33 steps on the K = 64, V = 16
+# case, against 1-5 with the other two gates), so that no two implementations agree element by
+# element; w_scale 0.5 keeps those cases about the kernel's arithmetic.
+W_SCALE = {GATE_VALUE: 1.0, GATE_LOGIT: 1.0, GATE_PSI: 0.5}
+
 SHAPES = [
     # B, T, N, K, V, Nq, Nk       T spans several pipeline stages and a ragged tail
     (2, 100, 3, 16, 16, 0, 0),
@@ -28,12 +36,10 @@ SHAPES = [
 @pytest.mark.parametrize("gate_kind", [GATE_VALUE, GATE_LOGIT, GATE_PSI])
 def test_shapes_forward(oracle, shape, gate_kind):
     B, T, N, K, V, Nq, Nk = shape
-    # w_scale 0.5 keeps the recurrence contracting for every gate, so the comparison measures the
-    # kernel's arithmetic and not the inputs' sensitivity (see test_full_size_forward)
     cfg = ScanConfig("case", B=B, T=T, N=N, K=K, V=V, Nq=Nq, Nk=Nk, gate_kind=gate_kind, gate_mean=1.0,
-                     w_scale=0.5, seed=200 + T)
+                     w_scale=W_SCALE[gate_kind], seed=200 + T)
     errs = parity.check_fwd(oracle, cfg, residual=True)
-    assert max(errs.values()) < 1e-2          # typical error is a few 1e-3: bf16 rounding of H, tanh.approx
+    assert max(errs.values()) < 1.5e-2        # typical error is a few 1e-3: bf16 rounding of H, tanh.approx
 
 
 @pytest.mark.parametrize("K,V", [(32, 32), (48, 32), (64, 32), (32, 64), (48, 64), (64, 64), (32, 128), (96, 64), (64, 16)])
@@ -41,9 +47,9 @@ def test_more_units_than_sms(oracle, K, V):
     """152 (b, n) units: every CTA keeps a whole state (two to four 16-row slabs per CTA in the
     column-split kernel, six in the one-warp-per-slab kernel), the launch takes two waves."""
     B = 80 if V == 16 else 38          # V = 16: more than 296 units, three CTAs per SM
-    cfg = ScanConfig("many", B=B, T=37, N=4, K=K, V=V, gate_mean=1.0, w_scale=0.5, seed=300 + K + V)
+    cfg = ScanConfig("many", B=B, T=37, N=4, K=K, V=V, gate_mean=1.0, seed=300 + K + V)
     errs = parity.check_fwd(oracle, cfg)
-    assert max(errs.values()) < 1e-2
+    assert max(errs.values()) < 1.5e-2
 
 
 @pytest.mark.parametrize("K,V", [(16, 16), (64, 64), (128, 128)])
@@ -112,15 +118,12 @@ def _windows(T, width):
 
 @pytest.mark.parametrize("name", ["fwd_bf16"])
 def test_full_size_forward(oracle, name):
-    """The benchmark configuration at full size, in the launch configuration the bench times.
-
-    The map H -> f H + (1-f) tanh(H W + k v^T) with W ~ N(0, 1/V) sits at the edge of
-    stability: over thousands of steps two correct implementations drift apart at a rate set
-    by the inputs, not by the kernel (perturbing h0 by 1e-6 in the oracle itself grows to
-    1e-4 within 256 steps).  So the full scan is checked in two parts that together cover
-    every step: (1) windows of 256 steps restarted from the ORACLE's state must match the
-    oracle within 2e-2; (2) the one-shot full scan must equal, bit for bit, the same windows
-    chained through their own final states.
+    """The benchmark configuration at full size, in the launch configuration the bench times, cut
+    into windows (the free-running comparison over all 2048 steps is in test_full_size.py):
+    (1) windows of 256 steps restarted from the ORACLE's state must match the oracle within 2e-2 on
+    every sampled unit, also on the heads that amplify a difference over a long scan; (2) the
+    one-shot full scan must equal, bit for bit, the same windows chained through their own final
+    states.
     """
     cfg = CONFIGS[name]
     d = inputs.make_inputs(cfg)

@@ -48,7 +48,7 @@ def test_saturating_inputs(oracle, K, V):
     """tanh driven far from its linear range, so a wrong non-linearity cannot pass."""
     cfg = ScanConfig("sat", B=2, T=64, N=2, K=K, V=V, dtype="f32", dist="saturating", gate_mean=0.0, seed=7)
     parity.check_fwd(oracle, cfg)
-    parity.check_bwd(oracle, cfg, tol=1e-3)   # dX = dZ (1 - Z^2) cancels where |Z| -> 1
+    parity.check_bwd(oracle, cfg)
 
 
 def test_no_initial_state_and_split_scan(oracle):
@@ -92,7 +92,7 @@ def test_decode_chain_equals_scan(oracle):
 
 def test_state_gradient_clipping(oracle):
     cfg = ScanConfig("clip", B=2, T=24, N=2, K=16, V=32, dtype="f32", dist="saturating", gate_mean=1.0, seed=9)
-    parity.check_bwd(oracle, cfg, dh_clip=0.05, tol=1e-3)
+    parity.check_bwd(oracle, cfg, dh_clip=0.05)
 
 
 def test_backward_repeats_bit_for_bit(oracle):
