@@ -2,6 +2,9 @@
 // No allocation, no synchronisation, no state kept between calls.
 #include <cuda_runtime.h>
 
+#include <cstdlib>
+#include <cstring>
+
 #include "internal.h"
 #include "m2rnn.h"
 
@@ -49,8 +52,22 @@ BwdPlan plan_bwd(int B, int N, int K, int V, int io_dtype) {
   return pl;
 }
 
+bool fwd_use_tc(int B, int N, int K, int V, int io_dtype) {
+  if (io_dtype != M2RNN_BF16) return false;
+  const char *variant = getenv("M2RNN_FWD_VARIANT");
+  if (variant && !strcmp(variant, "tc")) return true;
+  if (variant && (!strcmp(variant, "mma") || !strcmp(variant, "wide"))) return false;
+  // Measured (B200): the round trip of a tcgen05 step (operand store, proxy fence, barrier, eight
+  // MMAs at ~30 cycles of issue each, commit, mbarrier, tcgen05.ld) is ~400 cycles before any
+  // arithmetic, against ~30 for mma.sync on registers.  It pays only where the register kernels
+  // are bound by the legacy tensor path and there are rows to amortise it over: V = 128 with at
+  // least one 64-row CTA per SM (the K = V = 128 point of the state-size sweep: 6.8 against 7.8 ms).
+  return V == 128 && K % 64 == 0 && (long)(B > 0 ? B : 1) * N * (K / 64) >= sm_count();
+}
+
 int plan_fwd_rows(int B, int N, int K, int V, int io_dtype) {
   if (io_dtype == M2RNN_F32) return K;
+  if (fwd_use_tc(B, N, K, V, io_dtype)) return fwd_tc_rows_per_cta(B, N, K, V);
   // The smallest slab (a multiple of 16 rows that divides K) that still gives every CTA an SM of
   // its own; with more units than SMs the whole state stays in one CTA.  V = 128 keeps the slab
   // at 64 rows or fewer for the sake of registers.
@@ -181,7 +198,8 @@ size_t m2rnn_ckpt_bytes(const m2rnn_params *params) {
 
 size_t m2rnn_fwd_workspace_bytes(const m2rnn_params *params) {
   if (check_params(params, true) != M2RNN_OK) return 0;
-  const int RS = params->K / plan_fwd_rows(params->B, params->N, params->K, params->V, params->io_dtype);
+  const int kcf = plan_fwd_rows(params->B, params->N, params->K, params->V, params->io_dtype);
+  const int RS = (params->K + kcf - 1) / kcf;
   if (RS <= 1) return 0;
   return align_up((size_t)RS * params->B * params->T * params->N * params->V * sizeof(float));
 }
@@ -212,7 +230,7 @@ int m2rnn_fwd(const m2rnn_params *params, const void *q, const void *k, const vo
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   cudaError_t e = params->io_dtype == M2RNN_F32 ? launch_fwd_f32(a, s) : launch_fwd_bf16(a, s);
   if (e == cudaSuccess && a.y_part)
-    e = launch_reduce_slabs(a.y_part, y, params->io_dtype, params->K / a.KCf,
+    e = launch_reduce_slabs(a.y_part, y, params->io_dtype, (params->K + a.KCf - 1) / a.KCf,
                             (size_t)params->B * params->T * params->N * params->V, s);
   return e == cudaSuccess ? M2RNN_OK : cuda_failed();
 }

@@ -51,6 +51,12 @@ struct BwdPlan {
 int sm_count();   // SMs of the current device (148 when there is none to ask)
 BwdPlan plan_bwd(int B, int N, int K, int V, int io_dtype);
 int plan_fwd_rows(int B, int N, int K, int V, int io_dtype);   // state rows per CTA of the forward kernel
+// Which bf16 forward kernel takes a problem: the tcgen05 kernel (scan_fwd_tc.cu) or the mma.sync
+// kernels (scan_fwd_bf16*.cu).  The environment variable M2RNN_FWD_VARIANT = tc | mma | wide
+// overrides the choice (benchmarking only).
+bool fwd_use_tc(int B, int N, int K, int V, int io_dtype);
+int fwd_tc_rows_per_cta(int B, int N, int K, int V);                 // scan_fwd_tc.cu: 32 or 64
+cudaError_t launch_fwd_bf16_tc(const ScanArgs &a, cudaStream_t s);  // scan_fwd_tc.cu
 size_t bwd_bf16_smem_bytes(int KC, int V, int C);  // scan_bwd_bf16.cu
 
 // fp32 FMA path (scan_f32.cu)

@@ -468,6 +468,7 @@ cudaError_t launch_v(const ScanArgs &a, cudaStream_t s) {
 // environment variable M2RNN_FWD_VARIANT=wide forces the one-warp-per-slab kernel of this file
 // (benchmarking only).
 cudaError_t launch_fwd_bf16(const ScanArgs &a, cudaStream_t s) {
+  if (fwd_use_tc(a.B, a.N, a.K, a.V, M2RNN_BF16)) return launch_fwd_bf16_tc(a, s);
   const char *variant = getenv("M2RNN_FWD_VARIANT");
   if (fwd_cs_supported(a) && !(variant && !strcmp(variant, "wide"))) return launch_fwd_bf16_cs(a, s);
   switch (a.V) {

@@ -27,8 +27,9 @@ def test_wait_runs_out_and_reports(limit):
     status, waited = binding.m2rnn_wait_selftest(limit)
     torch.cuda.synchronize()
     assert status == -7                                     # M2RNN_ERR_TIMEOUT
-    # the wait lasted at least its limit and not much longer (the clock is read every 32nd poll)
-    assert waited >= limit and waited <= limit + 200_000, (limit, waited)
+    # the wait lasted at least its limit and not much longer (the clock is read every 32nd poll, and
+    # the polls sleep in between: a millisecond of slack at 2 GHz)
+    assert waited >= limit and waited <= limit + 2_000_000, (limit, waited)
     # the kernel returned normally: the same context runs a scan right after, status word clean
     cfg = ScanConfig("after", B=1, T=8, N=1, K=16, V=16, seed=1)
     g = {k: (v.cuda() if isinstance(v, torch.Tensor) else v) for k, v in inputs.make_inputs(cfg).items()}
