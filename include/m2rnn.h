@@ -13,7 +13,8 @@
  * Conventions for every entry point
  *   - All tensor pointers are DEVICE pointers owned by the caller, contiguous in the
  *     stated layout and 16-byte aligned.  `params` is a HOST pointer.
- *   - Layouts are the paper's (Algorithm 1/2 I/O lists): token-major, heads interleaved.
+ *   - Layouts are the paper's (Algorithm 1/2 I/O lists): token-major, heads interleaved
+ *     (variable-length batches and strided q/k/v: see m2rnn_params).
  *       q [B,T,Nq,K]  k [B,T,Nk,K]  v [B,T,N,V]  gate [B,T,N]  W [N,V,V]
  *       h0,hT [B,N,K,V]  y,dy [B,T,N,V]  alpha,beta [N]  w_r [N,V]
  *     Head n reads q-head n/(N/Nq) and k-head n/(N/Nk) (contiguous groups);
@@ -76,6 +77,20 @@ typedef struct {
   float dh_clip;         /* <= 0: off.  Else the state gradient carried to the previous step is
                             clamped elementwise to [-dh_clip, dh_clip] after every reverse step
                             (section "Gradient Clipping"; the paper gives no threshold or form) */
+  /* Token addressing of the scan calls (m2rnn_fwd, m2rnn_bwd; ignored by the decoding step).
+   * All zero / NULL = the dense layouts above. */
+  int64_t q_stride, k_stride, v_stride; /* elements between consecutive tokens of q, k, v; 0 = dense
+                            (Nq K, Nk K, N V).  A larger stride lets q, k and v be views into one fused
+                            projection output [tokens, Nq K + Nk K + N V + ...]; a token's heads stay
+                            contiguous.  Multiples of 16 bytes.  Outputs and gradients are always dense. */
+  int64_t total_tokens;  /* packed batches (cu_seqlens != NULL): tokens in the batch; else 0 */
+  const int32_t *cu_seqlens; /* DEVICE pointer to B + 1 token offsets, or NULL.  With it the B sequences
+                            are packed one after the other along the token axis: q [total_tokens,Nq,K],
+                            k, v, gate [total_tokens,N], y, dy and the gradients likewise; sequence b is
+                            tokens cu_seqlens[b] .. cu_seqlens[b+1]-1; T is the LONGEST sequence (it
+                            sizes checkpoints and workspaces; a longer sequence is cut to T).  Offsets
+                            are non-decreasing from 0 to total_tokens; a sequence may be empty (its
+                            hT = h0, its dh0 = d_hT).  States stay [B,N,K,V]. */
 } m2rnn_params;
 
 /* Library version: major*10000 + minor*100 + patch. */

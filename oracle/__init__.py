@@ -262,3 +262,49 @@ def bwd_f32(q, k, v, gate, W, h0, dy, *, gate_kind=GATE_LOGIT):
     if rc != 0:
         raise RuntimeError(f"m2rnn_ref_bwd (fp32 build) failed: {rc}")
     return out
+
+
+# ------------------------------------------------------------------ packed variable-length batches
+# A packed batch is B independent sequences laid one after the other along the token axis
+# (sequence b = tokens cu_seqlens[b] .. cu_seqlens[b+1]-1).  The recurrence never couples
+# sequences, so the definition is the dense scan applied to every sequence by itself; dW adds over
+# sequences as it adds over batch entries.
+def fwd_varlen(q, k, v, gate, W, cu_seqlens, h0=None, **kw):
+    """q [tokens,Nq,K], k, v [tokens,N,V], gate [tokens,N], h0 [B,N,K,V] -> (y [tokens,N,V], hT [B,N,K,V])."""
+    q, k, v, gate = (np.asarray(a, dtype=np.float64) for a in (q, k, v, gate))
+    cu = [int(x) for x in cu_seqlens]
+    B, N, K, V = len(cu) - 1, v.shape[1], q.shape[2], v.shape[2]
+    y = np.zeros((q.shape[0], N, V))
+    hT = np.zeros((B, N, K, V))
+    for b in range(B):
+        s, e = cu[b], cu[b + 1]
+        hb = None if h0 is None else np.asarray(h0, dtype=np.float64)[b:b + 1]
+        if e == s:      # an empty sequence leaves its state as it is
+            hT[b] = 0.0 if hb is None else hb[0]
+            continue
+        yb, hTb = fwd(q[None, s:e], k[None, s:e], v[None, s:e], gate[None, s:e], W, hb, **kw)
+        y[s:e], hT[b] = yb[0], hTb[0]
+    return y, hT
+
+
+def bwd_varlen(q, k, v, gate, W, cu_seqlens, h0, dy, d_hT=None, **kw):
+    """Gradients of a packed batch: dq, dk, dv, dgate packed like their tensors, dW summed over the
+    sequences, dh0 [B,N,K,V]."""
+    q, k, v, gate, dy = (np.asarray(a, dtype=np.float64) for a in (q, k, v, gate, dy))
+    cu = [int(x) for x in cu_seqlens]
+    B, N, K, V = len(cu) - 1, v.shape[1], q.shape[2], v.shape[2]
+    out = dict(dq=np.zeros(q.shape), dk=np.zeros(k.shape), dv=np.zeros(v.shape), dgate=np.zeros(gate.shape),
+               dW=np.zeros((N, V, V)), dh0=np.zeros((B, N, K, V)))
+    for b in range(B):
+        s, e = cu[b], cu[b + 1]
+        hb = None if h0 is None else np.asarray(h0, dtype=np.float64)[b:b + 1]
+        db = None if d_hT is None else np.asarray(d_hT, dtype=np.float64)[b:b + 1]
+        if e == s:      # no step: the state gradient passes through unchanged
+            out["dh0"][b] = 0.0 if db is None else db[0]
+            continue
+        r = bwd(q[None, s:e], k[None, s:e], v[None, s:e], gate[None, s:e], W, hb, dy[None, s:e], db, **kw)
+        for x in ("dq", "dk", "dv", "dgate"):
+            out[x][s:e] = r[x][0]
+        out["dW"] += r["dW"]
+        out["dh0"][b] = r["dh0"][0]
+    return out

@@ -42,7 +42,9 @@ class Params(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("T", ctypes.c_int32), ("N", ctypes.c_int32),
                 ("Nq", ctypes.c_int32), ("Nk", ctypes.c_int32), ("K", ctypes.c_int32),
                 ("V", ctypes.c_int32), ("io_dtype", ctypes.c_int32), ("gate_kind", ctypes.c_int32),
-                ("ckpt_interval", ctypes.c_int32), ("dh_clip", ctypes.c_float)]
+                ("ckpt_interval", ctypes.c_int32), ("dh_clip", ctypes.c_float),
+                ("q_stride", ctypes.c_int64), ("k_stride", ctypes.c_int64), ("v_stride", ctypes.c_int64),
+                ("total_tokens", ctypes.c_int64), ("cu_seqlens", ctypes.c_void_p)]
 
 
 _LIB = None
@@ -103,7 +105,7 @@ def _io_code(dtype: torch.dtype) -> int:
     raise TypeError(f"unsupported I/O dtype {dtype}")
 
 
-def _chk(t, name, shape, dtype):
+def _chk(t, name, shape, dtype, strided_tokens=False):
     if t is None:
         return
     if not t.is_cuda:
@@ -112,7 +114,7 @@ def _chk(t, name, shape, dtype):
         raise ValueError(f"{name}: expected shape {tuple(shape)}, got {tuple(t.shape)}")
     if t.dtype != dtype:
         raise TypeError(f"{name}: expected {dtype}, got {t.dtype}")
-    if not t.is_contiguous():
+    if not t.is_contiguous() and not strided_tokens:     # (q, k, v: _token_stride checks the layout)
         raise ValueError(f"{name} must be contiguous")
 
 
@@ -150,14 +152,37 @@ def m2rnn_wait_selftest(limit_cycles: int, device=None, stream=None):
     return int(status.item()), int(waited.item())
 
 
-def _params(q, k, v, W, gate_kind, ckpt_interval=0, dh_clip=0.0, decode=False) -> Params:
+def _token_stride(t, name) -> int:
+    """Elements between consecutive tokens of q, k or v ([B,T,heads,dim] or packed [tokens,heads,dim]).
+    A token's heads must be contiguous and the token axis regular, so that the tensor may be a view
+    into a fused projection output; 0 stands for the dense layout."""
+    if t.stride(-1) != 1 or t.stride(-2) != t.shape[-1]:
+        raise ValueError(f"{name}: the heads of a token must be contiguous")
+    tok = t.stride(-3)
+    if t.dim() == 4 and t.shape[0] > 1 and t.stride(0) != t.shape[1] * tok:
+        raise ValueError(f"{name}: batch entries must follow one another along the token axis")
+    return 0 if tok == t.shape[-2] * t.shape[-1] else tok
+
+
+def _params(q, k, v, W, gate_kind, ckpt_interval=0, dh_clip=0.0, decode=False, cu_seqlens=None,
+            max_seqlen=None) -> Params:
     if decode:
         B, Nq, K = q.shape
         T, Nk, (N, V) = 1, k.shape[1], v.shape[1:]
+        return Params(B, T, N, Nq, Nk, K, V, _io_code(q.dtype), gate_kind, ckpt_interval, dh_clip, 0, 0, 0, 0, None)
+    if cu_seqlens is not None:   # packed variable-length batch: q [tokens, Nq, K]
+        if cu_seqlens.dtype != torch.int32 or not cu_seqlens.is_cuda or not cu_seqlens.is_contiguous():
+            raise TypeError("cu_seqlens must be a contiguous int32 CUDA tensor of B + 1 offsets")
+        if max_seqlen is None:
+            raise ValueError("max_seqlen (the longest sequence) is required with cu_seqlens")
+        total, Nq, K = q.shape
+        B, T, Nk, (N, V) = cu_seqlens.numel() - 1, int(max_seqlen), k.shape[1], v.shape[1:]
     else:
         B, T, Nq, K = q.shape
-        Nk, (N, V) = k.shape[2], v.shape[2:]
-    return Params(B, T, N, Nq, Nk, K, V, _io_code(q.dtype), gate_kind, ckpt_interval, dh_clip)
+        total, Nk, (N, V) = 0, k.shape[2], v.shape[2:]
+    return Params(B, T, N, Nq, Nk, K, V, _io_code(q.dtype), gate_kind, ckpt_interval, dh_clip,
+                  _token_stride(q, "q"), _token_stride(k, "k"), _token_stride(v, "v"), total,
+                  None if cu_seqlens is None else cu_seqlens.data_ptr())
 
 
 def m2rnn_version() -> int:
@@ -187,20 +212,25 @@ def m2rnn_fwd_workspace_bytes(p: Params) -> int:
 
 
 def m2rnn_fwd(q, k, v, gate, W, h0=None, *, gate_kind=GATE_LOGIT, alpha=None, beta=None, w_r=None,
-              save_ckpt=False, ckpt_interval=0, want_hT=True, out=None, workspace=None, stream=None):
+              save_ckpt=False, ckpt_interval=0, want_hT=True, out=None, workspace=None, stream=None,
+              cu_seqlens=None, max_seqlen=None):
     """Forward scan.  Returns (y, hT, ckpt); hT / ckpt are None when not requested.
     ``out`` may hold preallocated ``y`` / ``hT`` / ``ckpt`` tensors to write into; ``workspace``
-    a preallocated uint8 tensor of at least ``m2rnn_fwd_workspace_bytes`` bytes."""
-    p = _params(q, k, v, W, gate_kind, ckpt_interval)
+    a preallocated uint8 tensor of at least ``m2rnn_fwd_workspace_bytes`` bytes.
+    q, k, v may be strided views along the token axis (e.g. slices of one fused projection output).
+    With ``cu_seqlens`` (int32 [B+1], CUDA) and ``max_seqlen`` the batch is packed: q [tokens,Nq,K],
+    k, v, gate [tokens,N], y [tokens,N,V]; states stay [B,N,K,V]."""
+    p = _params(q, k, v, W, gate_kind, ckpt_interval, cu_seqlens=cu_seqlens, max_seqlen=max_seqlen)
     B, T, N, K, V, io = p.B, p.T, p.N, p.K, p.V, q.dtype
-    _chk(q, "q", (B, T, p.Nq, K), io); _chk(k, "k", (B, T, p.Nk, K), io); _chk(v, "v", (B, T, N, V), io)
-    _chk(gate, "gate", (B, T, N), torch.float32); _chk(W, "W", (N, V, V), io)
+    lead = (B, T) if cu_seqlens is None else (q.shape[0],)
+    _chk(q, "q", (*lead, p.Nq, K), io, True); _chk(k, "k", (*lead, p.Nk, K), io, True); _chk(v, "v", (*lead, N, V), io, True)
+    _chk(gate, "gate", (*lead, N), torch.float32); _chk(W, "W", (N, V, V), io)
     _chk(h0, "h0", (B, N, K, V), torch.float32); _chk(w_r, "w_r", (N, V), io)
     _chk(alpha, "alpha", (N,), torch.float32); _chk(beta, "beta", (N,), torch.float32)
     out = out or {}
     y = out.get("y")
     if y is None:
-        y = torch.empty((B, T, N, V), dtype=io, device=q.device)
+        y = torch.empty((*lead, N, V), dtype=io, device=q.device)
     hT = out.get("hT")
     if hT is None and want_hT:
         hT = torch.empty((B, N, K, V), dtype=torch.float32, device=q.device)
@@ -208,7 +238,7 @@ def m2rnn_fwd(q, k, v, gate, W, h0=None, *, gate_kind=GATE_LOGIT, alpha=None, be
     if ckpt is None and save_ckpt:
         C = m2rnn_ckpt_interval(p)
         ckpt = torch.empty((B, N, (T + C - 1) // C, K, V), dtype=torch.float32, device=q.device)
-    _chk(y, "y", (B, T, N, V), io); _chk(hT, "hT", (B, N, K, V), torch.float32)
+    _chk(y, "y", (*lead, N, V), io); _chk(hT, "hT", (B, N, K, V), torch.float32)
     need = m2rnn_fwd_workspace_bytes(p)
     if workspace is None and need > 0:
         workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
@@ -223,15 +253,17 @@ def m2rnn_fwd(q, k, v, gate, W, h0=None, *, gate_kind=GATE_LOGIT, alpha=None, be
 
 def m2rnn_bwd(q, k, v, gate, W, h0, dy, d_hT=None, *, ckpt=None, gate_kind=GATE_LOGIT, alpha=None,
               beta=None, w_r=None, ckpt_interval=0, dh_clip=0.0, want_dh0=True, workspace=None,
-              out=None, stream=None):
-    """Backward through time.  Returns dict(dq, dk, dv, dgate, dW, dh0)."""
-    p = _params(q, k, v, W, gate_kind, ckpt_interval, dh_clip)
+              out=None, stream=None, cu_seqlens=None, max_seqlen=None):
+    """Backward through time.  Returns dict(dq, dk, dv, dgate, dW, dh0) (dense, whatever the strides
+    of q, k, v).  ``cu_seqlens`` / ``max_seqlen``: packed batch, as in ``m2rnn_fwd``."""
+    p = _params(q, k, v, W, gate_kind, ckpt_interval, dh_clip, cu_seqlens=cu_seqlens, max_seqlen=max_seqlen)
     B, T, N, K, V, io = p.B, p.T, p.N, p.K, p.V, q.dtype
-    _chk(q, "q", (B, T, p.Nq, K), io); _chk(k, "k", (B, T, p.Nk, K), io); _chk(v, "v", (B, T, N, V), io)
-    _chk(gate, "gate", (B, T, N), torch.float32); _chk(W, "W", (N, V, V), io)
+    lead = (B, T) if cu_seqlens is None else (q.shape[0],)
+    _chk(q, "q", (*lead, p.Nq, K), io, True); _chk(k, "k", (*lead, p.Nk, K), io, True); _chk(v, "v", (*lead, N, V), io, True)
+    _chk(gate, "gate", (*lead, N), torch.float32); _chk(W, "W", (N, V, V), io)
     _chk(h0, "h0", (B, N, K, V), torch.float32); _chk(w_r, "w_r", (N, V), io)
     _chk(alpha, "alpha", (N,), torch.float32); _chk(beta, "beta", (N,), torch.float32)
-    _chk(dy, "dy", (B, T, N, V), io); _chk(d_hT, "d_hT", (B, N, K, V), torch.float32)
+    _chk(dy, "dy", (*lead, N, V), io); _chk(d_hT, "d_hT", (B, N, K, V), torch.float32)
     if ckpt is not None and T > 0:
         C = m2rnn_ckpt_interval(p)
         _chk(ckpt, "ckpt", (B, N, (T + C - 1) // C, K, V), torch.float32)
@@ -239,12 +271,14 @@ def m2rnn_bwd(q, k, v, gate, W, h0, dy, d_hT=None, *, ckpt=None, gate_kind=GATE_
     out = out or {}
     g = dict(dq=out.get("dq"), dk=out.get("dk"), dv=out.get("dv"), dgate=out.get("dgate"),
              dW=out.get("dW"), dh0=out.get("dh0"))
-    if g["dq"] is None: g["dq"] = torch.empty_like(q)
-    if g["dk"] is None: g["dk"] = torch.empty_like(k)
-    if g["dv"] is None: g["dv"] = torch.empty_like(v)
+    if g["dq"] is None: g["dq"] = torch.empty(q.shape, dtype=io, device=dev)
+    if g["dk"] is None: g["dk"] = torch.empty(k.shape, dtype=io, device=dev)
+    if g["dv"] is None: g["dv"] = torch.empty(v.shape, dtype=io, device=dev)
     if g["dgate"] is None: g["dgate"] = torch.empty_like(gate)
     if g["dW"] is None: g["dW"] = torch.empty((N, V, V), dtype=torch.float32, device=dev)
     if g["dh0"] is None and want_dh0: g["dh0"] = torch.empty((B, N, K, V), dtype=torch.float32, device=dev)
+    for x in ("dq", "dk", "dv"):
+        _chk(g[x], x, {"dq": q, "dk": k, "dv": v}[x].shape, io)
     need = m2rnn_bwd_workspace_bytes(p, ckpt is not None)
     if workspace is None:
         workspace = torch.empty(max(need, 1), dtype=torch.uint8, device=dev)

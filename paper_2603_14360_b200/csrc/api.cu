@@ -107,8 +107,19 @@ int check_params(const m2rnn_params *p, bool need_T) {
     return M2RNN_ERR_UNSUPPORTED;
   // the bf16 kernels take steps in pairs and checkpoint between pairs
   if (p->io_dtype == M2RNN_BF16 && (p->ckpt_interval & 1)) return M2RNN_ERR_UNSUPPORTED;
+  // token strides: at least a token's heads, in 16-byte units
+  const int64_t unit16 = p->io_dtype == M2RNN_BF16 ? 8 : 4;
+  const int64_t dense[3] = {(int64_t)p->Nq * p->K, (int64_t)p->Nk * p->K, (int64_t)p->N * p->V};
+  const int64_t given[3] = {p->q_stride, p->k_stride, p->v_stride};
+  for (int x = 0; x < 3; ++x)
+    if (given[x] != 0 && (given[x] < dense[x] || given[x] % unit16)) return M2RNN_ERR_SHAPE;
+  if (p->total_tokens < 0 || (!p->cu_seqlens && p->total_tokens != 0)) return M2RNN_ERR_SHAPE;
+  if (p->cu_seqlens && (need_T && p->total_tokens > (int64_t)p->B * p->T)) return M2RNN_ERR_SHAPE;
   return M2RNN_OK;
 }
+
+// tokens in the batch
+size_t tokens_of(const m2rnn_params *p) { return p->cu_seqlens ? (size_t)p->total_tokens : (size_t)p->B * p->T; }
 
 int interval_of(const m2rnn_params *p) {
   return p->ckpt_interval ? p->ckpt_interval : plan_bwd(p->B, p->N, p->K, p->V, p->io_dtype).C;
@@ -129,16 +140,17 @@ Workspace layout(const m2rnn_params *p, bool have_ckpt) {
   const int RS = p->K / plan_bwd(p->B, p->N, p->K, p->V, p->io_dtype).KC;   // row slabs per state (1 on the fp32 path)
   w.dW_part = off;
   off += align_up(BN * RS * p->V * p->V * sizeof(float));
+  const size_t TT = tokens_of(p);
   w.dq_part = off;
-  if (p->Nq < p->N) off += align_up((size_t)p->B * p->T * p->N * p->K * sizeof(float));
+  if (p->Nq < p->N) off += align_up(TT * p->N * p->K * sizeof(float));
   w.dk_part = off;
-  if (p->Nk < p->N) off += align_up((size_t)p->B * p->T * p->N * p->K * sizeof(float));
+  if (p->Nk < p->N) off += align_up(TT * p->N * p->K * sizeof(float));
   w.chunk_states = off;
   if (p->io_dtype == M2RNN_F32) off += align_up(BN * C * KV * sizeof(float));
   w.dv_part = off;
-  if (RS > 1) off += align_up((size_t)RS * p->B * p->T * p->N * p->V * sizeof(float));
+  if (RS > 1) off += align_up((size_t)RS * TT * p->N * p->V * sizeof(float));
   w.dgate_part = off;
-  if (RS > 1) off += align_up((size_t)RS * p->B * p->T * p->N * sizeof(float));
+  if (RS > 1) off += align_up((size_t)RS * TT * p->N * sizeof(float));
   w.total = off;
   return w;
 }
@@ -152,6 +164,11 @@ ScanArgs base_args(const m2rnn_params *p) {
   a.C = interval_of(p);
   a.nchunks = p->T > 0 ? (p->T + a.C - 1) / a.C : 0;
   a.dh_clip = p->dh_clip;
+  a.qs = p->q_stride ? p->q_stride : (long long)p->Nq * p->K;
+  a.ks = p->k_stride ? p->k_stride : (long long)p->Nk * p->K;
+  a.vs = p->v_stride ? p->v_stride : (long long)p->N * p->V;
+  a.TT = (long long)tokens_of(p);
+  a.cu = p->cu_seqlens;
   return a;
 }
 
@@ -201,7 +218,7 @@ size_t m2rnn_fwd_workspace_bytes(const m2rnn_params *params) {
   const int kcf = plan_fwd_rows(params->B, params->N, params->K, params->V, params->io_dtype);
   const int RS = (params->K + kcf - 1) / kcf;
   if (RS <= 1) return 0;
-  return align_up((size_t)RS * params->B * params->T * params->N * params->V * sizeof(float));
+  return align_up((size_t)RS * tokens_of(params) * params->N * params->V * sizeof(float));
 }
 
 int m2rnn_fwd(const m2rnn_params *params, const void *q, const void *k, const void *v,
@@ -210,7 +227,7 @@ int m2rnn_fwd(const m2rnn_params *params, const void *q, const void *k, const vo
               void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream) {
   int rc = check_params(params, true);
   if (rc != M2RNN_OK) return rc;
-  if (params->B == 0 || params->T == 0) return M2RNN_OK;
+  if (params->B == 0 || params->T == 0 || tokens_of(params) == 0) return M2RNN_OK;
   if (!q || !k || !v || !gate || !W || !y) return M2RNN_ERR_NULL;
   if (params->gate_kind == M2RNN_GATE_PSI && (!alpha || !beta)) return M2RNN_ERR_NULL;
   const void *ptrs[] = {q, k, v, gate, W, h0, w_r, y, hT, ckpt};
@@ -231,7 +248,7 @@ int m2rnn_fwd(const m2rnn_params *params, const void *q, const void *k, const vo
   cudaError_t e = params->io_dtype == M2RNN_F32 ? launch_fwd_f32(a, s) : launch_fwd_bf16(a, s);
   if (e == cudaSuccess && a.y_part)
     e = launch_reduce_slabs(a.y_part, y, params->io_dtype, (params->K + a.KCf - 1) / a.KCf,
-                            (size_t)params->B * params->T * params->N * params->V, s);
+                            tokens_of(params) * params->N * params->V, s);
   return e == cudaSuccess ? M2RNN_OK : cuda_failed();
 }
 
@@ -250,7 +267,7 @@ int m2rnn_bwd(const m2rnn_params *params, const void *q, const void *k, const vo
   if (rc != M2RNN_OK) return rc;
   if (!dW) return M2RNN_ERR_NULL;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (params->B == 0 || params->T == 0) {
+  if (params->B == 0 || params->T == 0 || tokens_of(params) == 0) {
     // empty scan: the only defined outputs are dW = 0 and dh0 = d_hT (or 0)
     if (!aligned16(dW) || !aligned16(dh0) || !aligned16(d_hT)) return M2RNN_ERR_ALIGN;
     cudaError_t e = cudaMemsetAsync(dW, 0, sizeof(float) * params->N * params->V * params->V, s);
@@ -300,7 +317,7 @@ int m2rnn_bwd(const m2rnn_params *params, const void *q, const void *k, const vo
   if (e != cudaSuccess) return cuda_failed();
   e = launch_reduce_dW(a.dW_part, dW, params->B * RS, params->N, params->V, s);
   if (e != cudaSuccess) return cuda_failed();
-  const size_t BT = (size_t)params->B * params->T;
+  const size_t BT = tokens_of(params);
   if (RS > 1) {
     e = launch_reduce_slabs(a.dv_part, dv, params->io_dtype, RS, BT * params->N * params->V, s);
     if (e != cudaSuccess) return cuda_failed();

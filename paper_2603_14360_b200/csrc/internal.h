@@ -36,7 +36,25 @@ struct ScanArgs {
   float *dk_part;      // [B,T,N,K] fp32 per-head dk when Nk < N, else null
   float *chunk_states; // fp32 path: [B*N, C, K, V] scratch for the recomputed states
   int32_t *dev_status;
+  // token addressing: elements between consecutive tokens of q, k, v (dense: Nq K, Nk K, N V; larger
+  // when they alias one fused projection output), the tokens in the batch (B T, or the packed total)
+  // and, for packed variable-length batches, the device array of B + 1 token offsets
+  long long qs, ks, vs;
+  long long TT;
+  const int32_t *cu;
 };
+
+// First token and length of batch entry b: a slice [cu[b], cu[b+1]) of a packed batch, else b T .. b T + T
+struct UnitSpan { size_t tok0; int T; };
+#ifdef __CUDACC__
+__device__ __forceinline__ UnitSpan unit_span(const ScanArgs &a, int b) {
+  if (a.cu) {   // lengths outside 0 .. T are cut to that range: nothing is addressed beyond what T sized
+    const int s = a.cu[b], len = a.cu[b + 1] - s;
+    return UnitSpan{(size_t)s, len < 0 ? 0 : (len > a.T ? a.T : len)};
+  }
+  return UnitSpan{(size_t)b * a.T, a.T};
+}
+#endif
 
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }

@@ -137,12 +137,16 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), V == 16 ? 2 : 1) bwd_bf
   constexpr int NSET = 1;   // accumulator sets of the state x W product, as in the forward kernel
   extern __shared__ __align__(128) unsigned char smem[];
 
-  const int K = a.K, N = a.N, T = a.T, C = a.C, nch = a.nchunks;
+  const int K = a.K, N = a.N, C = a.C;
   const int RS = K / KC;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, c = lane & 3;
   const int unit = blockIdx.x / RS, rs = blockIdx.x % RS;
   const int b = unit / N, n = unit % N;
+  const UnitSpan span = unit_span(a, b);   // this batch entry's tokens (a slice of a packed batch, or b T ..)
+  const int T = span.T;
+  const size_t tok0 = span.tok0;
+  const int nch = (T + C - 1) / C;             // chunks of this unit (a.nchunks is the checkpoint tensor's extent)
   const int rbase = rs * KC;                   // first state row of this CTA
   const size_t KV = (size_t)K * V;
   const BwdLayout L = bwd_layout<V>(KC, C, kWInSmem);
@@ -258,7 +262,7 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), V == 16 ? 2 : 1) bwd_bf
       const int len = chunk_len(j);
       // the chunk's starting state: ckpt[b][n][chunk] = H before step t0 (fp32)
       float H[NT][4];
-      const float *ck = a.ckpt + ((size_t)unit * nch + (nch - 1 - j)) * KV;
+      const float *ck = a.ckpt + ((size_t)unit * a.nchunks + (nch - 1 - j)) * KV;
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         const float *src = ck + (size_t)(rbase + r0 + 8 * h) * V + SEG * c;
@@ -670,11 +674,11 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), V == 16 ? 2 : 1) bwd_bf
     const __nv_bfloat16 *qg = static_cast<const __nv_bfloat16 *>(a.q), *kg = static_cast<const __nv_bfloat16 *>(a.k);
     const __nv_bfloat16 *vg = static_cast<const __nv_bfloat16 *>(a.v), *dyg = static_cast<const __nv_bfloat16 *>(a.dy);
     const __nv_bfloat16 *wr = static_cast<const __nv_bfloat16 *>(a.w_r);
-    const size_t BT = (size_t)a.B * T;
+    const size_t BT = (size_t)a.TT;
     auto fill = [&](int j) {
       float *sf = slot_f(j);
       const int t0 = chunk_t0(j), len = chunk_len(j);
-      const size_t bt0 = (size_t)b * T + t0;
+      const size_t bt0 = tok0 + t0;
       const int kc8 = KC / 8, v8 = V / 8;
       uint4 *kb = reinterpret_cast<uint4 *>(sf + L.oKB), *vb = reinterpret_cast<uint4 *>(sf + L.oVB);
       uint4 *dyb = reinterpret_cast<uint4 *>(sf + L.oDYB);
@@ -687,12 +691,12 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), V == 16 ? 2 : 1) bwd_bf
         uint4 qr, kr, vr, dr;
         if (x < nk) {
           const int t = x / kc8, i = (x % kc8) * 8;
-          qr = *reinterpret_cast<const uint4 *>(qg + ((bt0 + t) * a.Nq + hq) * K + rbase + i);
-          kr = *reinterpret_cast<const uint4 *>(kg + ((bt0 + t) * a.Nk + hk) * K + rbase + i);
+          qr = *reinterpret_cast<const uint4 *>(qg + (bt0 + t) * a.qs + hq * K + rbase + i);
+          kr = *reinterpret_cast<const uint4 *>(kg + (bt0 + t) * a.ks + hk * K + rbase + i);
         }
         if (x < nv) {
           const int t = x / v8, i = (x % v8) * 8;
-          vr = *reinterpret_cast<const uint4 *>(vg + ((bt0 + t) * N + n) * V + i);
+          vr = *reinterpret_cast<const uint4 *>(vg + (bt0 + t) * a.vs + n * V + i);
           dr = *reinterpret_cast<const uint4 *>(dyg + ((bt0 + t) * N + n) * V + i);
         }
         if (x < nk) {
@@ -720,7 +724,7 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), V == 16 ? 2 : 1) bwd_bf
     auto flush = [&](int j) {
       const float *sf = slot_f(j);
       const int t0 = chunk_t0(j), len = chunk_len(j);
-      const size_t bt0 = (size_t)b * T + t0;
+      const size_t bt0 = tok0 + t0;
       // dq, dk: this CTA's rows
       for (int x = lane; x < len * (KC / 2); x += 32) {
         const int t = x / (KC / 2), i = (x % (KC / 2)) * 2;

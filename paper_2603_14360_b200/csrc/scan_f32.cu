@@ -64,11 +64,14 @@ __device__ __forceinline__ void store_cols(float *__restrict__ base, int c, int 
 template <int NJ4>
 __global__ void __launch_bounds__(1024) fwd_f32_kernel(ScanArgs a, int TPR) {
   extern __shared__ __align__(16) float smem[];
-  const int K = a.K, V = a.V, N = a.N, T = a.T, HP = V + kPad;
+  const int K = a.K, V = a.V, N = a.N, HP = V + kPad;
   const int tid = threadIdx.x, nthreads = blockDim.x, lane = tid & 31, warp = tid >> 5;
   const int nwarps = nthreads >> 5;
   const int i = tid / TPR, c = tid % TPR;
   const int bn = blockIdx.x, b = bn / N, n = bn % N;
+  const UnitSpan span = unit_span(a, b);   // this batch entry's tokens (a slice of a packed batch, or b T ..)
+  const int T = span.T;
+  const size_t tok0 = span.tok0;
   const int hq = n / (N / a.Nq), hk = n / (N / a.Nk);
 
   float *Ws = smem;                    // [V][HP]
@@ -96,14 +99,14 @@ __global__ void __launch_bounds__(1024) fwd_f32_kernel(ScanArgs a, int TPR) {
   __syncthreads();
 
   for (int t = 0; t < T; ++t) {
-    const size_t bt = (size_t)b * T + t;
+    const size_t bt = tok0 + t;
     if (a.ckpt && (t % a.C) == 0)
       store_cols<NJ4>(a.ckpt + ((size_t)bn * a.nchunks + t / a.C) * KV + (size_t)i * V, c, TPR, h);
-    const float k_i = kg[(bt * a.Nk + hk) * K + i];
-    const float q_i = qg[(bt * a.Nq + hq) * K + i];
+    const float k_i = kg[bt * a.ks + hk * K + i];
+    const float q_i = qg[bt * a.qs + hq * K + i];
     const float f = gate_value(a.gate_kind, a.gate[bt * N + n], al, be, nullptr);
     float4 v4[NJ4];
-    load_cols<NJ4>(vg + (bt * N + n) * V, c, TPR, v4);
+    load_cols<NJ4>(vg + bt * a.vs + n * V, c, TPR, v4);
 
     store_cols<NJ4>(Hs + i * HP, c, TPR, h);
     __syncwarp();
@@ -125,7 +128,7 @@ __global__ void __launch_bounds__(1024) fwd_f32_kernel(ScanArgs a, int TPR) {
     if (tid < V) {
       float s = 0.f;
       for (int w = 0; w < nwarps; ++w) s += ypart[((t & 1) * nwarps + w) * V + tid];
-      if (wr) s += wr[(size_t)n * V + tid] * vg[(bt * N + n) * V + tid];
+      if (wr) s += wr[(size_t)n * V + tid] * vg[bt * a.vs + n * V + tid];
       yg[(bt * N + n) * V + tid] = s;
     }
   }
@@ -136,11 +139,14 @@ __global__ void __launch_bounds__(1024) fwd_f32_kernel(ScanArgs a, int TPR) {
 template <int NJ4>
 __global__ void __launch_bounds__(1024) bwd_f32_kernel(ScanArgs a, int TPR) {
   extern __shared__ __align__(16) float smem[];
-  const int K = a.K, V = a.V, N = a.N, T = a.T, HP = V + kPad;
+  const int K = a.K, V = a.V, N = a.N, HP = V + kPad;
   const int tid = threadIdx.x, nthreads = blockDim.x, lane = tid & 31, warp = tid >> 5;
   const int nwarps = nthreads >> 5;
   const int i = tid / TPR, c = tid % TPR;
   const int bn = blockIdx.x, b = bn / N, n = bn % N;
+  const UnitSpan span = unit_span(a, b);   // this batch entry's tokens (a slice of a packed batch, or b T ..)
+  const int T = span.T;
+  const size_t tok0 = span.tok0;
   const int hq = n / (N / a.Nq), hk = n / (N / a.Nk);
 
   float *Ws = smem;                 // [V][HP]
@@ -177,7 +183,7 @@ __global__ void __launch_bounds__(1024) bwd_f32_kernel(ScanArgs a, int TPR) {
   const int ndw = V * V / 4;
   __syncthreads();
 
-  for (int ch = a.nchunks - 1; ch >= 0; --ch) {
+  for (int ch = (T + a.C - 1) / a.C - 1; ch >= 0; --ch) {   // this unit's chunks; a.nchunks is the checkpoint tensor's extent
     const int t0 = ch * a.C, len = min(a.C, T - t0);
     // pass 1 for this chunk: states H_{t0} .. H_{t0+len-1}, each the H_{t-1} of one step
     float h[NJ4 * 4];
@@ -190,11 +196,11 @@ __global__ void __launch_bounds__(1024) bwd_f32_kernel(ScanArgs a, int TPR) {
     for (int s = 0; s < len; ++s) {
       store_cols<NJ4>(scratch + (size_t)s * KV + (size_t)i * V, c, TPR, h);
       if (s == len - 1) break;
-      const size_t bt = (size_t)b * T + t0 + s;
-      const float k_i = kg[(bt * a.Nk + hk) * K + i];
+      const size_t bt = tok0 + t0 + s;
+      const float k_i = kg[bt * a.ks + hk * K + i];
       const float f = gate_value(a.gate_kind, a.gate[bt * N + n], al, be, nullptr);
       float4 v4[NJ4];
-      load_cols<NJ4>(vg + (bt * N + n) * V, c, TPR, v4);
+      load_cols<NJ4>(vg + bt * a.vs + n * V, c, TPR, v4);
       store_cols<NJ4>(Hs + i * HP, c, TPR, h);
       __syncwarp();
       float z[NJ4 * 4];
@@ -206,13 +212,13 @@ __global__ void __launch_bounds__(1024) bwd_f32_kernel(ScanArgs a, int TPR) {
     __syncthreads();
     // pass 2: reverse sweep over the chunk
     for (int s = len - 1; s >= 0; --s) {
-      const size_t bt = (size_t)b * T + t0 + s;
-      const float k_i = kg[(bt * a.Nk + hk) * K + i];
-      const float q_i = qg[(bt * a.Nq + hq) * K + i];
+      const size_t bt = tok0 + t0 + s;
+      const float k_i = kg[bt * a.ks + hk * K + i];
+      const float q_i = qg[bt * a.qs + hq * K + i];
       float dfdx;
       const float f = gate_value(a.gate_kind, a.gate[bt * N + n], al, be, &dfdx);
       float4 v4[NJ4], dy4[NJ4], hp4[NJ4];
-      load_cols<NJ4>(vg + (bt * N + n) * V, c, TPR, v4);
+      load_cols<NJ4>(vg + bt * a.vs + n * V, c, TPR, v4);
       load_cols<NJ4>(dyg + (bt * N + n) * V, c, TPR, dy4);
       load_cols<NJ4>(scratch + (size_t)s * KV + (size_t)i * V, c, TPR, hp4);
       float hp[NJ4 * 4], vv[NJ4 * 4], dyv[NJ4 * 4];

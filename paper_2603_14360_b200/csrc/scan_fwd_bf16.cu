@@ -61,7 +61,7 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
   constexpr int NSET = V == 128 ? 1 : (KT >= 2 ? 2 : 1);
   extern __shared__ __align__(16) unsigned char smem_raw[];
 
-  const int Kf = a.K, N = a.N, T = a.T;              // rows of the whole state
+  const int Kf = a.K, N = a.N;                       // rows of the whole state
   const int K = NWT ? 16 * NWT : a.KCf;              // rows of this CTA's slab
   const int RS = Kf / K;
   const int NW = NWT ? NWT : (K >> 4);
@@ -69,6 +69,9 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
   constexpr int TC = FwdSmem<V>::tc(MAXW * 16);   // K > 64 <=> MAXW == 8
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int bn = blockIdx.x / RS, rs = blockIdx.x % RS, b = bn / N, n = bn % N;
+  const UnitSpan span = unit_span(a, b);   // this batch entry's tokens (a slice of a packed batch, or b T ..)
+  const int T = span.T;
+  const size_t tok0 = span.tok0;
   const int rbase = rs * K;   // first state row of this CTA
   const int stage_floats = FwdSmem<V>::stage_floats(K, TC);
 
@@ -114,7 +117,7 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
     auto fill = [&](int ch) {
       const int s = ch % kStages, t0 = ch * TC, len = min(TC, T - t0);
       float *qS = stages + (size_t)s * stage_floats, *kS = qS + TC * K, *vS = kS + TC * K, *fS = vS + TC * V;
-      const size_t bt0 = (size_t)b * T + t0;
+      const size_t bt0 = tok0 + t0;
       const int kq8 = K / 8, v8 = V / 8;
       uint4 rk[kPerLane], rq[kPerLane], rv[kPerLane];
       float gt = 0.f;
@@ -123,12 +126,12 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
         const int x = lane + 32 * i;
         if (x < len * kq8) {
           const int t = x / kq8, j = (x % kq8) * 8;
-          rk[i] = *reinterpret_cast<const uint4 *>(kg + ((bt0 + t) * a.Nk + hk) * Kf + rbase + j);
-          if (want_y) rq[i] = *reinterpret_cast<const uint4 *>(qg + ((bt0 + t) * a.Nq + hq) * Kf + rbase + j);
+          rk[i] = *reinterpret_cast<const uint4 *>(kg + (bt0 + t) * a.ks + hk * Kf + rbase + j);
+          if (want_y) rq[i] = *reinterpret_cast<const uint4 *>(qg + (bt0 + t) * a.qs + hq * Kf + rbase + j);
         }
         if (x < len * v8) {
           const int t = x / v8, j = (x % v8) * 8;
-          rv[i] = *reinterpret_cast<const uint4 *>(vg + ((bt0 + t) * N + n) * V + j);
+          rv[i] = *reinterpret_cast<const uint4 *>(vg + (bt0 + t) * a.vs + n * V + j);
         }
       }
       if (lane < len) gt = a.gate[(bt0 + lane) * N + n];
@@ -175,9 +178,9 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[e] = fmaf(__bfloat162float(wr[(size_t)n * V + j + e]), vS[t * V + j + e], acc[e]);
           }
-          const size_t yo = (((size_t)b * T + t0 + t) * N + n) * V + j;
+          const size_t yo = ((tok0 + t0 + t) * N + n) * V + j;
           if (a.y_part) {   // this slab's share of y, fp32; the slabs are added by a second kernel
-            float *yp = a.y_part + (size_t)rs * a.B * T * N * V + yo;
+            float *yp = a.y_part + (size_t)rs * a.TT * N * V + yo;
             *reinterpret_cast<float4 *>(yp) = make_float4(acc[0], acc[1], acc[2], acc[3]);
             *reinterpret_cast<float4 *>(yp + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
           } else {

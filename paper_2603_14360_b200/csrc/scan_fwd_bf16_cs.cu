@@ -59,10 +59,13 @@ __global__ void __launch_bounds__((SP * NW + cs_service_warps(SP * NW)) * 32, OC
   extern __shared__ __align__(16) unsigned char smem_raw[];
 
   constexpr int K = 16 * NW;              // rows of this CTA's slab group (NW slabs of 16 rows): a.KCf
-  const int Kf = a.K, N = a.N, T = a.T;   // rows of the whole state
+  const int Kf = a.K, N = a.N;            // rows of the whole state
   const int RS = Kf / K;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int bn = blockIdx.x / RS, rs = blockIdx.x % RS, b = bn / N, n = bn % N;
+  const UnitSpan span = unit_span(a, b);   // this batch entry's tokens (a slice of a packed batch, or b T ..)
+  const int T = span.T;
+  const size_t tok0 = span.tok0;
   const int rbase = rs * K;
   constexpr int stage_floats = CsSmem<V>::stage_floats(K, TC);
 
@@ -102,7 +105,7 @@ __global__ void __launch_bounds__((SP * NW + cs_service_warps(SP * NW)) * 32, OC
     auto fill = [&](int ch) {
       const int s = ch % kStages, t0 = ch * TC, len = min(TC, T - t0);
       float *qS = stages + (size_t)s * stage_floats, *kS = qS + TC * K, *vS = kS + TC * K, *fS = vS + TC * V;
-      const size_t bt0 = (size_t)b * T + t0;
+      const size_t bt0 = tok0 + t0;
       const int kq8 = K / 8, v8 = V / 8;
       uint4 rk[kPerLane], rq[kPerLane], rv[kPerLane];
       float gt = 0.f;
@@ -112,12 +115,12 @@ __global__ void __launch_bounds__((SP * NW + cs_service_warps(SP * NW)) * 32, OC
         const int x = lane + 32 * i;
         if (x < len * kq8) {
           const int t = x / kq8, j = (x % kq8) * 8;
-          rk[i] = *reinterpret_cast<const uint4 *>(kg + ((bt0 + t) * a.Nk + hk) * Kf + rbase + j);
-          if (want_y) rq[i] = *reinterpret_cast<const uint4 *>(qg + ((bt0 + t) * a.Nq + hq) * Kf + rbase + j);
+          rk[i] = *reinterpret_cast<const uint4 *>(kg + (bt0 + t) * a.ks + hk * Kf + rbase + j);
+          if (want_y) rq[i] = *reinterpret_cast<const uint4 *>(qg + (bt0 + t) * a.qs + hq * Kf + rbase + j);
         }
         if (x < len * v8) {
           const int t = x / v8, j = (x % v8) * 8;
-          rv[i] = *reinterpret_cast<const uint4 *>(vg + ((bt0 + t) * N + n) * V + j);
+          rv[i] = *reinterpret_cast<const uint4 *>(vg + (bt0 + t) * a.vs + n * V + j);
         }
       }
       if (sw == kSvc - 1 && lane < len) gt = a.gate[(bt0 + lane) * N + n];
@@ -165,9 +168,9 @@ __global__ void __launch_bounds__((SP * NW + cs_service_warps(SP * NW)) * 32, OC
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[e] = fmaf(__bfloat162float(wr[(size_t)n * V + j + e]), vS[t * V + j + e], acc[e]);
           }
-          const size_t yo = (((size_t)b * T + t0 + t) * N + n) * V + j;
+          const size_t yo = ((tok0 + t0 + t) * N + n) * V + j;
           if (a.y_part) {   // this slab's share of y, fp32; the slabs are added by a second kernel
-            float *yp = a.y_part + (size_t)rs * a.B * T * N * V + yo;
+            float *yp = a.y_part + (size_t)rs * a.TT * N * V + yo;
             *reinterpret_cast<float4 *>(yp) = make_float4(acc[0], acc[1], acc[2], acc[3]);
             *reinterpret_cast<float4 *>(yp + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
           } else {

@@ -120,7 +120,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) fwd_tc_kernel(ScanArgs a) {
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(mma_done + kGroups);
   float *stages = reinterpret_cast<float *>(base + S::oStage);
 
-  const int K = a.K, N = a.N, T = a.T;
+  const int K = a.K, N = a.N;
   // the warp index by way of a shuffle: the compiler then knows it is the same in all lanes, and
   // what is derived from it (the group's tiles and barriers, the MMA descriptors) stays in uniform
   // registers; an MMA issued from values it takes for per-thread ones cost ~65 cycles each
@@ -129,6 +129,9 @@ __global__ void __launch_bounds__(kThreadsTc, 1) fwd_tc_kernel(ScanArgs a) {
   const int RS = (K + kRowsCta - 1) / kRowsCta;   // CTAs per (b, head group)
   const int rs = blockIdx.x % RS, hg = (blockIdx.x / RS) % NG, b = blockIdx.x / (RS * NG);
   const int rbase = rs * kRowsCta;
+  const UnitSpan span = unit_span(a, b);   // this batch entry's tokens (a slice of a packed batch, or b T ..)
+  const int T = span.T;
+  const size_t tok0 = span.tok0;
   const int groups_live = min(kGroups, (K - rbase) / kRowsG);
   const int nchunks = (T + TC - 1) / TC;
   const bool want_y = a.y != nullptr || a.y_part != nullptr;
@@ -189,15 +192,15 @@ __global__ void __launch_bounds__(kThreadsTc, 1) fwd_tc_kernel(ScanArgs a) {
     auto fill = [&](int ch) {
       const int s = ch % kStagesTc, t0 = ch * TC, len = min(TC, T - t0);
       float *st = stages + (size_t)s * S::stage_floats;
-      const size_t bt0 = (size_t)b * T + t0;
+      const size_t bt0 = tok0 + t0;
       // k and q: per (step, head slot) rows_cta bf16 = rows_cta / 8 chunks of 16 bytes
       const int cpr = rows_cta / 8, nkq = len * heads_live * cpr;
       for (int x = sl; x < nkq; x += kSvc) {
         const int c = x % cpr, hs = (x / cpr) % heads_live, t = x / (cpr * heads_live), n = hg * HS + hs;
-        const uint4 rk = *reinterpret_cast<const uint4 *>(kg + ((bt0 + t) * a.Nk + n / dk) * K + rbase + 8 * c);
+        const uint4 rk = *reinterpret_cast<const uint4 *>(kg + (bt0 + t) * a.ks + (n / dk) * K + rbase + 8 * c);
         store8_bf16_as_f32(st + S::kOff + (t * HS + hs) * kRowsCta + 8 * c, rk);
         if (want_y) {
-          const uint4 rq = *reinterpret_cast<const uint4 *>(qg + ((bt0 + t) * a.Nq + n / dq) * K + rbase + 8 * c);
+          const uint4 rq = *reinterpret_cast<const uint4 *>(qg + (bt0 + t) * a.qs + (n / dq) * K + rbase + 8 * c);
           store8_bf16_as_f32(st + S::qOff + (t * HS + hs) * kRowsCta + 8 * c, rq);
         }
       }
@@ -205,7 +208,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) fwd_tc_kernel(ScanArgs a) {
       const int vpr = heads_live * V / 8, nv = len * vpr;
       for (int x = sl; x < nv; x += kSvc) {
         const int c = x % vpr, t = x / vpr;
-        const uint4 rv = *reinterpret_cast<const uint4 *>(vg + ((bt0 + t) * N + hg * HS) * V + 8 * c);
+        const uint4 rv = *reinterpret_cast<const uint4 *>(vg + (bt0 + t) * a.vs + hg * HS * V + 8 * c);
         store8_bf16_as_f32(st + S::vOff + t * 128 + 8 * c, rv);
       }
       for (int x = sl; x < len * heads_live; x += kSvc) {
@@ -243,9 +246,9 @@ __global__ void __launch_bounds__(kThreadsTc, 1) fwd_tc_kernel(ScanArgs a) {
             for (int e = 0; e < 8; ++e)
               acc[e] = fmaf(__bfloat162float(wr[(size_t)hg * 128 + 8 * c + e]), st[S::vOff + t * 128 + 8 * c + e], acc[e]);
           }
-          const size_t yo = (((size_t)b * T + t0 + t) * N + hg * HS) * V + 8 * c;
+          const size_t yo = ((tok0 + t0 + t) * N + hg * HS) * V + 8 * c;
           if (a.y_part) {   // this CTA's share of y, fp32; the shares are added by a second kernel
-            float *yp = a.y_part + (size_t)rs * a.B * T * N * V + yo;
+            float *yp = a.y_part + (size_t)rs * a.TT * N * V + yo;
             *reinterpret_cast<float4 *>(yp) = make_float4(acc[0], acc[1], acc[2], acc[3]);
             *reinterpret_cast<float4 *>(yp + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
           } else {
