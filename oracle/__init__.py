@@ -69,6 +69,10 @@ def load(path: str | None = None) -> ctypes.CDLL:
     lib.m2rnn_ref_gated_norm_fwd.argtypes = [ctypes.c_long, ctypes.c_int] + [_dp] * 3 + [ctypes.c_double, ctypes.c_int] + [_dp] * 2
     lib.m2rnn_ref_gated_norm_bwd.restype = ctypes.c_int
     lib.m2rnn_ref_gated_norm_bwd.argtypes = [ctypes.c_long, ctypes.c_int] + [_dp] * 3 + [ctypes.c_double, ctypes.c_int] + [_dp] * 4
+    lib.m2rnn_ref_conv_silu_fwd.restype = ctypes.c_int
+    lib.m2rnn_ref_conv_silu_fwd.argtypes = [ctypes.c_int] * 3 + [_dp] * 5
+    lib.m2rnn_ref_conv_silu_bwd.restype = ctypes.c_int
+    lib.m2rnn_ref_conv_silu_bwd.argtypes = [ctypes.c_int] * 3 + [_dp] * 9
     return lib
 
 
@@ -204,6 +208,35 @@ def gated_norm_bwd(y, g_in, w, dout, *, eps=0.0, silu=True, lib=None):
                                       _p(out["dy"]), _p(out["dg"]), _p(out["dw"]))
     if rc != 0:
         raise RuntimeError(f"m2rnn_ref_gated_norm_bwd failed: {rc}")
+    return out
+
+
+def conv_silu_fwd(x, w, bias=None, prev=None, *, lib=None):
+    """SiLU(depthwise causal conv1d of width 4 along time): x [B,T,C], w [C,4] (w[:,3] weighs the
+    current token), bias [C], prev [B,3,C] (the three inputs before t = 0; None = zeros) -> out [B,T,C]."""
+    lib = lib or _get()
+    x = _c(x)
+    B, T, C = x.shape
+    w, bias, prev = _c(w, (C, 4)), (None if bias is None else _c(bias, (C,))), (None if prev is None else _c(prev, (B, 3, C)))
+    out = np.empty((B, T, C))
+    rc = lib.m2rnn_ref_conv_silu_fwd(B, T, C, _p(x), _p(w), _p(bias), _p(prev), _p(out))
+    if rc != 0:
+        raise RuntimeError(f"m2rnn_ref_conv_silu_fwd failed: {rc}")
+    return out
+
+
+def conv_silu_bwd(x, w, dout, bias=None, prev=None, *, lib=None):
+    """Backward of conv_silu_fwd -> dict(dx [B,T,C], dw [C,4], dbias [C], dprev [B,3,C])."""
+    lib = lib or _get()
+    x = _c(x)
+    B, T, C = x.shape
+    w, dout = _c(w, (C, 4)), _c(dout, (B, T, C))
+    bias, prev = (None if bias is None else _c(bias, (C,))), (None if prev is None else _c(prev, (B, 3, C)))
+    out = dict(dx=np.empty((B, T, C)), dw=np.empty((C, 4)), dbias=np.empty((C,)), dprev=np.empty((B, 3, C)))
+    rc = lib.m2rnn_ref_conv_silu_bwd(B, T, C, _p(x), _p(w), _p(bias), _p(prev), _p(dout), _p(out["dx"]), _p(out["dw"]),
+                                     _p(out["dbias"]), _p(out["dprev"]))
+    if rc != 0:
+        raise RuntimeError(f"m2rnn_ref_conv_silu_bwd failed: {rc}")
     return out
 
 

@@ -310,3 +310,58 @@ int m2rnn_ref_gated_norm_bwd(long tokens, int d, const double *y, const double *
   }
   return 0;
 }
+
+/* ---------------------------------------------------------------------------------------------
+ * Input path before the scan ("M2RNN block" equations): q_t, k_t, v_t = SiLU(conv1d(projection)),
+ * a depthwise causal convolution of width 4 along time, one filter per channel:
+ *     pre[t][c] = bias[c] + sum_{s=0..3} w[c][s] * x[t-3+s][c],     out = SiLU(pre),
+ * so w[c][3] weighs the current token and w[c][0] the one three steps back (the layout of a
+ * cross-correlation with three zeros padded on the left).  Inputs before t = 0 are zero, or the
+ * three rows of `prev` (the last three inputs of the segment before this one). */
+static double conv_in(const double *x, const double *prev, long b, int T, int C, int t, int c) {
+  if (t >= 0) return x[((size_t)b * T + t) * C + c];
+  return prev ? prev[((size_t)b * 3 + (3 + t)) * C + c] : 0.0;
+}
+
+int m2rnn_ref_conv_silu_fwd(int B, int T, int C, const double *x, const double *w, const double *bias,
+                            const double *prev, double *out) {
+  if (!x || !w || !out || B < 0 || T < 0 || C <= 0) return -1;
+  for (long b = 0; b < B; ++b)
+    for (int t = 0; t < T; ++t)
+      for (int c = 0; c < C; ++c) {
+        double pre = bias ? bias[c] : 0.0;
+        for (int s = 0; s < 4; ++s) pre += w[c * 4 + s] * conv_in(x, prev, b, T, C, t - 3 + s, c);
+        out[((size_t)b * T + t) * C + c] = silu_fn(pre, NULL);
+      }
+  return 0;
+}
+
+/* Its backward: dpre = dout * SiLU'(pre);  dx[t'] = sum_s w[c][s] dpre[t'+3-s] (the steps that
+ * read x[t']);  dw[c][s] = sum_{b,t} dpre[t] x[t-3+s];  dbias[c] = sum_{b,t} dpre[t];
+ * dprev [B,3,C] likewise for the rows of `prev` (may be NULL). */
+int m2rnn_ref_conv_silu_bwd(int B, int T, int C, const double *x, const double *w, const double *bias,
+                            const double *prev, const double *dout, double *dx, double *dw,
+                            double *dbias, double *dprev) {
+  if (!x || !w || !dout || !dx || !dw || B < 0 || T < 0 || C <= 0) return -1;
+  for (int i = 0; i < C * 4; ++i) dw[i] = 0.0;
+  if (dbias) for (int c = 0; c < C; ++c) dbias[c] = 0.0;
+  for (size_t i = 0; i < (size_t)B * T * C; ++i) dx[i] = 0.0;
+  if (dprev) for (size_t i = 0; i < (size_t)B * 3 * C; ++i) dprev[i] = 0.0;
+  for (long b = 0; b < B; ++b)
+    for (int t = 0; t < T; ++t)
+      for (int c = 0; c < C; ++c) {
+        double pre = bias ? bias[c] : 0.0;
+        for (int s = 0; s < 4; ++s) pre += w[c * 4 + s] * conv_in(x, prev, b, T, C, t - 3 + s, c);
+        double dsilu;
+        (void)silu_fn(pre, &dsilu);
+        const double dpre = dout[((size_t)b * T + t) * C + c] * dsilu;
+        if (dbias) dbias[c] += dpre;
+        for (int s = 0; s < 4; ++s) {
+          const int ts = t - 3 + s;
+          dw[c * 4 + s] += dpre * conv_in(x, prev, b, T, C, ts, c);
+          if (ts >= 0) dx[((size_t)b * T + ts) * C + c] += w[c * 4 + s] * dpre;
+          else if (dprev) dprev[((size_t)b * 3 + (3 + ts)) * C + c] += w[c * 4 + s] * dpre;
+        }
+      }
+  return 0;
+}

@@ -79,6 +79,20 @@ int m2rnn_ref_gated_norm_bwd(long tokens, int d, const double *y, const double *
                              double eps, int silu, const double *dout, double *dy, double *dg_in,
                              double *dw);
 
+/* Input path before the scan ("M2RNN block" equations: q_t, k_t, v_t = SiLU(conv1d(projection))):
+ * depthwise causal convolution of width 4 along time, then SiLU.
+ *     pre[b][t][c] = bias[c] + sum_{s=0..3} w[c][s] x[b][t-3+s][c],   out = pre / (1 + exp(-pre))
+ * x, out [B,T,C]; w [C,4] (w[c][3] weighs the current token); bias [C] or NULL; prev [B,3,C] or NULL:
+ * the inputs at t = -3, -2, -1 (NULL: zeros). */
+int m2rnn_ref_conv_silu_fwd(int B, int T, int C, const double *x, const double *w, const double *bias,
+                            const double *prev, double *out);
+
+/* Its backward: dx [B,T,C], dw [C,4] and dbias [C] (may be NULL) summed over batch and time,
+ * dprev [B,3,C] (may be NULL). */
+int m2rnn_ref_conv_silu_bwd(int B, int T, int C, const double *x, const double *w, const double *bias,
+                            const double *prev, const double *dout, double *dx, double *dw,
+                            double *dbias, double *dprev);
+
 #ifdef __cplusplus
 }
 #endif

@@ -37,6 +37,14 @@ MUTANTS = [
     ("norm_bwd_dg_uses_gate", "dg_in[t * d + j] = dx * yt[j] * dsilu;", "dg_in[t * d + j] = dx * g * dsilu;"),
     ("norm_bwd_dw_without_s", "dw[j] += dot[j] * x * s;", "dw[j] += dot[j] * x;"),
     ("norm_bwd_silu_derivative", "if (dx) *dx = sg * (1.0 + x * (1.0 - sg));", "if (dx) *dx = sg * (1.0 - sg);"),
+    ("conv_taps_reversed", "pre += w[c * 4 + s] * conv_in(x, prev, b, T, C, t - 3 + s, c);\n        out", "pre += w[c * 4 + 3 - s] * conv_in(x, prev, b, T, C, t - 3 + s, c);\n        out"),
+    ("conv_not_causal", "conv_in(x, prev, b, T, C, t - 3 + s, c);\n        out", "conv_in(x, prev, b, T, C, (t + s < T ? t + s : T - 1), c);\n        out"),
+    ("conv_prev_rows_reversed", "prev[((size_t)b * 3 + (3 + t)) * C + c]", "prev[((size_t)b * 3 + (-1 - t)) * C + c]"),
+    ("conv_bias_dropped", "double pre = bias ? bias[c] : 0.0;\n        for (int s = 0; s < 4; ++s) pre += w[c * 4 + s] * conv_in(x, prev, b, T, C, t - 3 + s, c);\n        out",
+     "double pre = 0.0;\n        for (int s = 0; s < 4; ++s) pre += w[c * 4 + s] * conv_in(x, prev, b, T, C, t - 3 + s, c);\n        out"),
+    ("conv_bwd_silu_slope_dropped", "const double dpre = dout[((size_t)b * T + t) * C + c] * dsilu;", "const double dpre = dout[((size_t)b * T + t) * C + c];"),
+    ("conv_bwd_dx_wrong_tap", "dx[((size_t)b * T + ts) * C + c] += w[c * 4 + s] * dpre;", "dx[((size_t)b * T + ts) * C + c] += w[c * 4 + 3 - s] * dpre;"),
+    ("conv_bwd_dw_uses_current_token", "dw[c * 4 + s] += dpre * conv_in(x, prev, b, T, C, ts, c);", "dw[c * 4 + s] += dpre * conv_in(x, prev, b, T, C, t, c);"),
     ("bwd_dh0_seed_ignored", "if (d_hT) memcpy(C, d_hT + bn * KV, sizeof(double) * KV);\n      else memset", "memset"),
 ]
 
@@ -48,12 +56,14 @@ PIN_CALLS = [
     functools.partial(pins.test_bwd_matches_finite_differences, gate_kind=2, shared=True),
     pins.test_gated_norm_by_hand, pins.test_gated_norm_invariants, pins.test_gated_norm_bwd_matches_autograd,
     functools.partial(pins.test_gated_norm_bwd_matches_finite_differences, silu=True),
+    pins.test_conv_silu_by_hand, pins.test_conv_silu_matches_torch_and_is_causal, pins.test_conv_silu_bwd_matches_autograd,
+    pins.test_conv_silu_bwd_matches_finite_differences,
 ]
 
 
 def _proxy(oracle, lib):
     ns = types.SimpleNamespace()
-    for name in ("fwd", "bwd", "decode_step", "gate_fn", "gated_norm_fwd", "gated_norm_bwd"):
+    for name in ("fwd", "bwd", "decode_step", "gate_fn", "gated_norm_fwd", "gated_norm_bwd", "conv_silu_fwd", "conv_silu_bwd"):
         setattr(ns, name, functools.partial(getattr(oracle, name), lib=lib))
     return ns
 

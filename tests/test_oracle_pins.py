@@ -402,3 +402,77 @@ def test_gated_norm_bwd_matches_autograd(oracle):
     np.testing.assert_allclose(got["dy"], ty.grad.numpy(), rtol=1e-12, atol=1e-14)
     np.testing.assert_allclose(got["dg"], tg.grad.numpy(), rtol=1e-12, atol=1e-14)
     np.testing.assert_allclose(got["dw"], tw.grad.numpy(), rtol=1e-12, atol=1e-14)
+
+
+# ---------------------------------------------------------------- input path: SiLU(conv1d(.))
+def test_conv_silu_by_hand(oracle):
+    """One channel, taps (w0..w3) = (1, 10, 100, 1000) on x = (1, 2, 3, 4, 5): the current token is
+    weighed by w3 and the window is causal, so pre = (1000, 2100, 3210, 4321, 5432); a bias adds
+    to every step.  SiLU is checked at values where e^-x is a rational number."""
+    x = np.arange(1.0, 6.0).reshape(1, 5, 1)
+    w = np.array([[1.0, 10.0, 100.0, 1000.0]])
+    big = oracle.conv_silu_fwd(x, w)                       # pre >= 1000: SiLU(pre) = pre to fp64
+    np.testing.assert_allclose(big.reshape(-1), [1000.0, 2100.0, 3210.0, 4321.0, 5432.0], rtol=1e-15)
+    prev = np.array([[[7.0], [8.0], [9.0]]])               # inputs at t = -3, -2, -1
+    withprev = oracle.conv_silu_fwd(x, w, prev=prev)
+    np.testing.assert_allclose(withprev.reshape(-1)[:3], [1000 + 900 + 80 + 7, 2100 + 90 + 8, 3210 + 9], rtol=1e-15)
+    np.testing.assert_allclose(withprev.reshape(-1)[3:], big.reshape(-1)[3:], rtol=0)
+    # SiLU(ln 3) = ln 3 / (1 + 1/3);  SiLU(-ln 3) = -ln 3 / (1 + 3)
+    ln3 = np.log(3.0)
+    small = oracle.conv_silu_fwd(np.array([[[1.0], [-1.0]]]), np.array([[0.0, 0.0, 0.0, ln3]]))
+    np.testing.assert_allclose(small.reshape(-1), [0.75 * ln3, -0.25 * ln3], rtol=1e-15)
+    withbias = oracle.conv_silu_fwd(np.zeros((1, 2, 1)), np.array([[0.0, 0.0, 0.0, 1.0]]), bias=np.array([ln3]))
+    np.testing.assert_allclose(withbias.reshape(-1), [0.75 * ln3] * 2, rtol=1e-15)
+
+
+def test_conv_silu_matches_torch_and_is_causal(oracle):
+    rng = np.random.default_rng(61)
+    B, T, C = 3, 11, 5
+    x, w, bias = rng.standard_normal((B, T, C)), rng.standard_normal((C, 4)), rng.standard_normal(C)
+    out = oracle.conv_silu_fwd(x, w, bias)
+    # library routine: depthwise cross-correlation over time with three zeros on the left, then SiLU
+    xt = torch.nn.functional.pad(torch.from_numpy(x).transpose(1, 2), (3, 0))
+    ref = torch.nn.functional.silu(torch.nn.functional.conv1d(xt, torch.from_numpy(w)[:, None, :], torch.from_numpy(bias), groups=C))
+    np.testing.assert_allclose(out, ref.transpose(1, 2).numpy(), rtol=1e-13, atol=1e-15)
+    # causal: changing inputs after step 6 changes no output up to step 6
+    x2 = x.copy()
+    x2[:, 7:] += 1.0
+    np.testing.assert_array_equal(oracle.conv_silu_fwd(x2, w, bias)[:, :7], out[:, :7])
+    # a segment continued through `prev` equals the one-shot result
+    tail = oracle.conv_silu_fwd(x[:, 6:], w, bias, prev=x[:, 3:6])
+    np.testing.assert_allclose(tail, out[:, 6:], rtol=1e-14, atol=1e-16)
+    # channels are independent: permuting them permutes the output
+    perm = np.array([3, 0, 4, 1, 2])
+    np.testing.assert_array_equal(oracle.conv_silu_fwd(x[..., perm], w[perm], bias[perm]), out[..., perm])
+
+
+def test_conv_silu_bwd_matches_autograd(oracle):
+    rng = np.random.default_rng(62)
+    B, T, C = 2, 9, 4
+    x, w, bias = rng.standard_normal((B, T, C)), rng.standard_normal((C, 4)), rng.standard_normal(C)
+    prev, dout = rng.standard_normal((B, 3, C)), rng.standard_normal((B, T, C))
+    got = oracle.conv_silu_bwd(x, w, dout, bias, prev)
+    tx, tw, tb, tp = (torch.tensor(a, requires_grad=True) for a in (x, w, bias, prev))
+    full = torch.cat([tp, tx], dim=1).transpose(1, 2)
+    y = torch.nn.functional.silu(torch.nn.functional.conv1d(full, tw[:, None, :], tb, groups=C)).transpose(1, 2)
+    y.backward(torch.from_numpy(dout))
+    for name, t in (("dx", tx), ("dw", tw), ("dbias", tb), ("dprev", tp)):
+        np.testing.assert_allclose(got[name], t.grad.numpy(), rtol=1e-12, atol=1e-14, err_msg=name)
+
+
+def test_conv_silu_bwd_matches_finite_differences(oracle):
+    rng = np.random.default_rng(63)
+    B, T, C = 1, 6, 2
+    x, w, bias = rng.standard_normal((B, T, C)), rng.standard_normal((C, 4)), rng.standard_normal(C)
+    prev, dout = rng.standard_normal((B, 3, C)), rng.standard_normal((B, T, C))
+    got = oracle.conv_silu_bwd(x, w, dout, bias, prev)
+    loss = lambda **kw: float((oracle.conv_silu_fwd(kw.get("x", x), kw.get("w", w), kw.get("bias", bias), kw.get("prev", prev)) * dout).sum())
+    eps = 1e-6
+    for name, arr, key in (("dx", x, "x"), ("dw", w, "w"), ("dbias", bias, "bias"), ("dprev", prev, "prev")):
+        num = np.zeros_like(arr)
+        for idx in np.ndindex(arr.shape):
+            p, m = arr.copy(), arr.copy()
+            p[idx] += eps
+            m[idx] -= eps
+            num[idx] = (loss(**{key: p}) - loss(**{key: m})) / (2 * eps)
+        np.testing.assert_allclose(got[name], num, rtol=1e-6, atol=1e-8, err_msg=name)
