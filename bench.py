@@ -494,6 +494,128 @@ def main_out_norm(args):
         dist.destroy_process_group()
 
 
+def main_in_conv(args):
+    """`--workload in_conv`: the input path before the scan (SiLU of a depthwise causal conv1d of width
+    4), forward + backward, on the fused q/k/v projection of the fwd_bf16 workload (B=8, T=2048,
+    C = Nq K + Nk K + N V = 3072, bf16).  HBM-bound: 4C bytes per token forward (x in, out), 6C backward
+    (x, dout in, dx out)."""
+    from paper_2603_14360_b200 import binding
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_
+        dist_.init_process_group("nccl", device_id=dev)
+        dist = dist_
+    base = CONFIGS["fwd_bf16"]
+    B, T = base.B, base.T
+    C = (base.nq + base.nk) * base.K + base.N * base.V
+    tokens = B * T
+    steps = args.steps or 200
+    warmup = max(args.warmup or 10, 3)
+    R = 4                                              # 4 x 200 MB of inputs cycled: above L2
+    host = [{k: v.pin_memory() for k, v in inputs.make_conv_inputs(B, T, C, "bf16", seed=rank_input_seed(11, rank, r), prev=False).items()
+             if v is not None} for r in range(R)]
+    sets = [{k: v.to(dev) for k, v in h.items()} for h in host]
+    outs = [dict(out=torch.empty_like(sets[0]["x"]), dx=torch.empty_like(sets[0]["x"]),
+                 dw=torch.empty((C, 4), dtype=torch.float32, device=dev), dbias=torch.empty((C,), dtype=torch.float32, device=dev))
+            for _ in range(2)]
+    ws = torch.empty(max(1, binding._lib().m2rnn_conv_silu_bwd_workspace_bytes(B, T, C)), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(i, s=None, ob=0):
+        s = s or sets[i % R]
+        o = outs[ob]
+        binding.m2rnn_conv_silu_fwd(s["x"], s["w"], s["bias"], out=o["out"], stream=stream)
+        binding.m2rnn_conv_silu_bwd(s["x"], s["w"], s["dout"], s["bias"], out=o, workspace=ws, stream=stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for i in range(warmup):
+        step(i)
+    barrier()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    with ClockSampler(local) as clocks:
+        barrier()
+        ev[0].record(stream)
+        for i in range(steps):
+            step(i)
+        ev[1].record(stream)
+        barrier()
+    ms_total = ev[0].elapsed_time(ev[1])
+    ms_e2e, e2e_steps, h2d, d2h = 0.0, 0, 0, 0
+    if not args.no_e2e:
+        stages = [{k: torch.empty_like(v) for k, v in sets[0].items()} for _ in range(2)]
+        hout = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in outs[0].items()}
+        h2d = sum(nbytes(t) for t in stages[0].values())
+        d2h = sum(nbytes(t) for t in hout.values())
+        e2e_steps = 20
+
+        def copy_in(i, b):
+            for k, t in stages[b].items():
+                t.copy_(host[i % R][k], non_blocking=True)
+
+        def copy_out(b):
+            for k, t in hout.items():
+                t.copy_(outs[b][k], non_blocking=True)
+
+        e2e_pipeline(stream, dev, 3, copy_in, lambda i, b: step(i, s=stages[b], ob=b), copy_out)
+        barrier()
+        ev2 = e2e_pipeline(stream, dev, e2e_steps, copy_in, lambda i, b: step(i, s=stages[b], ob=b), copy_out)
+        barrier()
+        ms_e2e = ev2[0].elapsed_time(ev2[1])
+    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], dist, dev)
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+    ms_step = ms_total / steps
+    peaks = measured_peaks()
+    alg_bytes = tokens * C * 2 * (2 + 3)               # x, out | x, dout, dx (bf16)
+    achieved = alg_bytes / (ms_step * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": whole_job_tokens_per_s(tokens, world, ms_step), "unit": "tokens/s", "n_gpus": world,
+        "steps": steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "in_conv", "pass": "fwd+bwd of SiLU(conv1d) on the fused q/k/v projection", "B": B, "T": T, "C": C,
+                   "per_gpu_batch": B, "l2": f"{R} input sets cycled; bytes touched per step {int(alg_bytes / 1e6)} MB vs 126 MB L2"},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"], "traffic": None, "call": "m2rnn_conv_silu_fwd + m2rnn_conv_silu_bwd",
+                     "peak_source": f"{peaks['source']} HBM copy", "algorithmic_bytes_per_step": alg_bytes},
+        "gpu_launches": steps * 3,
+        "clocks": clocks.summary(),
+    }
+    if not args.no_e2e:
+        line["e2e"] = {"value": tokens * world / (ms_e2e / e2e_steps * 1e-3), "unit": "tokens/s",
+                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+    if not args.no_cpu_baseline:
+        import oracle
+        f = inputs.to_f64
+        n_t = 64                                        # a bounded sample: the first steps of every batch entry
+        hs = {k: (v[:, :n_t] if v.dim() == 3 else v) for k, v in host[0].items()}
+        t0 = time.perf_counter()
+        reps = 0
+        while time.perf_counter() - t0 < 10.0:
+            oracle.conv_silu_fwd(f(hs["x"]), f(hs["w"]), f(hs["bias"]))
+            oracle.conv_silu_bwd(f(hs["x"]), f(hs["w"]), f(hs["dout"]), f(hs["bias"]))
+            reps += 1
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": reps * B * n_t / dt, "unit": "tokens/s", "cores": 1, "kind": "oracle",
+                                "sample": f"{reps} x the first {n_t} steps of the {B} batch entries, forward + backward", "seconds": dt}
+    print(json.dumps(line), flush=True)
+    if dist:
+        dist.destroy_process_group()
+
+
 def pick_config(args, workload):
     cfg = CONFIGS["paper_layer" if workload == "paper_layer_bptt" else workload]
     if workload == "paper_layer_bptt":
@@ -510,7 +632,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=0, help="0: a default per workload")
     ap.add_argument("--warmup", type=int, default=0)
-    ap.add_argument("--workload", default=None, choices=sorted(CONFIGS) + ["paper_layer_bptt", "out_norm"],
+    ap.add_argument("--workload", default=None, choices=sorted(CONFIGS) + ["paper_layer_bptt", "out_norm", "in_conv"],
                     help="default: fwd_bf16 as the line's value, with bptt_bf16 (forward + backward) as the sub-object 'bptt'")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -523,11 +645,11 @@ def main():
     args = ap.parse_args()
     both_halves = args.workload is None and not args.no_bptt and not args.seq_len
     workload = args.workload or "fwd_bf16"
-    if workload == "out_norm" and args.impl == "ours":
-        main_out_norm(args)
+    if workload in ("out_norm", "in_conv") and args.impl == "ours":
+        (main_out_norm if workload == "out_norm" else main_in_conv)(args)
         return
-    if workload == "out_norm":
-        raise SystemExit("--impl reference times the scan workloads; the out_norm line carries its own cpu_baseline")
+    if workload in ("out_norm", "in_conv"):
+        raise SystemExit("--impl reference times the scan workloads; the out_norm and in_conv lines carry their own cpu_baseline")
     cfg, pas = pick_config(args, workload)
 
     if args.impl == "reference":

@@ -232,6 +232,39 @@ int m2rnn_gated_norm_bwd(int64_t tokens, int32_t d, int32_t io_dtype, const void
                          const void *w, const float *rstd, int32_t silu, const void *dout, void *dy,
                          void *dg_in, float *dw, void *workspace, size_t workspace_bytes, void *stream);
 
+/* ---- Input path before the scan ("M2RNN block" equations: q_t, k_t, v_t = SiLU(conv1d(projection)):
+ * a depthwise causal convolution of width 4 along time, one filter per channel, then SiLU).
+ *     pre[b][t][c] = bias[c] + sum_{s=0..3} w[c][s] x[b][t-3+s][c],     out = pre / (1 + exp(-pre))
+ * (w[c][3] weighs the current token, w[c][0] the one three steps back; the paper gives the
+ * convolution no bias of its own: bias = NULL.)
+ *   in : x [B,T,C] with `x_stride` elements between tokens (0 = C); w [C,4]; bias [C] or NULL;
+ *        prev [B,3,C] or NULL: the inputs at t = -3, -2, -1 (the last three of the segment before;
+ *        NULL = zeros), io_dtype all
+ *   out: out [B,T,C] with `out_stride` elements between tokens (0 = C); may be x itself only if
+ *        nothing else reads x afterwards AND the call is the only one on those rows (in place is
+ *        not supported: a tile reads three rows that its neighbour writes).
+ * The strides let the three projections be handled as ONE tensor: x = the fused projection output
+ * [B,T,Nq K + Nk K + N V], out of the same shape, whose column slices are then the q, k, v of
+ * m2rnn_fwd (see m2rnn_params.q_stride).  C is a multiple of 16 bytes of channels.  B = 0 or T = 0
+ * is a valid empty call.  Device pointers, 16-byte aligned, asynchronous on `stream`. */
+int m2rnn_conv_silu_fwd(int32_t B, int32_t T, int32_t C, int32_t io_dtype, const void *x, int64_t x_stride,
+                        const void *w, const void *bias, const void *prev, void *out, int64_t out_stride,
+                        void *stream);
+
+/* Bytes of workspace m2rnn_conv_silu_bwd needs (per-tile partial sums of dw and dbias). */
+size_t m2rnn_conv_silu_bwd_workspace_bytes(int32_t B, int32_t T, int32_t C);
+
+/* Backward of m2rnn_conv_silu_fwd: with dpre = dout (.) SiLU'(pre) (pre recomputed from x),
+ *     dx[t] = sum_s w[c][s] dpre[t+3-s],   dw[c][s] = sum_{b,t} dpre[t] x[t-3+s],   dbias[c] = sum_{b,t} dpre[t].
+ *   in : x, w, bias, prev as in the forward call; dout [B,T,C] (token stride dout_stride)
+ *   out: dx [B,T,C] (token stride dx_stride); dw [C,4] fp32; dbias [C] fp32 or NULL; dprev [B,3,C]
+ *        io_dtype or NULL; all overwritten; sums in a fixed order (bitwise repeatable)
+ *   workspace: 256-byte aligned device memory of at least the queried size. */
+int m2rnn_conv_silu_bwd(int32_t B, int32_t T, int32_t C, int32_t io_dtype, const void *x, int64_t x_stride,
+                        const void *w, const void *bias, const void *prev, const void *dout,
+                        int64_t dout_stride, void *dx, int64_t dx_stride, float *dw, float *dbias,
+                        void *dprev, void *workspace, size_t workspace_bytes, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -63,6 +63,10 @@ EXPORTS = {
     "m2rnn_bwd": (ctypes.c_int, [_pp] + [_vp] * 19 + [ctypes.c_size_t, _vp, _vp]),
     "m2rnn_bwd_static_scratch": (ctypes.c_int, [_pp] + [_vp] * 20),
     "m2rnn_decode_step": (ctypes.c_int, [_pp] + [_vp] * 12),
+    "m2rnn_conv_silu_fwd": (ctypes.c_int, [ctypes.c_int32] * 4 + [_vp, ctypes.c_int64, _vp, _vp, _vp, _vp, ctypes.c_int64, _vp]),
+    "m2rnn_conv_silu_bwd_workspace_bytes": (ctypes.c_size_t, [ctypes.c_int32] * 3),
+    "m2rnn_conv_silu_bwd": (ctypes.c_int, [ctypes.c_int32] * 4 + [_vp, ctypes.c_int64, _vp, _vp, _vp, _vp, ctypes.c_int64, _vp,
+                                             ctypes.c_int64, _vp, _vp, _vp, _vp, ctypes.c_size_t, _vp]),
     "m2rnn_wait_selftest": (ctypes.c_int, [ctypes.c_int64, _vp, _vp, _vp]),
     "m2rnn_gated_norm_fwd": (ctypes.c_int, [ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, _vp, _vp, _vp, ctypes.c_float,
                                             ctypes.c_int32, _vp, _vp, _vp]),
@@ -156,6 +160,8 @@ def _token_stride(t, name) -> int:
     """Elements between consecutive tokens of q, k or v ([B,T,heads,dim] or packed [tokens,heads,dim]).
     A token's heads must be contiguous and the token axis regular, so that the tensor may be a view
     into a fused projection output; 0 stands for the dense layout."""
+    if t.numel() == 0:
+        return 0
     if t.stride(-1) != 1 or t.stride(-2) != t.shape[-1]:
         raise ValueError(f"{name}: the heads of a token must be contiguous")
     tok = t.stride(-3)
@@ -394,3 +400,52 @@ def m2rnn_gated_norm_bwd(y, g_in, w, rstd, dout, *, silu=True, workspace=None, o
     if rc != 0:
         raise M2RNNError(rc, "m2rnn_gated_norm_bwd")
     return dict(dy=dy, dg=dg, dw=dw)
+
+
+def _rows(t, name):
+    """[B,T,C] with contiguous channels and a regular token axis -> token stride in elements."""
+    if t.dim() == 3 and t.numel() == 0:
+        return t.shape[2]
+    if t.dim() != 3 or t.stride(2) != 1 or (t.shape[0] > 1 and t.stride(0) != t.shape[1] * t.stride(1)):
+        raise ValueError(f"{name}: expected [B,T,C] with contiguous channels and batch entries one after the other")
+    return t.stride(1)
+
+
+def m2rnn_conv_silu_fwd(x, w, bias=None, prev=None, *, out=None, stream=None):
+    """SiLU(depthwise causal conv1d of width 4 along time) of x [B,T,C] (a view into a wider tensor is
+    fine); w [C,4], bias [C], prev [B,3,C] (the three inputs before t = 0).  Returns out [B,T,C]."""
+    B, T, C = x.shape
+    io = x.dtype
+    _chk(w, "w", (C, 4), io); _chk(bias, "bias", (C,), io); _chk(prev, "prev", (B, 3, C), io)
+    if out is None:
+        out = torch.empty((B, T, C), dtype=io, device=x.device)
+    _chk(out, "out", (B, T, C), io, True)
+    rc = _lib().m2rnn_conv_silu_fwd(B, T, C, _io_code(io), _ptr(x), _rows(x, "x"), _ptr(w), _ptr(bias), _ptr(prev),
+                                    _ptr(out), _rows(out, "out"), _stream(stream))
+    if rc != 0:
+        raise M2RNNError(rc, "m2rnn_conv_silu_fwd")
+    return out
+
+
+def m2rnn_conv_silu_bwd(x, w, dout, bias=None, prev=None, *, out=None, workspace=None, stream=None):
+    """Backward of ``m2rnn_conv_silu_fwd`` -> dict(dx [B,T,C], dw [C,4] fp32, dbias [C] fp32, dprev [B,3,C])."""
+    B, T, C = x.shape
+    io, dev = x.dtype, x.device
+    _chk(w, "w", (C, 4), io); _chk(bias, "bias", (C,), io); _chk(prev, "prev", (B, 3, C), io)
+    _chk(dout, "dout", (B, T, C), io, True)
+    out = dict(out or {})
+    if out.get("dx") is None: out["dx"] = torch.empty((B, T, C), dtype=io, device=dev)
+    if out.get("dw") is None: out["dw"] = torch.empty((C, 4), dtype=torch.float32, device=dev)
+    if out.get("dbias") is None: out["dbias"] = torch.empty((C,), dtype=torch.float32, device=dev)
+    if out.get("dprev") is None and prev is not None: out["dprev"] = torch.empty((B, 3, C), dtype=io, device=dev)
+    _chk(out["dx"], "dx", (B, T, C), io, True); _chk(out["dw"], "dw", (C, 4), torch.float32)
+    need = _lib().m2rnn_conv_silu_bwd_workspace_bytes(B, T, C)
+    if workspace is None:
+        workspace = torch.empty(max(need, 1), dtype=torch.uint8, device=dev)
+    rc = _lib().m2rnn_conv_silu_bwd(B, T, C, _io_code(io), _ptr(x), _rows(x, "x"), _ptr(w), _ptr(bias), _ptr(prev), _ptr(dout),
+                                    _rows(dout, "dout"), _ptr(out["dx"]), _rows(out["dx"], "dx"), _ptr(out["dw"]),
+                                    _ptr(out.get("dbias")), _ptr(out.get("dprev")), _ptr(workspace), workspace.numel(),
+                                    _stream(stream))
+    if rc != 0:
+        raise M2RNNError(rc, "m2rnn_conv_silu_bwd")
+    return out

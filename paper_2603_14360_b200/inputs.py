@@ -149,3 +149,15 @@ def make_gated_norm_inputs(B: int, T: int, N: int, V: int, dtype: str = "bf16", 
 def to_f64(t):
     """Exact widening of a (possibly bf16) tensor to a numpy float64 array; None stays None."""
     return None if t is None else t.detach().to("cpu", torch.float64).numpy()
+
+
+def make_conv_inputs(B: int, T: int, C: int, dtype: str, seed: int = 0, prev: bool = True) -> dict:
+    """Inputs of the path before the scan (SiLU of a depthwise causal conv1d over the projections):
+    x, dout ~ N(0,1), filter taps w ~ N(0, 1/4) (so that the pre-activation has unit scale), bias ~
+    N(0, 0.1^2), the three carried rows ~ N(0,1); rounded to the I/O dtype."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    io = torch_dtype(dtype)
+    out = dict(x=_normal(rng, (B, T, C)).to(io), w=_normal(rng, (C, 4), 0.5).to(io), bias=_normal(rng, (C,), 0.1).to(io),
+               dout=_normal(rng, (B, T, C)).to(io))
+    out["prev"] = _normal(rng, (B, 3, C)).to(io) if prev else None
+    return out
