@@ -60,9 +60,10 @@ bool fwd_use_tc(int B, int N, int K, int V, int io_dtype) {
   // Measured (B200): the round trip of a tcgen05 step (operand store, proxy fence, barrier, eight
   // MMAs at ~30 cycles of issue each, commit, mbarrier, tcgen05.ld) is ~400 cycles before any
   // arithmetic, against ~30 for mma.sync on registers.  It pays only where the register kernels
-  // are bound by the legacy tensor path and there are rows to amortise it over: V = 128 with at
-  // least one 64-row CTA per SM (the K = V = 128 point of the state-size sweep: 6.8 against 7.8 ms).
-  return V == 128 && K % 64 == 0 && (long)(B > 0 ? B : 1) * N * (K / 64) >= sm_count();
+  // are bound by the legacy tensor path and there are rows to amortise it over: V = 128 with 64-row
+  // CTAs on at least three quarters of the SMs (the K = V = 128 point of the state-size sweep: 6.8
+  // against 7.8 ms).
+  return V == 128 && K % 64 == 0 && 4L * (B > 0 ? B : 1) * N * (K / 64) >= 3L * sm_count();
 }
 
 int plan_fwd_rows(int B, int N, int K, int V, int io_dtype) {

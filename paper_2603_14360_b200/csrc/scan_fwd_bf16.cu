@@ -67,7 +67,7 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
   const int NW = NWT ? NWT : (K >> 4);
   constexpr bool kPacked = V <= 64;                  // packed fp32x2 arithmetic (spills at V = 128)
   constexpr int TC = FwdSmem<V>::tc(MAXW * 16);   // K > 64 <=> MAXW == 8
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x, warp = __shfl_sync(0xffffffffu, tid >> 5, 0), lane = tid & 31;   // (through a shuffle: known to be warp-uniform)
   const int bn = blockIdx.x / RS, rs = blockIdx.x % RS, b = bn / N, n = bn % N;
   const UnitSpan span = unit_span(a, b);   // this batch entry's tokens (a slice of a packed batch, or b T ..)
   const int T = span.T;

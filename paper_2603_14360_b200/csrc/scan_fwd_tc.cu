@@ -422,7 +422,7 @@ int fwd_tc_rows_per_cta(int B, int N, int K, int V) {
   } else {
     const int HS = 128 / V;
     const long tiles = (long)(B > 0 ? B : 1) * ((N + HS - 1) / HS);
-    r = (K % 64 == 0 && tiles * (K / 64) >= sm_count()) ? 64 : 32;
+    r = (K % 64 == 0 && 4 * tiles * (K / 64) >= 3L * sm_count()) ? 64 : 32;
   }
   if (r == 64 && K % 32) r = 32;
   return r;
