@@ -56,6 +56,21 @@ template <> __device__ __forceinline__ float sigmoid_of<float>(float x) {
 }
 template <> __device__ __forceinline__ float sigmoid_of<__nv_bfloat16>(float x) { return fmaf(0.5f, tanh_approx(0.5f * x), 0.5f); }
 
+// both halves of a pair (the arithmetic below is in packed fp32 pairs: one instruction per two channels)
+template <typename T> __device__ __forceinline__ float2 sigmoid2(float2 x) {
+  if constexpr (sizeof(T) == 2) {
+    const float2 h = __fmul2_rn(x, make_float2(0.5f, 0.5f));
+    return __ffma2_rn(make_float2(tanh_approx(h.x), tanh_approx(h.y)), make_float2(0.5f, 0.5f), make_float2(0.5f, 0.5f));
+  } else {
+    return make_float2(sigmoid_of<T>(x.x), sigmoid_of<T>(x.y));
+  }
+}
+template <int CH>
+__device__ __forceinline__ void to_pairs(const float (&v)[CH], float2 (&p)[CH / 2]) {
+#pragma unroll
+  for (int e = 0; e < CH / 2; ++e) p[e] = make_float2(v[2 * e], v[2 * e + 1]);
+}
+
 // row t of batch entry b: x for t >= 0, the carried rows `prev` [B,3,C] for t = -3..-1 (zeros without)
 template <typename T, int CH>
 __device__ __forceinline__ void load_row(const T *x, long long xs, const T *prev, int b, int Tn, int C, int t, int c0, float (&v)[CH]) {
@@ -66,7 +81,7 @@ __device__ __forceinline__ void load_row(const T *x, long long xs, const T *prev
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kConvThreads, 8) conv_silu_fwd_kernel(int B, int Tn, int C, const T *__restrict__ x, long long xs,
+__global__ void __launch_bounds__(kConvThreads, 6) conv_silu_fwd_kernel(int B, int Tn, int C, const T *__restrict__ x, long long xs,
                                                                      const T *__restrict__ w, const T *__restrict__ bias,
                                                                      const T *__restrict__ prev, T *__restrict__ out, long long os) {
   constexpr int CH = Chunk<T>::CH;
@@ -75,17 +90,22 @@ __global__ void __launch_bounds__(kConvThreads, 8) conv_silu_fwd_kernel(int B, i
   const int c0 = cc * CH, ntile = (Tn + kTileFwd - 1) / kTileFwd;
   const int b = blockIdx.y / ntile, t0 = (blockIdx.y % ntile) * kTileFwd + sub * kStepsFwd, t1 = min(Tn, t0 + kStepsFwd);
   if (t0 >= Tn) return;
-  float wv[CH][4], bv[CH];
+  constexpr int CP = CH / 2;            // channel pairs
+  float2 w2[4][CP], b2[CP];             // w2[s][p] = tap s of channels 2p, 2p+1
 #pragma unroll
-  for (int e = 0; e < CH; ++e) {
+  for (int e = 0; e < CP; ++e) {
 #pragma unroll
-    for (int s = 0; s < 4; ++s) wv[e][s] = to_f32<T>(w[(size_t)(c0 + e) * 4 + s]);
-    bv[e] = bias ? to_f32<T>(bias[c0 + e]) : 0.f;
+    for (int s = 0; s < 4; ++s) w2[s][e] = make_float2(to_f32<T>(w[(size_t)(c0 + 2 * e) * 4 + s]), to_f32<T>(w[(size_t)(c0 + 2 * e + 1) * 4 + s]));
+    b2[e] = bias ? make_float2(to_f32<T>(bias[c0 + 2 * e]), to_f32<T>(bias[c0 + 2 * e + 1])) : make_float2(0.f, 0.f);
   }
-  float xm3[CH], xm2[CH], xm1[CH];
-  load_row<T, CH>(x, xs, prev, b, Tn, C, t0 - 3, c0, xm3);
-  load_row<T, CH>(x, xs, prev, b, Tn, C, t0 - 2, c0, xm2);
-  load_row<T, CH>(x, xs, prev, b, Tn, C, t0 - 1, c0, xm1);
+  float2 xm3[CP], xm2[CP], xm1[CP];
+  {
+    float r3[CH], r2[CH], r1[CH];
+    load_row<T, CH>(x, xs, prev, b, Tn, C, t0 - 3, c0, r3);
+    load_row<T, CH>(x, xs, prev, b, Tn, C, t0 - 2, c0, r2);
+    load_row<T, CH>(x, xs, prev, b, Tn, C, t0 - 1, c0, r1);
+    to_pairs<CH>(r3, xm3); to_pairs<CH>(r2, xm2); to_pairs<CH>(r1, xm1);
+  }
   // the loads of eight steps are issued before the first is used: with three dozen warps per SM that
   // keeps enough bytes in flight to cover the latency of HBM
   constexpr int U = 8;
@@ -99,12 +119,15 @@ __global__ void __launch_bounds__(kConvThreads, 8) conv_silu_fwd_kernel(int B, i
       raw[u] = tb + u < t1 ? *reinterpret_cast<const Raw *>(xp + u * xs) : Raw{};
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      float x0[CH], o[CH];
-      Chunk<T>::unpack(raw[u], x0);
+      float xr[CH], o[CH];
+      float2 x0[CP];
+      Chunk<T>::unpack(raw[u], xr);
+      to_pairs<CH>(xr, x0);
 #pragma unroll
-      for (int e = 0; e < CH; ++e) {
-        const float pre = fmaf(wv[e][3], x0[e], fmaf(wv[e][2], xm1[e], fmaf(wv[e][1], xm2[e], fmaf(wv[e][0], xm3[e], bv[e]))));
-        o[e] = pre * sigmoid_of<T>(pre);
+      for (int e = 0; e < CP; ++e) {
+        const float2 pre = __ffma2_rn(w2[3][e], x0[e], __ffma2_rn(w2[2][e], xm1[e], __ffma2_rn(w2[1][e], xm2[e], __ffma2_rn(w2[0][e], xm3[e], b2[e]))));
+        const float2 r = __fmul2_rn(pre, sigmoid2<T>(pre));
+        o[2 * e] = r.x; o[2 * e + 1] = r.y;
         xm3[e] = xm2[e]; xm2[e] = xm1[e]; xm1[e] = x0[e];
       }
       if (tb + u < t1) Chunk<T>::store(op + u * os, o);     // (past the end: arithmetic on stale registers, nothing stored)
@@ -114,7 +137,7 @@ __global__ void __launch_bounds__(kConvThreads, 8) conv_silu_fwd_kernel(int B, i
 
 // partial sums of a tile: part[tile][5][C] = dw taps 0..3 and dbias
 template <typename T>
-__global__ void __launch_bounds__(kConvThreads, 5) conv_silu_bwd_kernel(int B, int Tn, int C, const T *__restrict__ x, long long xs,
+__global__ void __launch_bounds__(kConvThreads, 4) conv_silu_bwd_kernel(int B, int Tn, int C, const T *__restrict__ x, long long xs,
                                                                      const T *__restrict__ w, const T *__restrict__ bias,
                                                                      const T *__restrict__ prev, const T *__restrict__ dout, long long ds,
                                                                      T *__restrict__ dx, long long dxs, T *__restrict__ dprev,
@@ -127,29 +150,32 @@ __global__ void __launch_bounds__(kConvThreads, 5) conv_silu_bwd_kernel(int B, i
   const int c0 = live ? cc * CH : 0, ntile = (Tn + kTileBwd - 1) / kTileBwd;
   const int b = blockIdx.y / ntile, t0 = (blockIdx.y % ntile) * kTileBwd + sub * kStepsBwd;
   const int t1 = max(t0, min(Tn, t0 + kStepsBwd));   // an empty run when the sequence ends before it
-  float wv[CH][4], bv[CH];
+  constexpr int CP = CH / 2;            // channel pairs
+  float2 w2[4][CP], b2[CP];
 #pragma unroll
-  for (int e = 0; e < CH; ++e) {
+  for (int e = 0; e < CP; ++e) {
 #pragma unroll
-    for (int s = 0; s < 4; ++s) wv[e][s] = to_f32<T>(w[(size_t)(c0 + e) * 4 + s]);
-    bv[e] = bias ? to_f32<T>(bias[c0 + e]) : 0.f;
+    for (int s = 0; s < 4; ++s) w2[s][e] = make_float2(to_f32<T>(w[(size_t)(c0 + 2 * e) * 4 + s]), to_f32<T>(w[(size_t)(c0 + 2 * e + 1) * 4 + s]));
+    b2[e] = bias ? make_float2(to_f32<T>(bias[c0 + 2 * e]), to_f32<T>(bias[c0 + 2 * e + 1])) : make_float2(0.f, 0.f);
   }
-  float dwv[CH][4], dbv[CH];
+  float2 dw2[4][CP], db2[CP];
 #pragma unroll
-  for (int e = 0; e < CH; ++e) { dwv[e][0] = dwv[e][1] = dwv[e][2] = dwv[e][3] = 0.f; dbv[e] = 0.f; }
-  // The first tile of a batch entry also emits the gradient of the carried rows (t' = -3..-1): its
+  for (int e = 0; e < CP; ++e) { dw2[0][e] = dw2[1][e] = dw2[2][e] = dw2[3][e] = db2[e] = make_float2(0.f, 0.f); }
+  // The run that starts a sequence also emits the gradient of the carried rows (t' = -3..-1): its
   // sweep starts three steps early with dpre = 0 there.
-  const int ts = t0 == 0 ? -3 : t0;         // first t' whose dx this thread emits (the run that starts the sequence: also the carried rows)
-  float xm3[CH], xm2[CH], xm1[CH];
+  const int ts = t0 == 0 ? -3 : t0;         // first t' whose dx this thread emits
+  float2 xm3[CP], xm2[CP], xm1[CP];
   const bool work = live && t1 > t0;        // (an empty run loads nothing: its halo rows may lie past the end)
   if (work) {
-    load_row<T, CH>(x, xs, prev, b, Tn, C, t0 - 3, c0, xm3);
-    load_row<T, CH>(x, xs, prev, b, Tn, C, t0 - 2, c0, xm2);
-    load_row<T, CH>(x, xs, prev, b, Tn, C, t0 - 1, c0, xm1);
+    float r3[CH], r2[CH], r1[CH];
+    load_row<T, CH>(x, xs, prev, b, Tn, C, t0 - 3, c0, r3);
+    load_row<T, CH>(x, xs, prev, b, Tn, C, t0 - 2, c0, r2);
+    load_row<T, CH>(x, xs, prev, b, Tn, C, t0 - 1, c0, r1);
+    to_pairs<CH>(r3, xm3); to_pairs<CH>(r2, xm2); to_pairs<CH>(r1, xm1);
   }
-  float d3[CH], d2[CH], d1[CH];             // dpre at t-3, t-2, t-1
+  float2 d3[CP], d2[CP], d1[CP];            // dpre at t-3, t-2, t-1
 #pragma unroll
-  for (int e = 0; e < CH; ++e) d3[e] = d2[e] = d1[e] = 0.f;
+  for (int e = 0; e < CP; ++e) d3[e] = d2[e] = d1[e] = make_float2(0.f, 0.f);
   // t runs three steps past the run: dx[t'] needs dpre[t' .. t'+3].  The loads of four steps are
   // issued before the first is used.
   constexpr int U = 4;
@@ -157,6 +183,7 @@ __global__ void __launch_bounds__(kConvThreads, 5) conv_silu_bwd_kernel(int B, i
   const T *xp = x + ((size_t)b * Tn + t0) * xs + c0, *gp = dout + ((size_t)b * Tn + t0) * ds + c0;
   T *dxp = dx + ((size_t)b * Tn + t0 - 3) * dxs + c0;       // three steps behind
   const int tend = min(Tn, t1 + 3);                          // steps with inputs to read
+  const float2 one = make_float2(1.f, 1.f), mone = make_float2(-1.f, -1.f);
   for (int tb = t0; tb < t1 + 3 && work; tb += U, xp += U * xs, gp += U * ds, dxp += U * dxs) {
     Raw rx[U], rg[U];
 #pragma unroll
@@ -167,38 +194,52 @@ __global__ void __launch_bounds__(kConvThreads, 5) conv_silu_bwd_kernel(int B, i
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int t = tb + u;
-      float d0[CH];
+      float2 d0[CP];
       if (t < tend) {
-        float x0[CH], g[CH];
-        Chunk<T>::unpack(rx[u], x0);
-        Chunk<T>::unpack(rg[u], g);
+        float xr[CH], gr[CH];
+        float2 x0[CP], g[CP];
+        Chunk<T>::unpack(rx[u], xr);
+        Chunk<T>::unpack(rg[u], gr);
+        to_pairs<CH>(xr, x0); to_pairs<CH>(gr, g);
 #pragma unroll
-        for (int e = 0; e < CH; ++e) {
-          const float pre = fmaf(wv[e][3], x0[e], fmaf(wv[e][2], xm1[e], fmaf(wv[e][1], xm2[e], fmaf(wv[e][0], xm3[e], bv[e]))));
-          const float sg = sigmoid_of<T>(pre);
-          d0[e] = g[e] * sg * fmaf(pre, 1.f - sg, 1.f);      // dout * SiLU'(pre)
+        for (int e = 0; e < CP; ++e) {
+          const float2 pre = __ffma2_rn(w2[3][e], x0[e], __ffma2_rn(w2[2][e], xm1[e], __ffma2_rn(w2[1][e], xm2[e], __ffma2_rn(w2[0][e], xm3[e], b2[e]))));
+          const float2 sg = sigmoid2<T>(pre);
+          // dout * SiLU'(pre),  SiLU'(x) = sg (1 + x (1 - sg))
+          d0[e] = __fmul2_rn(__fmul2_rn(g[e], sg), __ffma2_rn(pre, __ffma2_rn(sg, mone, one), one));
           if (t < t1) {                                      // sums over this run's own steps only
-            dwv[e][0] = fmaf(d0[e], xm3[e], dwv[e][0]); dwv[e][1] = fmaf(d0[e], xm2[e], dwv[e][1]);
-            dwv[e][2] = fmaf(d0[e], xm1[e], dwv[e][2]); dwv[e][3] = fmaf(d0[e], x0[e], dwv[e][3]);
-            dbv[e] += d0[e];
+            dw2[0][e] = __ffma2_rn(d0[e], xm3[e], dw2[0][e]); dw2[1][e] = __ffma2_rn(d0[e], xm2[e], dw2[1][e]);
+            dw2[2][e] = __ffma2_rn(d0[e], xm1[e], dw2[2][e]); dw2[3][e] = __ffma2_rn(d0[e], x0[e], dw2[3][e]);
+            db2[e] = __fadd2_rn(db2[e], d0[e]);
           }
           xm3[e] = xm2[e]; xm2[e] = xm1[e]; xm1[e] = x0[e];
         }
       } else {
 #pragma unroll
-        for (int e = 0; e < CH; ++e) d0[e] = 0.f;
+        for (int e = 0; e < CP; ++e) d0[e] = make_float2(0.f, 0.f);
       }
       const int tp = t - 3;                                  // dx[tp] = w3 dpre[tp] + w2 dpre[tp+1] + w1 dpre[tp+2] + w0 dpre[tp+3]
       if (tp >= ts && tp < t1) {
         float o[CH];
 #pragma unroll
-        for (int e = 0; e < CH; ++e) o[e] = fmaf(wv[e][3], d3[e], fmaf(wv[e][2], d2[e], fmaf(wv[e][1], d1[e], wv[e][0] * d0[e])));
+        for (int e = 0; e < CP; ++e) {
+          const float2 r = __ffma2_rn(w2[3][e], d3[e], __ffma2_rn(w2[2][e], d2[e], __ffma2_rn(w2[1][e], d1[e], __fmul2_rn(w2[0][e], d0[e]))));
+          o[2 * e] = r.x; o[2 * e + 1] = r.y;
+        }
         if (tp >= 0) Chunk<T>::store(dxp + u * dxs, o);
         else if (dprev) Chunk<T>::store(dprev + ((size_t)b * 3 + (3 + tp)) * C + c0, o);
       }
 #pragma unroll
-      for (int e = 0; e < CH; ++e) { d3[e] = d2[e]; d2[e] = d1[e]; d1[e] = d0[e]; }
+      for (int e = 0; e < CP; ++e) { d3[e] = d2[e]; d2[e] = d1[e]; d1[e] = d0[e]; }
     }
+  }
+  // the sums, channel by channel, for the hand-over below
+  float dwv[CH][4], dbv[CH];
+#pragma unroll
+  for (int e = 0; e < CP; ++e) {
+#pragma unroll
+    for (int s = 0; s < 4; ++s) { dwv[2 * e][s] = dw2[s][e].x; dwv[2 * e + 1][s] = dw2[s][e].y; }
+    dbv[2 * e] = db2[e].x; dbv[2 * e + 1] = db2[e].y;
   }
   // (dprev of the first tile: the three steps before t = 0 were emitted while t = 0, 1, 2 -- with
   // d3/d2/d1 still zero where they stand for dpre at negative times)
