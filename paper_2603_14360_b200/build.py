@@ -15,7 +15,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libm2rnn.so")
 
-SOURCES = ["api.cu", "reduce.cu", "scan_f32.cu", "scan_fwd_bf16.cu", "scan_fwd_bf16_cs.cu", "scan_fwd_tc.cu", "scan_bwd_bf16.cu", "decode_bf16.cu", "decode_tc_bf16.cu",
+SOURCES = ["api.cu", "reduce.cu", "scan_f32.cu", "scan_fwd_bf16.cu", "scan_fwd_bf16_cs.cu", "scan_fwd_tc.cu", "scan_bwd_bf16.cu", "scan_bwd_tc.cu", "decode_bf16.cu", "decode_tc_bf16.cu",
            "bwd_static_scratch.cu", "gated_norm.cu", "conv_silu.cu", "selftest.cu"]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -22,10 +22,22 @@ int sm_count() {
   return sms;
 }
 
+bool bwd_use_tc(int B, int N, int K, int V, int io_dtype) {
+  if (io_dtype != M2RNN_BF16 || V != 128) return false;
+  const char *variant = getenv("M2RNN_BWD_VARIANT");
+  if (variant && !strcmp(variant, "mma")) return false;
+  (void)B; (void)N; (void)K;
+  return true;
+}
+
 BwdPlan plan_bwd(int B, int N, int K, int V, int io_dtype) {
   BwdPlan pl{};
   if (io_dtype == M2RNN_F32) {  // recomputed states live in global scratch
     pl.KC = K; pl.C = 16; pl.C_max = 64;
+    return pl;
+  }
+  if (bwd_use_tc(B, N, K, V, io_dtype)) {   // 16-row CTAs, chunks of four steps
+    pl.KC = bwd_tc_rows_per_cta(); pl.C = pl.C_max = bwd_tc_chunk();
     return pl;
   }
   // Rows per CTA: the largest slab that still spreads the problem over the SMs (rows are independent
@@ -314,7 +326,8 @@ int m2rnn_bwd(const m2rnn_params *params, const void *q, const void *k, const vo
   const int RS = params->K / a.KC;
   a.dv_part = RS > 1 ? reinterpret_cast<float *>(ws + w.dv_part) : nullptr;
   a.dgate_part = RS > 1 ? reinterpret_cast<float *>(ws + w.dgate_part) : nullptr;
-  e = f32 ? launch_bwd_f32(a, s) : launch_bwd_bf16(a, s);
+  e = f32 ? launch_bwd_f32(a, s)
+          : (bwd_use_tc(params->B, params->N, params->K, params->V, params->io_dtype) ? launch_bwd_bf16_tc(a, s) : launch_bwd_bf16(a, s));
   if (e != cudaSuccess) return cuda_failed();
   e = launch_reduce_dW(a.dW_part, dW, params->B * RS, params->N, params->V, s);
   if (e != cudaSuccess) return cuda_failed();

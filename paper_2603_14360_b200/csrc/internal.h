@@ -86,6 +86,12 @@ cudaError_t launch_fwd_bf16(const ScanArgs &a, cudaStream_t s);     // scan_fwd_
 bool fwd_cs_supported(const ScanArgs &a);                            // scan_fwd_bf16_cs.cu
 cudaError_t launch_fwd_bf16_cs(const ScanArgs &a, cudaStream_t s);  // scan_fwd_bf16_cs.cu: two or four warps per 16-row slab
 cudaError_t launch_bwd_bf16(const ScanArgs &a, cudaStream_t s);     // scan_bwd_bf16.cu
+// The tcgen05 backward kernel (scan_bwd_tc.cu) takes V = 128; M2RNN_BWD_VARIANT = tc | mma overrides
+// the choice (benchmarking only).
+bool bwd_use_tc(int B, int N, int K, int V, int io_dtype);
+int bwd_tc_rows_per_cta();
+int bwd_tc_chunk();
+cudaError_t launch_bwd_bf16_tc(const ScanArgs &a, cudaStream_t s);  // scan_bwd_tc.cu
 cudaError_t launch_decode_bf16(const ScanArgs &a, cudaStream_t s);  // decode_bf16.cu: picks a kernel
 bool decode_tc_supported(const ScanArgs &a);                         // decode_tc_bf16.cu
 cudaError_t launch_decode_tc_bf16(const ScanArgs &a, cudaStream_t s);  // decode_tc_bf16.cu: tcgen05 path

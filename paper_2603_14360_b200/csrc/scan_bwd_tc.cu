@@ -1,0 +1,527 @@
+// bf16 backward through time (Algorithm 2 with the carried state gradient) for V = 128 on the
+// 5th-generation tensor cores: every product of a step is a tcgen05.mma with its accumulator in
+// tensor memory.
+//
+// At V = 128 the register kernels are bound by the legacy mma.sync path (W and W^T fragments no
+// longer fit in registers, 130-150 MMAs and as many shared-memory loads per chain warp and step);
+// here W^T and W sit in tensor memory for the whole scan and the products are issued by one thread.
+// As in the tcgen05 forward kernel the products are computed transposed, M = 128 lanes = state
+// columns, N = 16 state rows of the CTA, K = 128:
+//     recompute   P^T  = W^T . H_{t-1}^T      (A = W^T in tensor memory, B = H_{t-1} slab, bf16, shared memory)
+//     reverse     (dX W^T)^T = W . dX^T        (A = W   in tensor memory, B = dX slab)
+//     dW += H_{t-1}^T dX                      (both slabs read MN-major from shared memory, one MMA per
+//                                              step, accumulator 128 x 128 in tensor memory until the end)
+// A thread owns one state column and 8 rows, so v_t[j], dy_t[j], f_t are per-thread scalars, k_t[i],
+// q_t[i] warp-uniform broadcasts, and dv_j = sum_i dX[i][j] k_i is a sum over a thread's registers.
+// Sums over columns (dq = H_t dy, dk = dX v) are small mma.sync products that helper warps take
+// from the same shared-memory slabs, off the chain.
+//
+// One CTA per (b, n, 16-row slab).  Time is walked in chunks of C steps, last chunk first:
+//   recompute warps (8)  redo a chunk's forward steps from its checkpoint; per step they leave the
+//                        H_{t-1} slab (bf16, the B operand) and, per thread, Z_t and H_{t-1} - Z_t (fp16);
+//   reverse warps   (8)  carry C = dL/dH in registers: G = C + q dy^T, df, dX = (1-f) G (1 - Z^2),
+//                        C <- f G + dX W^T; dv; the dX slab;
+//   helper warps    (4)  issue the dW product, compute dq and dk;
+//   loader, writer  (2)  stage q, k, v, dy and the gate of coming chunks / reduce and write dq, dk,
+//                        dv, dgate of finished ones.
+// The recompute warps work a chunk ahead of the reverse warps (two state buffers).  Hand-over is
+// by mbarriers; every wait is bounded and reports through dev_status; a common exit frees the
+// tensor memory.  Row-slab sums (dv, dgate, dW) are finished by the second-stage kernels.
+#include <cuda_fp16.h>
+
+#include "device_common.cuh"
+#include "internal.h"
+#include "mma_tile.cuh"
+#include "pipeline.cuh"
+#include "tc_common.cuh"
+#include "tile.cuh"
+
+namespace m2rnn {
+namespace {
+
+constexpr int kV = 128;
+constexpr int kNR = 16;              // state rows per CTA = N of the MMAs
+constexpr int kNT = 8;               // state rows per thread
+constexpr int kChainWarps = 8;       // per role: lane quarter (warp % 4) x row half (warp / 4)
+constexpr int kHelpWarps = 4;
+constexpr int kWarps = 2 * kChainWarps + kHelpWarps + 2;
+constexpr int kThreads = kWarps * 32;
+constexpr int kRingTc = 4;           // chunk slots of staged inputs / outputs in flight
+constexpr int kCTc = 4;              // steps per chunk = checkpoint interval of this kernel
+// tensor-memory columns: W^T, W (two bf16 per column), the two chain accumulators, dW
+constexpr uint32_t kColWT = 0, kColW = 64, kColP = 128, kColC = 144, kColDW = 256, kTmemColsBwd = 512;
+
+constexpr uint32_t kTileBytes = kNR * 256;                   // a 16 x 128 bf16 slab: 2 blocks of [16 rows][128 bytes]
+constexpr uint32_t kPrivBytes = 2 * kChainWarps * 32 * 16;   // per thread 8 x fp16 = 16 bytes, Z and H - Z apart
+constexpr uint32_t kStepBytes = kTileBytes + kPrivBytes;     // 12 288: keeps every tile on a 1024-byte boundary
+
+struct TcBwdSmem {
+  // byte offsets from the 1024-byte aligned base
+  static constexpr uint32_t oBar = 0, oState = 1024;
+  static constexpr uint32_t state_bytes = 2u * (kCTc + 1) * kStepBytes;       // [2][C + 1] step blocks
+  static constexpr uint32_t oDx = oState + state_bytes, oRing = oDx + 2 * kTileBytes;
+  // words of a ring slot.  In: q, k [C][16], v, dy [C][128] as fp32, f and its slope [C], dy and v
+  // once more as raw bf16 pairs (operands of the helper products).  Out: the helpers' shares of dq
+  // and dk [C][4][16], dv [C][128], one df partial per reverse thread [C][256].
+  static constexpr uint32_t oQ = 0, oK = oQ + kCTc * kNR, oVv = oK + kCTc * kNR, oDY = oVv + kCTc * kV, oF = oDY + kCTc * kV,
+                            oDF = oF + 4, oDYB = oDF + 4, oVB = oDYB + kCTc * kV / 2, oDQ = oVB + kCTc * kV / 2,
+                            oDK = oDQ + kCTc * kHelpWarps * kNR, oDV = oDK + kCTc * kHelpWarps * kNR, oDFP = oDV + kCTc * kV,
+                            slot_words = oDFP + kCTc * 256;
+  static constexpr uint32_t slot_bytes = slot_words * 4;
+  static constexpr uint32_t total = oRing + kRingTc * slot_bytes + 1024;      // + slack to align the base
+};
+static_assert(kCTc == 4, "the slot layout keeps f and its slope in four words each");
+
+// byte offset of element (row i, column l) of a slab: block l / 64, 16-byte chunk ((l % 64) / 8) ^ (i % 8)
+__device__ __forceinline__ uint32_t slab_off(int i, int l) {
+  return (uint32_t)(l >> 6) * (kNR * 128) + (uint32_t)i * 128u + ((((uint32_t)(l & 63) >> 3) ^ (uint32_t)(i & 7)) << 4) + (uint32_t)(l & 7) * 2u;
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ float2 unpack_f16x2(uint32_t x) { return __half22float2(*reinterpret_cast<const __half2 *>(&x)); }
+
+__global__ void __launch_bounds__(kThreads, 1) bwd_tc_kernel(ScanArgs a) {
+  using S = TcBwdSmem;
+  constexpr int V = kV;
+  const int C = a.C;                 // steps per chunk (<= kCTc, which sizes the buffers)
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t base_sa = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char *base = smem_dyn + (base_sa - smem_u32(smem_dyn));
+  uint64_t *bars = reinterpret_cast<uint64_t *>(base + S::oBar);
+  uint64_t *in_full = bars;                    // [kRingTc] a chunk's inputs are staged
+  uint64_t *out_full = in_full + kRingTc;      // [kRingTc] its dq, dk, dv, df shares are in the slot
+  uint64_t *slot_free = out_full + kRingTc;    // [kRingTc] ... and written out
+  uint64_t *st_ready = slot_free + kRingTc;    // [2] a chunk's recomputed steps are in the state buffer
+  uint64_t *st_free = st_ready + 2;            // [2] ... and read by everybody
+  uint64_t *dx_full = st_free + 2;             // [2] a step's dX slab is written
+  uint64_t *dx_free = dx_full + 2;             // [2] ... and read by the helpers and the dW product
+  uint64_t *rec_done = dx_free + 2;            // the recompute product has landed in tensor memory
+  uint64_t *rev_done = rec_done + 1;           // the reverse product has landed
+  uint64_t *dw_done = rev_done + 1;            // every dW product has landed
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(dw_done + 1);
+
+  const int K = a.K, N = a.N;
+  const int tid = threadIdx.x, warp = __shfl_sync(0xffffffffu, tid >> 5, 0), lane = tid & 31;
+  const int RS = K / kNR;
+  const int unit = blockIdx.x / RS, rs = blockIdx.x % RS, b = unit / N, n = unit % N;
+  const int rbase = rs * kNR;
+  const UnitSpan span = unit_span(a, b);
+  const int T = span.T;
+  const size_t tok0 = span.tok0;
+  const int nch = (T + C - 1) / C;
+  const size_t KV = (size_t)K * V;
+  auto chunk_t0 = [&](int j) { return (nch - 1 - j) * C; };      // chunk j of the sweep = time chunk nch-1-j
+  auto chunk_len = [&](int j) { return min(C, T - chunk_t0(j)); };
+  auto slot_f = [&](int j) { return reinterpret_cast<float *>(base + S::oRing + (uint32_t)(j & (kRingTc - 1)) * S::slot_bytes); };
+  auto step_sa = [&](int j, int s) { return base_sa + S::oState + (uint32_t)((j & 1) * (kCTc + 1) + s) * kStepBytes; };
+
+  if (tid == 0) {
+    for (int s = 0; s < kRingTc; ++s) { mbar_init(&in_full[s], 1); mbar_init(&out_full[s], kChainWarps + kHelpWarps); mbar_init(&slot_free[s], 1); }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&st_ready[s], kChainWarps);
+      mbar_init(&st_free[s], kChainWarps + kHelpWarps + 1);     // reverse warps, helpers, and the dW product's commit
+      mbar_init(&dx_full[s], kChainWarps);
+      mbar_init(&dx_free[s], kHelpWarps + 1);
+    }
+    mbar_init(rec_done, 1); mbar_init(rev_done, 1); mbar_init(dw_done, 1);
+    fence_mbar_init();
+  }
+  if (warp == 0) {
+    __syncwarp();
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemColsBwd) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
+  if (warp < 8) {
+    // W^T (warps 0-3) and W (warps 4-7) into tensor memory, lane = row, column c = elements 2c, 2c+1:
+    // W^T row j = W[:, j]; W row l = W[l, :]
+    const int r = 32 * (warp & 3) + lane;
+    const uint16_t *w = reinterpret_cast<const uint16_t *>(a.W) + (size_t)n * V * V;
+    const bool transposed = warp < 4;
+#pragma unroll 1
+    for (int c0 = 0; c0 < 64; c0 += 8) {
+      uint32_t v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int x = 2 * (c0 + e);
+        v[e] = transposed ? ((uint32_t)w[(size_t)x * V + r] | ((uint32_t)w[(size_t)(x + 1) * V + r] << 16))
+                          : *reinterpret_cast<const uint32_t *>(w + (size_t)r * V + x);
+      }
+      tmem_st8(tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (transposed ? kColWT : kColW) + (uint32_t)c0, v);
+    }
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  bool failed = false;
+
+  if (warp < 2 * kChainWarps) {
+    // ================================================================= chain warps
+    const bool is_rec = warp < kChainWarps;
+    const int wg = warp % kChainWarps, quarter = wg & 3, half = wg >> 2;
+    const int j = 32 * quarter + lane;                 // this thread's state column = tensor-memory lane
+    const int i0 = kNT * half;                         // its first row inside the CTA's slab
+    const int ct = 128 * half + j;                     // index among the role's 256 threads
+    uint32_t el[kNT];                                  // its 2-byte elements inside a slab
+#pragma unroll
+    for (int x = 0; x < kNT; ++x) el[x] = slab_off(i0 + x, j);
+    const uint32_t priv = kTileBytes + (uint32_t)ct * 16u;     // its 16 bytes of Z inside a step block; H - Z follows 4 096 bytes on
+    const uint32_t lane_tm = tmem_base + ((uint32_t)(32 * quarter) << 16) + (uint32_t)i0;
+    constexpr uint32_t idesc = idesc_bf16(128, kNR);
+    // eight MMAs of 16 K indices: 8 columns of A in tensor memory, 32 bytes inside a 128-byte row of
+    // the slab (then the next 64-index block); issued by one elected lane of the role's first warp
+    auto issue = [&](uint32_t d_col, uint32_t a_col, uint32_t slab_sa, uint64_t *bar) {
+      if (wg == 0 && elect_one()) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)
+          umma_bf16_ts(tmem_base + d_col, tmem_base + a_col + 8u * kk,
+                       smem_desc_sw128(slab_sa + (uint32_t)(kk >> 2) * (kNR * 128) + (uint32_t)(kk & 3) * 32u), idesc, kk > 0);
+        umma_commit_tc(bar);
+      }
+    };
+    auto store_slab = [&](uint32_t slab_sa, const float (&x)[kNT]) {
+#pragma unroll
+      for (int i = 0; i < kNT; i += 2) {
+        const uint32_t pk = pack_bf16(x[i], x[i + 1]);
+        asm volatile("st.shared.b16 [%0], %1;" ::"r"(slab_sa + el[i]), "h"((uint16_t)(pk & 0xffffu)) : "memory");
+        asm volatile("st.shared.b16 [%0], %1;" ::"r"(slab_sa + el[i + 1]), "h"((uint16_t)(pk >> 16)) : "memory");
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy writes -> visible to the tensor core
+    };
+    auto role_sync = [&]() {
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      asm volatile("bar.sync %0, %1;" ::"r"(is_rec ? 1 : 2), "n"(kChainWarps * 32) : "memory");
+    };
+
+    if (is_rec) {
+      // --------------------------------------------------------------- recompute
+      uint32_t nprod = 0;
+      for (int jc = 0; jc < nch && !failed; ++jc) {
+        const int len = chunk_len(jc);
+        float H[kNT];
+        const float *ck = a.ckpt + ((size_t)unit * a.nchunks + (nch - 1 - jc)) * KV + (size_t)(rbase + i0) * V + j;
+#pragma unroll
+        for (int x = 0; x < kNT; ++x) H[x] = ck[(size_t)x * V];
+        if (!mbar_wait(&in_full[jc & (kRingTc - 1)], (jc / kRingTc) & 1)) { failed = true; break; }
+        if (jc >= 2 && !mbar_wait(&st_free[jc & 1], ((jc >> 1) - 1) & 1)) { failed = true; break; }
+        const float *sf = slot_f(jc);
+        for (int s = 0; s < len; ++s) {
+          const uint32_t blk = step_sa(jc, s);
+          store_slab(blk, H);                            // H_{t-1}: this step's B operand, and what dW and dq read
+          role_sync();
+          issue(kColP, kColWT, blk, rec_done);
+          float kk[kNT];
+#pragma unroll
+          for (int x = 0; x < kNT / 4; ++x) {
+            const float4 k4 = *reinterpret_cast<const float4 *>(sf + S::oK + s * kNR + i0 + 4 * x);
+            kk[4 * x] = k4.x; kk[4 * x + 1] = k4.y; kk[4 * x + 2] = k4.z; kk[4 * x + 3] = k4.w;
+          }
+          const float vj = sf[S::oVv + s * V + j], f = sf[S::oF + s];
+          if (!mbar_wait(rec_done, nprod & 1u)) { failed = true; break; }
+          ++nprod;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          float P[kNT];
+          tmem_ld(lane_tm + kColP, P);
+          uint32_t zw[kNT / 2], dw[kNT / 2];
+#pragma unroll
+          for (int x = 0; x < kNT; x += 2) {
+            const float2 pre = __ffma2_rn(make_float2(kk[x], kk[x + 1]), make_float2(vj, vj), make_float2(P[x], P[x + 1]));
+            const float2 z = make_float2(tanh_approx(pre.x), tanh_approx(pre.y));                            // Eq. 1
+            const float2 d = __ffma2_rn(z, make_float2(-1.f, -1.f), make_float2(H[x], H[x + 1]));             // H_{t-1} - Z
+            const float2 h = __ffma2_rn(make_float2(f, f), d, z);                                           // Eq. 2
+            H[x] = h.x; H[x + 1] = h.y;
+            zw[x / 2] = pack_f16x2(z.x, z.y);
+            dw[x / 2] = pack_f16x2(d.x, d.y);
+          }
+          *reinterpret_cast<uint4 *>(base + (blk - base_sa) + priv) = make_uint4(zw[0], zw[1], zw[2], zw[3]);
+          *reinterpret_cast<uint4 *>(base + (blk - base_sa) + priv + 4096u) = make_uint4(dw[0], dw[1], dw[2], dw[3]);
+        }
+        if (failed) break;
+        store_slab(step_sa(jc, len), H);                 // the state after the chunk's last step: H_t of its last step's dq
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&st_ready[jc & 1]);
+      }
+    } else {
+      // --------------------------------------------------------------- reverse
+      float Cg[kNT];
+      if (a.d_hT) {
+#pragma unroll
+        for (int x = 0; x < kNT; ++x) Cg[x] = a.d_hT[(size_t)unit * KV + (size_t)(rbase + i0 + x) * V + j];
+      } else {
+#pragma unroll
+        for (int x = 0; x < kNT; ++x) Cg[x] = 0.f;
+      }
+      const float clip = a.dh_clip;
+      uint32_t nstep = 0;          // steps taken so far: picks the dX slab and the phase of rev_done
+      bool pending = false;        // a product dX W^T is in flight and not yet added to Cg
+      auto absorb = [&]() -> bool {   // Cg <- f G (already there) + dX W^T
+        if (!mbar_wait(rev_done, (nstep - 1u) & 1u)) return false;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        float Pp[kNT];
+        tmem_ld(lane_tm + kColC, Pp);
+#pragma unroll
+        for (int x = 0; x < kNT; ++x) {
+          Cg[x] += Pp[x];
+          if (clip > 0.f) Cg[x] = fminf(fmaxf(Cg[x], -clip), clip);
+        }
+        pending = false;
+        return true;
+      };
+      for (int jc = 0; jc < nch && !failed; ++jc) {
+        const int len = chunk_len(jc);
+        if (!mbar_wait(&in_full[jc & (kRingTc - 1)], (jc / kRingTc) & 1)) { failed = true; break; }
+        if (!mbar_wait(&st_ready[jc & 1], (jc >> 1) & 1)) { failed = true; break; }
+        float *sf = slot_f(jc);
+        for (int s = len - 1; s >= 0; --s, ++nstep) {
+          const uint32_t blk = step_sa(jc, s);
+          const uint4 zr = *reinterpret_cast<const uint4 *>(base + (blk - base_sa) + priv);
+          const uint4 dr = *reinterpret_cast<const uint4 *>(base + (blk - base_sa) + priv + 4096u);
+          float qq[kNT], kk[kNT];
+#pragma unroll
+          for (int x = 0; x < kNT / 4; ++x) {
+            const float4 q4 = *reinterpret_cast<const float4 *>(sf + S::oQ + s * kNR + i0 + 4 * x);
+            const float4 k4 = *reinterpret_cast<const float4 *>(sf + S::oK + s * kNR + i0 + 4 * x);
+            qq[4 * x] = q4.x; qq[4 * x + 1] = q4.y; qq[4 * x + 2] = q4.z; qq[4 * x + 3] = q4.w;
+            kk[4 * x] = k4.x; kk[4 * x + 1] = k4.y; kk[4 * x + 2] = k4.z; kk[4 * x + 3] = k4.w;
+          }
+          const float dyj = sf[S::oDY + s * V + j], f = sf[S::oF + s], omf = 1.f - f;
+          if (pending && !absorb()) { failed = true; break; }
+          const uint32_t zw[4] = {zr.x, zr.y, zr.z, zr.w}, dw[4] = {dr.x, dr.y, dr.z, dr.w};
+          float dX[kNT];
+          float2 df2 = make_float2(0.f, 0.f), dv2 = make_float2(0.f, 0.f);
+#pragma unroll
+          for (int x = 0; x < kNT; x += 2) {
+            const float2 z = unpack_f16x2(zw[x / 2]), hmz = unpack_f16x2(dw[x / 2]);
+            const float2 G = __ffma2_rn(make_float2(qq[x], qq[x + 1]), make_float2(dyj, dyj), make_float2(Cg[x], Cg[x + 1]));   // G = C + q dy^T
+            df2 = __ffma2_rn(G, hmz, df2);                                                                                  // df = sum G (.) (H_{t-1} - Z)
+            const float2 x2 = __fmul2_rn(__fmul2_rn(make_float2(-omf, -omf), G), __ffma2_rn(z, z, make_float2(-1.f, -1.f)));   // (1-f) G (1 - Z^2)
+            const float2 c2 = __fmul2_rn(make_float2(f, f), G);                                                             // gated path into H_{t-1}
+            dv2 = __ffma2_rn(x2, make_float2(kk[x], kk[x + 1]), dv2);                                                       // dv = dX^T k, this thread's rows
+            dX[x] = x2.x; dX[x + 1] = x2.y;
+            Cg[x] = c2.x; Cg[x + 1] = c2.y;
+          }
+          // dv: the two row halves of a column are added by the writer; df: one partial per thread
+          sf[S::oDFP + s * 256 + ct] = df2.x + df2.y;
+          if (half == 0) sf[S::oDV + s * V + j] = dv2.x + dv2.y;
+          const int xb = nstep & 1u;
+          if (nstep >= 2 && !mbar_wait(&dx_free[xb], ((nstep >> 1) - 1u) & 1u)) { failed = true; break; }
+          const uint32_t dx_sa = base_sa + S::oDx + (uint32_t)xb * kTileBytes;
+          store_slab(dx_sa, dX);
+          role_sync();
+          if (half == 1) sf[S::oDV + s * V + j] += dv2.x + dv2.y;   // (after the barrier: half 0 has stored)
+          issue(kColC, kColW, dx_sa, rev_done);
+          pending = true;
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&dx_full[xb]);
+        }
+        if (failed) break;
+        __syncwarp();
+        if (lane == 0) { mbar_arrive(&st_free[jc & 1]); mbar_arrive(&out_full[jc & (kRingTc - 1)]); }
+      }
+      if (!failed && pending && !absorb()) failed = true;   // the last step's product (nstep has moved past it)
+      if (a.dh0 && !failed) {
+#pragma unroll
+        for (int x = 0; x < kNT; ++x) a.dh0[(size_t)unit * KV + (size_t)(rbase + i0 + x) * V + j] = Cg[x];
+      }
+    }
+  } else if (warp < 2 * kChainWarps + kHelpWarps) {
+    // ================================================================= helper warps
+    const int h = warp - 2 * kChainWarps, g = lane >> 2, c = lane & 3;
+    // ldmatrix of a 16 x 16 A fragment (k-tile kt) of a slab: lane supplies row (lane % 8) + 8 ((lane / 8) % 2)
+    // of the 16-byte chunk 2 kt + lane / 16
+    const int lrow = (lane & 7) + 8 * ((lane >> 3) & 1);
+    uint32_t aoff[2];
+#pragma unroll
+    for (int x = 0; x < 2; ++x) aoff[x] = slab_off(lrow, 16 * (2 * h + x) + 8 * (lane >> 4));
+    constexpr uint32_t idesc_dw = idesc_bf16_mn(128, V);
+    uint32_t nstep = 0;
+    for (int jc = 0; jc < nch && !failed; ++jc) {
+      const int len = chunk_len(jc);
+      if (!mbar_wait(&st_ready[jc & 1], (jc >> 1) & 1)) { failed = true; break; }
+      float *sf = slot_f(jc);
+      for (int s = len - 1; s >= 0; --s, ++nstep) {
+        const int xb = nstep & 1u;
+        if (!mbar_wait(&dx_full[xb], (nstep >> 1) & 1u)) { failed = true; break; }
+        const uint32_t ht = step_sa(jc, s), hn = step_sa(jc, s + 1), xt = base_sa + S::oDx + (uint32_t)xb * kTileBytes;
+        if (h == 0 && elect_one()) {
+          // dW += H_{t-1}^T dX: M = l (two 64-element blocks kNR * 128 bytes apart), N = j likewise,
+          // K = the slab's 16 rows (two 8-row atoms 1024 bytes apart)
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          umma_bf16_ss(tmem_base + kColDW, smem_desc_mn_sw128(ht, kNR * 128), smem_desc_mn_sw128(xt, kNR * 128), idesc_dw, nstep > 0 ? 1u : 0u);
+          umma_commit_tc(&dx_free[xb]);
+          if (s == 0) umma_commit_tc(&st_free[jc & 1]);
+        }
+        __syncwarp();
+        // dq = H_t dy and dk = dX v over this warp's 32 columns (two k-tiles), rows g and g + 8
+        float dq[4] = {0.f, 0.f, 0.f, 0.f}, dk[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+          const int kt = 2 * h + x;
+          uint32_t A[4], bq0, bq1, bk0, bk1;
+          const float *dyb = sf + S::oDYB + s * (V / 2) + 8 * kt, *vb = sf + S::oVB + s * (V / 2) + 8 * kt;
+          bq0 = __float_as_uint(dyb[c]); bq1 = __float_as_uint(dyb[4 + c]);
+          bk0 = __float_as_uint(vb[c]); bk1 = __float_as_uint(vb[4 + c]);
+          ldmatrix_x4(hn + aoff[x], A);
+          mma_bf16_16816(dq, A, bq0, bq1);
+          ldmatrix_x4(xt + aoff[x], A);
+          mma_bf16_16816(dk, A, bk0, bk1);
+        }
+        if (c == 0) {
+          sf[S::oDQ + (s * kHelpWarps + h) * kNR + g] = dq[0]; sf[S::oDQ + (s * kHelpWarps + h) * kNR + g + 8] = dq[2];
+          sf[S::oDK + (s * kHelpWarps + h) * kNR + g] = dk[0]; sf[S::oDK + (s * kHelpWarps + h) * kNR + g + 8] = dk[2];
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&dx_free[xb]);
+      }
+      if (failed) break;
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(&st_free[jc & 1]); mbar_arrive(&out_full[jc & (kRingTc - 1)]); }
+    }
+    // the dW accumulator (lane = row l, column = j) goes to this CTA's partial sum
+    if (h == 0 && elect_one()) umma_commit_tc(dw_done);
+    __syncwarp();
+    const bool landed = mbar_wait(dw_done, 0);
+    if (!landed) failed = true;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    float *row = a.dW_part + ((size_t)(b * RS + rs) * N + n) * V * V + (size_t)(32 * h + lane) * V;
+#pragma unroll 1
+    for (int x = 0; x < V / 8; ++x) {
+      float r[8];
+      if (landed && !failed && nstep > 0) {
+        tmem_ld(tmem_base + ((uint32_t)(32 * h) << 16) + kColDW + 8u * x, r);
+      } else {   // no step at all (an empty sequence): the sum is empty
+#pragma unroll
+        for (int e = 0; e < 8; ++e) r[e] = 0.f;
+      }
+      *reinterpret_cast<float4 *>(row + 8 * x) = make_float4(r[0], r[1], r[2], r[3]);
+      *reinterpret_cast<float4 *>(row + 8 * x + 4) = make_float4(r[4], r[5], r[6], r[7]);
+    }
+  } else {
+    // ================================================================= loader and writer warps
+    const bool is_loader = warp == 2 * kChainWarps + kHelpWarps;
+    const int hq = n / (N / a.Nq), hk = n / (N / a.Nk);
+    const float al = a.alpha ? a.alpha[n] : 1.f, be = a.beta ? a.beta[n] : 0.f;
+    const __nv_bfloat16 *qg = static_cast<const __nv_bfloat16 *>(a.q), *kg = static_cast<const __nv_bfloat16 *>(a.k);
+    const __nv_bfloat16 *vg = static_cast<const __nv_bfloat16 *>(a.v), *dyg = static_cast<const __nv_bfloat16 *>(a.dy);
+    const __nv_bfloat16 *wr = static_cast<const __nv_bfloat16 *>(a.w_r);
+    const size_t TT = (size_t)a.TT;
+    if (is_loader) {
+      for (int jc = 0; jc < nch; ++jc) {   // runs up to kRingTc chunks ahead of the writer
+        if (jc >= kRingTc && !mbar_wait<1000>(&slot_free[jc & (kRingTc - 1)], ((jc / kRingTc) - 1) & 1)) { failed = true; break; }
+        float *sf = slot_f(jc);
+        const int t0 = chunk_t0(jc), len = chunk_len(jc);
+        const size_t bt0 = tok0 + t0;
+        // q, k: 16 rows = 2 chunks of 16 bytes per step; v, dy: 16 chunks per step
+        if (lane < 2 * len) {
+          const int t = lane >> 1, i = (lane & 1) * 8;
+          const uint4 qr = *reinterpret_cast<const uint4 *>(qg + (bt0 + t) * a.qs + (size_t)hq * K + rbase + i);
+          const uint4 kr = *reinterpret_cast<const uint4 *>(kg + (bt0 + t) * a.ks + (size_t)hk * K + rbase + i);
+          store8_bf16_as_f32(sf + S::oQ + t * kNR + i, qr);
+          store8_bf16_as_f32(sf + S::oK + t * kNR + i, kr);
+        }
+        for (int x = lane; x < 16 * len; x += 32) {
+          const int t = x >> 4, i = (x & 15) * 8;
+          const uint4 vr = *reinterpret_cast<const uint4 *>(vg + (bt0 + t) * a.vs + (size_t)n * V + i);
+          const uint4 dr = *reinterpret_cast<const uint4 *>(dyg + ((bt0 + t) * N + n) * V + i);
+          store8_bf16_as_f32(sf + S::oVv + t * V + i, vr);
+          store8_bf16_as_f32(sf + S::oDY + t * V + i, dr);
+          reinterpret_cast<uint4 *>(sf + S::oVB)[x] = vr;
+          reinterpret_cast<uint4 *>(sf + S::oDYB)[x] = dr;
+        }
+        if (lane < len) {
+          float dfdx;
+          sf[S::oF + lane] = gate_value(a.gate_kind, a.gate[(bt0 + lane) * N + n], al, be, &dfdx);
+          sf[S::oDF + lane] = dfdx;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&in_full[jc & (kRingTc - 1)]);
+      }
+    } else {
+      for (int jc = 0; jc < nch; ++jc) {
+        if (!mbar_wait<1000>(&out_full[jc & (kRingTc - 1)], (jc / kRingTc) & 1)) { failed = true; break; }
+        const float *sf = slot_f(jc);
+        const int t0 = chunk_t0(jc), len = chunk_len(jc);
+        const size_t bt0 = tok0 + t0;
+        // dq, dk: the four helpers' shares of this CTA's 16 rows
+        if (lane < 16) {
+          for (int t = 0; t < len; ++t) {
+            float sq = 0.f, sk = 0.f;
+#pragma unroll
+            for (int hh = 0; hh < kHelpWarps; ++hh) {
+              sq += sf[S::oDQ + (t * kHelpWarps + hh) * kNR + lane];
+              sk += sf[S::oDK + (t * kHelpWarps + hh) * kNR + lane];
+            }
+            if (a.dq_part) a.dq_part[((bt0 + t) * N + n) * K + rbase + lane] = sq;
+            else static_cast<__nv_bfloat16 *>(a.dq)[((bt0 + t) * a.Nq + hq) * K + rbase + lane] = __float2bfloat16_rn(sq);
+            if (a.dk_part) a.dk_part[((bt0 + t) * N + n) * K + rbase + lane] = sk;
+            else static_cast<__nv_bfloat16 *>(a.dk)[((bt0 + t) * a.Nk + hk) * K + rbase + lane] = __float2bfloat16_rn(sk);
+          }
+        }
+        // dv of this CTA's rows (+ w_r (.) dy from Eq. 3, added by the first row slab only)
+        for (int x = lane; x < len * (V / 2); x += 32) {
+          const int t = x / (V / 2), jj = (x % (V / 2)) * 2;
+          const float2 p = *reinterpret_cast<const float2 *>(sf + S::oDV + t * V + jj);
+          float s0 = p.x, s1 = p.y;
+          if (wr && rs == 0) {
+            s0 = fmaf(__bfloat162float(wr[(size_t)n * V + jj]), sf[S::oDY + t * V + jj], s0);
+            s1 = fmaf(__bfloat162float(wr[(size_t)n * V + jj + 1]), sf[S::oDY + t * V + jj + 1], s1);
+          }
+          const size_t o = ((bt0 + t) * N + n) * V + jj;
+          if (a.dv_part) *reinterpret_cast<float2 *>(a.dv_part + (size_t)rs * TT * N * V + o) = make_float2(s0, s1);
+          else *reinterpret_cast<uint32_t *>(static_cast<__nv_bfloat16 *>(a.dv) + o) = pack_bf16(s0, s1);
+        }
+        // dgate: one df partial per reverse thread; fixed-order sum, then the gate's slope
+        for (int t = 0; t < len; ++t) {
+          float sdf = 0.f;
+#pragma unroll
+          for (int x = 0; x < 8; ++x) sdf += sf[S::oDFP + t * 256 + 32 * x + lane];
+#pragma unroll
+          for (int off = 16; off > 0; off >>= 1) sdf += __shfl_xor_sync(0xffffffffu, sdf, off);
+          if (lane == 0) {
+            sdf *= sf[S::oDF + t];
+            const size_t o = (bt0 + t) * N + n;
+            if (a.dgate_part) a.dgate_part[(size_t)rs * TT * N + o] = sdf;
+            else a.dgate[o] = sdf;
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&slot_free[jc & (kRingTc - 1)]);
+      }
+    }
+  }
+  if (failed) report_timeout(a.dev_status);
+  // common exit: every loop above ends after a bounded time
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemColsBwd) : "memory");
+  }
+}
+
+}  // namespace
+
+int bwd_tc_rows_per_cta() { return kNR; }
+int bwd_tc_chunk() { return kCTc; }
+
+cudaError_t launch_bwd_bf16_tc(const ScanArgs &a, cudaStream_t s) {
+  if (a.V != kV || a.KC != kNR || a.C < 1 || a.C > kCTc) return cudaErrorInvalidValue;
+  const size_t smem = TcBwdSmem::total;
+  cudaError_t e = cudaFuncSetAttribute(bwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  bwd_tc_kernel<<<a.B * a.N * (a.K / kNR), kThreads, smem, s>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace m2rnn
