@@ -23,10 +23,10 @@ int sm_count() {
 }
 
 bool bwd_use_tc(int B, int N, int K, int V, int io_dtype) {
-  if (io_dtype != M2RNN_BF16 || V != 128) return false;
+  if (io_dtype != M2RNN_BF16 || V != 128 || K % bwd_tc_rows_per_cta()) return false;   // 32-row CTAs
   const char *variant = getenv("M2RNN_BWD_VARIANT");
   if (variant && !strcmp(variant, "mma")) return false;
-  (void)B; (void)N; (void)K;
+  (void)B; (void)N;
   return true;
 }
 
@@ -36,7 +36,7 @@ BwdPlan plan_bwd(int B, int N, int K, int V, int io_dtype) {
     pl.KC = K; pl.C = 16; pl.C_max = 64;
     return pl;
   }
-  if (bwd_use_tc(B, N, K, V, io_dtype)) {   // 16-row CTAs, chunks of four steps
+  if (bwd_use_tc(B, N, K, V, io_dtype)) {   // 32-row CTAs, chunks of four steps
     pl.KC = bwd_tc_rows_per_cta(); pl.C = pl.C_max = bwd_tc_chunk();
     return pl;
   }

@@ -15,8 +15,9 @@ F = inputs.to_f64
 SHAPES = [
     # B, T, N, K, Nq, Nk        (V = 128)
     (1, 21, 2, 128, 0, 0),
-    (2, 37, 2, 16, 0, 0),       # one 16-row CTA per unit: dv and dgate written directly
-    (1, 26, 4, 48, 2, 4),       # three CTAs per unit, shared query heads
+    (2, 37, 2, 32, 0, 0),       # one 32-row CTA per unit: dv and dgate written directly
+    (1, 26, 4, 96, 2, 4),       # three CTAs per unit, shared query heads
+    (1, 13, 2, 48, 0, 0),       # K not a multiple of 32: the register kernel takes it either way
     (2, 9, 3, 32, 1, 1),        # the multi-value layout
     (3, 1, 2, 64, 0, 0),        # a single step
     (1, 4, 1, 64, 0, 0),        # exactly one chunk
@@ -45,7 +46,7 @@ def test_checkpoints_recomputed_when_not_passed(oracle):
 def test_saturating_inputs_and_clipping(oracle):
     cfg = ScanConfig("sat", B=2, T=48, N=2, K=128, V=128, dist="saturating", gate_mean=0.0, seed=7)
     parity.check_bwd(oracle, cfg)
-    cfg = ScanConfig("clip", B=2, T=24, N=2, K=16, V=128, dist="saturating", gate_mean=1.0, seed=9)
+    cfg = ScanConfig("clip", B=2, T=24, N=2, K=32, V=128, dist="saturating", gate_mean=1.0, seed=9)
     parity.check_bwd(oracle, cfg, dh_clip=0.5)
 
 
