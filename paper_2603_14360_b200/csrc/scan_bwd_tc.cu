@@ -60,7 +60,7 @@ constexpr int kCTc = 4;              // steps per chunk = checkpoint interval of
 // tensor-memory columns: W^T, W (two bf16 per column), the two chain accumulators, dW
 constexpr uint32_t kColWT = 0, kColW = 64, kColP = 128, kColC = 160, kColDW = 256, kTmemColsBwd = 512;
 
-constexpr uint32_t kTileBytes = kNR * 256;                   // a 32 x 128 bf16 slab: 2 blocks of [32 rows][128 bytes]
+constexpr uint32_t kTileBytes = kNR * 256;                   // a 32 x 128 bf16 slab: 128 columns of 64 bytes
 constexpr uint32_t kPrivBytes = kChainWarps * 32 * 16;       // per thread 8 x fp16 = 16 bytes of Z
 constexpr uint32_t kStepBytes = kTileBytes + kPrivBytes;     // 16 384: keeps every tile on a 1024-byte boundary
 
@@ -83,12 +83,16 @@ struct TcBwdSmem {
 };
 static_assert(kCTc == 4, "the slot layout keeps f and its slope in four words each");
 
-// byte offset of element (row i, column l) of a slab: block l / 64, 16-byte chunk ((l % 64) / 8) ^ (i % 8)
+// A slab holds 32 state rows x 128 columns of bf16 COLUMN by column: column l is a row of 64 bytes
+// (the 32 state rows, contiguous), 64-byte swizzled: the 16-byte chunk (i / 8) of column l sits at
+// chunk (i / 8) ^ ((l / 2) % 4).  A chain thread's 8 rows of its column are one 16-byte access; the
+// tensor core reads the slab N-major (N = state rows) as the B operand of the chain products and
+// K-major (K = state rows) as either operand of the dW product.
 __device__ __forceinline__ uint32_t slab_off(int i, int l) {
-  return (uint32_t)(l >> 6) * (kNR * 128) + (uint32_t)i * 128u + ((((uint32_t)(l & 63) >> 3) ^ (uint32_t)(i & 7)) << 4) + (uint32_t)(l & 7) * 2u;
+  return (uint32_t)l * 64u + ((((uint32_t)i >> 3) ^ (((uint32_t)l >> 1) & 3u)) << 4) + (uint32_t)(i & 7) * 2u;
 }
-__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
 }
 __device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
   uint32_t r;
@@ -184,18 +188,13 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_tc_kernel(ScanArgs a) {
     const int quarter = warp & 3, rg = warp >> 2;
     const int j = 32 * quarter + lane;                 // this thread's state column = tensor-memory lane
     const int i0 = kNT * rg;                           // its first row inside the CTA's slab
-    uint32_t el[kNT];                                  // its 2-byte elements inside a slab
-#pragma unroll
-    for (int x = 0; x < kNT; ++x) el[x] = slab_off(i0 + x, j);
+    static_assert(kNT == 8, "a thread's rows of its column are one 16-byte chunk of a slab");
+    const uint32_t own = slab_off(i0, j);              // its 16 bytes inside a slab
     const uint32_t priv = kTileBytes + (uint32_t)(128 * rg + j) * 16u;   // its 16 bytes of Z inside a step block
     const uint32_t lane_tm = tmem_base + ((uint32_t)(32 * quarter) << 16) + (uint32_t)i0;
     auto store_slab = [&](uint32_t slab_sa, const float (&x)[kNT]) {
-#pragma unroll
-      for (int i = 0; i < kNT; i += 2) {
-        const uint32_t pk = pack_bf16(x[i], x[i + 1]);
-        asm volatile("st.shared.b16 [%0], %1;" ::"r"(slab_sa + el[i]), "h"((uint16_t)(pk & 0xffffu)) : "memory");
-        asm volatile("st.shared.b16 [%0], %1;" ::"r"(slab_sa + el[i + 1]), "h"((uint16_t)(pk >> 16)) : "memory");
-      }
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slab_sa + own), "r"(pack_bf16(x[0], x[1])), "r"(pack_bf16(x[2], x[3])),
+                   "r"(pack_bf16(x[4], x[5])), "r"(pack_bf16(x[6], x[7])) : "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy writes -> visible to the tensor core
     };
     // a slab is complete when every chain warp has said so; the MMA warp takes it from there (its
@@ -263,6 +262,8 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_tc_kernel(ScanArgs a) {
           const uint32_t zw[kNT / 2] = {z0.x, z0.y, z0.z, z0.w};
           const float dyj = __uint_as_float((uint32_t)reinterpret_cast<const uint16_t *>(sfV + S::oDYB)[sv * V + j] << 16);
           const float f = sfV[S::oF + sv], omf = 1.f - f;
+          uint32_t hw[kNT / 2];   // H_{t-1}, this thread's own chunk of the slab it wrote a chunk ago
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(hw[0]), "=r"(hw[1]), "=r"(hw[2]), "=r"(hw[3]) : "r"(blkV + own));
           if (pending && !absorb()) { failed = true; break; }
           float dX[kNT];
           float2 df2 = make_float2(0.f, 0.f), dv2 = make_float2(0.f, 0.f);
@@ -270,10 +271,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_tc_kernel(ScanArgs a) {
           for (int r = 0; r < kNT; r += 2) {
             const float2 qq = *reinterpret_cast<const float2 *>(sfV + S::oQ + sv * kNR + i0 + r);
             const float2 kk = *reinterpret_cast<const float2 *>(sfV + S::oK + sv * kNR + i0 + r);
-            uint16_t h0, h1;      // H_{t-1}, this thread's own elements of the slab it wrote a chunk ago
-            asm volatile("ld.shared.b16 %0, [%1];" : "=h"(h0) : "r"(blkV + el[r]));
-            asm volatile("ld.shared.b16 %0, [%1];" : "=h"(h1) : "r"(blkV + el[r + 1]));
-            const float2 hp = make_float2(__uint_as_float((uint32_t)h0 << 16), __uint_as_float((uint32_t)h1 << 16));
+            const float2 hp = make_float2(__uint_as_float(hw[r / 2] << 16), __uint_as_float(hw[r / 2] & 0xffff0000u));
             const float2 z = unpack_f16x2(zw[r / 2]);
             const float2 G = __ffma2_rn(qq, make_float2(dyj, dyj), make_float2(Cg[r], Cg[r + 1]));                             // G = C + q dy^T
             df2 = __ffma2_rn(G, __ffma2_rn(z, make_float2(-1.f, -1.f), hp), df2);                                          // df = sum G (.) (H_{t-1} - Z)
@@ -337,15 +335,14 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_tc_kernel(ScanArgs a) {
   } else if (warp < kChainWarps + kHelpWarps) {
     // ================================================================= helper warps
     const int h = warp - kChainWarps, g = lane >> 2, c = lane & 3;
-    // ldmatrix of a 16 x 16 A fragment (rows 16 mt .., k-tile kt) of a slab: lane supplies row
-    // (lane % 8) + 8 ((lane / 8) % 2) of the 16-byte chunk 2 kt + lane / 16
-    const int lrow = (lane & 7) + 8 * ((lane >> 3) & 1);
+    // transposing ldmatrix of a 16 x 16 A fragment (state rows 16 mt .., columns 16 kt ..) of a slab:
+    // lane supplies column 16 kt + 8 (lane / 16) + lane % 8, rows 16 mt + 8 ((lane / 8) % 2) .. + 7
     uint32_t aoff[2][2];
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-      for (int x = 0; x < 2; ++x) aoff[mt][x] = slab_off(16 * mt + lrow, 16 * (2 * h + x) + 8 * (lane >> 4));
-    constexpr uint32_t idesc_dw = idesc_bf16_mn(128, V);
+      for (int x = 0; x < 2; ++x) aoff[mt][x] = slab_off(16 * mt + 8 * ((lane >> 3) & 1), 16 * (2 * h + x) + 8 * (lane >> 4) + (lane & 7));
+    constexpr uint32_t idesc_dw = idesc_bf16(128, V);
     uint32_t nstep = 0;
     for (int jc = 0; jc < nch && !failed; ++jc) {
       const int len = chunk_len(jc);
@@ -356,13 +353,13 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_tc_kernel(ScanArgs a) {
         if (!mbar_wait(&dx_full[xb], (nstep >> 1) & 1u)) { failed = true; break; }
         const uint32_t ht = step_sa(jc, s), hn = step_sa(jc, s + 1), xt = base_sa + S::oDx + (uint32_t)xb * kTileBytes;
         if (h == 0 && elect_one()) {
-          // dW += H_{t-1}^T dX: M = l (two 64-element blocks kNR * 128 bytes apart), N = j likewise,
-          // K = the slab's 32 rows in two MMAs of 16 (two 8-row atoms 1024 bytes apart each)
+          // dW += H_{t-1}^T dX: M = l and N = j are the slabs' columns, K = their 32 state rows (K-major),
+          // in two MMAs of 16 rows = 32 bytes of every column
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
           for (int kt = 0; kt < kNR / 16; ++kt)
-            umma_bf16_ss(tmem_base + kColDW, smem_desc_mn_sw128(ht + 2048u * kt, kNR * 128), smem_desc_mn_sw128(xt + 2048u * kt, kNR * 128),
-                         idesc_dw, (nstep > 0 || kt > 0) ? 1u : 0u);
+            umma_bf16_ss(tmem_base + kColDW, smem_desc_sw64(ht + 32u * kt), smem_desc_sw64(xt + 32u * kt), idesc_dw,
+                         (nstep > 0 || kt > 0) ? 1u : 0u);
           umma_commit_tc(&dx_free[xb]);
           if (s == 0) umma_commit_tc(&st_free[jc & 1]);
         }
@@ -380,9 +377,9 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_tc_kernel(ScanArgs a) {
 #pragma unroll
           for (int mt = 0; mt < 2; ++mt) {
             uint32_t A[4];
-            ldmatrix_x4(hn + aoff[mt][x], A);
+            ldmatrix_x4_trans(hn + aoff[mt][x], A);
             mma_bf16_16816(dq[mt], A, bq0, bq1);
-            ldmatrix_x4(xt + aoff[mt][x], A);
+            ldmatrix_x4_trans(xt + aoff[mt][x], A);
             mma_bf16_16816(dk[mt], A, bk0, bk1);
           }
         }
@@ -424,16 +421,15 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_tc_kernel(ScanArgs a) {
     // ================================================================= MMA warp
     // Follows the chain warps' schedule: per iteration and step first the recompute product, then
     // the reverse product, each as soon as its slab is complete.  Eight MMAs of 16 K indices: 8
-    // columns of A in tensor memory, 32 bytes inside a 128-byte row of the slab (then the next
-    // 64-index block).
-    constexpr uint32_t idesc = idesc_bf16(128, kNR);
+    // columns of A in tensor memory, 16 columns = 1024 bytes of the slab, read N-major.
+    constexpr uint32_t idesc = idesc_bf16(128, kNR) | (1u << 16);
     auto issue = [&](uint32_t d_col, uint32_t a_col, uint32_t slab_sa, uint64_t *bar) {
       if (elect_one()) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
           umma_bf16_ts(tmem_base + d_col, tmem_base + a_col + 8u * kk,
-                       smem_desc_sw128(slab_sa + (uint32_t)(kk >> 2) * (kNR * 128) + (uint32_t)(kk & 3) * 32u), idesc, kk > 0);
+                       smem_desc_sw64(slab_sa + 1024u * kk), idesc, kk > 0);
         umma_commit_tc(bar);
       }
       __syncwarp();

@@ -17,6 +17,14 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t sa) {
   return (uint64_t)((sa & 0x3ffffu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
          ((uint64_t)2 << 61);
 }
+// The same with 64-byte swizzling (mode 4): rows of 64 bytes = 32 bf16, groups of 8 rows 512 bytes
+// apart, the 16-byte chunks of a row XOR-ed with (row / 2) modulo 4.  Serves both readings of such a
+// tile: K-major (a row = one M/N index, 32 K indices) and MN-major (a row = one K index, 32 M/N
+// indices); the instruction descriptor's major bits say which.
+__device__ __forceinline__ uint64_t smem_desc_sw64(uint32_t sa) {
+  return (uint64_t)((sa & 0x3ffffu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(512 >> 4) << 32) | ((uint64_t)1 << 46) |
+         ((uint64_t)4 << 61);
+}
 // Instruction descriptor of kind::f16 with bf16 operands: fp32 accumulator (bits 4-5 = 1), bf16 A
 // and B (bits 7-9 and 10-12 = 1), both K-major (bits 15, 16 = 0), N >> 3 in bits 17-22, M >> 4 in
 // bits 24-28.
