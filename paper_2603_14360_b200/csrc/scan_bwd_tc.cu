@@ -228,9 +228,13 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_tc_kernel(ScanArgs a) {
       float Pp[kNT];
       tmem_ld(lane_tm + kColC, Pp);
 #pragma unroll
-      for (int x = 0; x < kNT; ++x) {
-        Cg[x] += Pp[x];
-        if (clip > 0.f) Cg[x] = fminf(fmaxf(Cg[x], -clip), clip);
+      for (int x = 0; x < kNT; x += 2) {
+        const float2 c = __fadd2_rn(make_float2(Cg[x], Cg[x + 1]), make_float2(Pp[x], Pp[x + 1]));
+        Cg[x] = c.x; Cg[x + 1] = c.y;
+      }
+      if (clip > 0.f) {
+#pragma unroll
+        for (int x = 0; x < kNT; ++x) Cg[x] = fminf(fmaxf(Cg[x], -clip), clip);
       }
       pending = false;
       return true;
@@ -267,10 +271,15 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_tc_kernel(ScanArgs a) {
           if (pending && !absorb()) { failed = true; break; }
           float dX[kNT];
           float2 df2 = make_float2(0.f, 0.f), dv2 = make_float2(0.f, 0.f);
+          float q8[kNT], k8[kNT];
+#pragma unroll
+          for (int r = 0; r < kNT; r += 4) {
+            *reinterpret_cast<float4 *>(q8 + r) = *reinterpret_cast<const float4 *>(sfV + S::oQ + sv * kNR + i0 + r);
+            *reinterpret_cast<float4 *>(k8 + r) = *reinterpret_cast<const float4 *>(sfV + S::oK + sv * kNR + i0 + r);
+          }
 #pragma unroll
           for (int r = 0; r < kNT; r += 2) {
-            const float2 qq = *reinterpret_cast<const float2 *>(sfV + S::oQ + sv * kNR + i0 + r);
-            const float2 kk = *reinterpret_cast<const float2 *>(sfV + S::oK + sv * kNR + i0 + r);
+            const float2 qq = make_float2(q8[r], q8[r + 1]), kk = make_float2(k8[r], k8[r + 1]);
             const float2 hp = make_float2(__uint_as_float(hw[r / 2] << 16), __uint_as_float(hw[r / 2] & 0xffff0000u));
             const float2 z = unpack_f16x2(zw[r / 2]);
             const float2 G = __ffma2_rn(qq, make_float2(dyj, dyj), make_float2(Cg[r], Cg[r + 1]));                             // G = C + q dy^T
@@ -303,9 +312,12 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_tc_kernel(ScanArgs a) {
           float P[kNT];
           tmem_ld(lane_tm + kColP, P);
           uint32_t zw[kNT / 2];
+          float k8[kNT];
+#pragma unroll
+          for (int r = 0; r < kNT; r += 4) *reinterpret_cast<float4 *>(k8 + r) = *reinterpret_cast<const float4 *>(sfR + S::oK + x * kNR + i0 + r);
 #pragma unroll
           for (int r = 0; r < kNT; r += 2) {
-            const float2 kk = *reinterpret_cast<const float2 *>(sfR + S::oK + x * kNR + i0 + r);
+            const float2 kk = make_float2(k8[r], k8[r + 1]);
             const float2 pre = __ffma2_rn(kk, make_float2(vj, vj), make_float2(P[r], P[r + 1]));
             const float2 z = make_float2(tanh_approx(pre.x), tanh_approx(pre.y));                            // Eq. 1
             const float2 d = __ffma2_rn(z, make_float2(-1.f, -1.f), make_float2(H[r], H[r + 1]));             // H_{t-1} - Z
