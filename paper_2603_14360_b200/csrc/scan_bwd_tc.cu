@@ -297,7 +297,8 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_tc_kernel(ScanArgs a) {
           for (int off = 16; off > 0; off >>= 1) df += __shfl_xor_sync(0xffffffffu, df, off);
           if (lane == 0) sfV[S::oDFP + sv * kChainWarps + warp] = df;
           sfV[S::oDV + (sv * kRowGroups + rg) * V + j] = dv2.x + dv2.y;
-          if (nrev >= 2 && !mbar_wait(&dx_free[xb], ((nrev >> 1) - 1u) & 1u)) { failed = true; break; }
+          // (the buffer is free: the MMA warp issued the previous step's product, whose result was
+          // added above, only after the helpers and the dW product were through with it)
           store_slab(dx_sa, dX);
           slab_done(rev_slab);
           ++nrev;
@@ -457,6 +458,10 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_tc_kernel(ScanArgs a) {
         }
         if (x < lenV) {
           if (!mbar_wait(rev_slab, nrev & 1u)) { failed = true; break; }
+          // the NEXT step's dX goes into the other buffer as soon as this product has been added to
+          // the carried gradient: hold the product back until that buffer's last readers (the
+          // helpers and the dW product of the step before this one) are through
+          if (nrev >= 1 && !mbar_wait(&dx_free[(nrev + 1u) & 1u], ((nrev - 1u) >> 1) & 1u)) { failed = true; break; }
           issue(kColC, kColW, base_sa + S::oDx + (uint32_t)(nrev & 1u) * kTileBytes, rev_done);
           ++nrev;
         }
