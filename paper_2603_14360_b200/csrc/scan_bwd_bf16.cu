@@ -160,13 +160,23 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), V == 16 ? 2 : 1) bwd_bf
   uint64_t *st_ready = bars + 2 * kRing;      // [2]
   uint64_t *st_free = st_ready + 2;           // [2]
   uint64_t *dx_full = st_free + 2;            // [2]
-  uint64_t *dx_free = dx_full + 2;            // [2]
+  uint64_t *dx_free = dx_full + 2;            // [2] (unused: see dx_read)
   uint64_t *slot_free = dx_free + 2;          // [kRing] chunk slot written out, free for the loader
+  // steps whose dX tile the dW warps are through with, summed over those warps.  A plain counter
+  // instead of an mbarrier: the reverse warps read it at the top of a step and look at the value
+  // only where they overwrite the tile, so the read's latency is off their dependency chain (an
+  // mbarrier wait at that point cost up to 10 % of a V = 16 step, 2 % at V = 64).  The dW warps
+  // add to it with release semantics after their last read of the tile; the overwrite of the tile
+  // is control-dependent on the value read (a store is never issued speculatively), and the slow
+  // path re-reads with acquire semantics
+  uint32_t *dx_read = reinterpret_cast<uint32_t *>(slot_free + kRing);
+  static_assert((3 * kRing + 8) * 8 + 4 <= kBarBytes, "barrier area");
   if (tid == 0) {
+    *dx_read = 0u;
     for (int s = 0; s < kRing; ++s) { mbar_init(&in_full[s], 1); mbar_init(&out_full[s], NWC + NDW); mbar_init(&slot_free[s], 1); }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&st_ready[s], NWC); mbar_init(&st_free[s], NWC + NDW);
-      mbar_init(&dx_full[s], NWC); mbar_init(&dx_free[s], NDW);
+      mbar_init(&dx_full[s], NWC);
     }
     fence_mbar_init();
   }
@@ -434,6 +444,7 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), V == 16 ? 2 : 1) bwd_bf
       }
       if constexpr (KT == 1) d[1][0] = d[1][2] = 0.f;
     };
+    const uint32_t dx_read_sa = smem_u32(dx_read);
     uint32_t hn[NT][2];   // H_t of the step at hand as bf16 pairs = the H_{t-1} tile of the step done before
     for (int j = 0; j < nch; ++j) {
       const int len = chunk_len(j);
@@ -459,6 +470,8 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), V == 16 ? 2 : 1) bwd_bf
 #define pDFP (kWalk ? run.dfp : sl + 4u * (L.oDFP + (s * NWC + w) * 32 + lane))
 #define pDQ (kWalk ? run.dq : sl + 4u * (L.oDQ + s * KC + r0))
 #define pDK (kWalk ? run.dk : sl + 4u * (L.oDK + s * KC + r0))
+        uint32_t dx_seen;
+        asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(dx_seen) : "r"(dx_read_sa) : "memory");
         uint32_t hp[NT][2];
         tile_load_at(st, w, toff, hp);
         const uint32_t zs = kWalk ? st + zoff : zfrag_sa(st, w);
@@ -519,7 +532,19 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), V == 16 ? 2 : 1) bwd_bf
         if constexpr (kPacked) df = df2.x + df2.y;
         // hand dX to the dW warps
         const int xb = nstep & 1;
-        if (nstep >= 2 && !mbar_wait(&dx_free[xb], ((nstep >> 1) - 1) & 1)) { report_timeout(a.dev_status); return; }
+        if (nstep >= 2) {   // the dW warps must be through with the tile written two steps ago
+          const uint32_t need = (uint32_t)NDW * (uint32_t)(nstep - 1);
+          bool ok = (int32_t)(dx_seen - need) >= 0;
+          if (!ok) {
+            const long long t0 = clock64();
+            do {
+              __nanosleep(20);
+              asm volatile("ld.acquire.cta.shared.u32 %0, [%1];" : "=r"(dx_seen) : "r"(dx_read_sa) : "memory");
+              ok = (int32_t)(dx_seen - need) >= 0;
+            } while (!ok && clock64() - t0 < kWaitCycles);
+          }
+          if (!__all_sync(0xffffffffu, ok)) { report_timeout(a.dev_status); return; }
+        }
         tile_store_at(sm0 + L.dx + (uint32_t)xb * (KC * V * 2), w, toff, xp);
         __syncwarp();
         if (lane == 0) mbar_arrive(&dx_full[xb]);
@@ -653,7 +678,7 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), V == 16 ? 2 : 1) bwd_bf
           sts64(dst + 32u, make_float2(dvacc[1][0], dvacc[1][1]));
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(&dx_free[xb]);
+        if (lane == 0) asm volatile("red.release.cta.shared.add.u32 [%0], 1;" ::"r"(smem_u32(dx_read)) : "memory");
       }
       __syncwarp();
       if (lane == 0) { mbar_arrive(&st_free[j & 1]); mbar_arrive(&out_full[j & (kRing - 1)]); }
