@@ -22,9 +22,12 @@ namespace {
 // A CTA is 32 channel chunks (one warp = 256 or 512 contiguous bytes of a token) x 4 time sub-tiles.
 constexpr int kLanes = 32, kSub = 4;
 constexpr int kConvThreads = kLanes * kSub;
-constexpr int kStepsFwd = 16;                    // time steps per thread of the forward kernel
+constexpr int kStepsFwd = 64;                    // time steps per thread of the forward kernel
+constexpr int kUFwd = 8;                         // ... of which a batch of this many is loaded ahead
 constexpr int kTileFwd = kSub * kStepsFwd;       // ... per CTA
-constexpr int kStepsBwd = 32;                    // backward: longer runs, fewer halo steps
+constexpr int kStepsBwd = 64;                    // backward: longer runs, fewer halo steps
+constexpr int kUBwd = 4;                         // batch of steps loaded ahead
+constexpr int kOccBwd = 4;                       // CTAs per SM the backward kernel is compiled for
 constexpr int kTileBwd = kSub * kStepsBwd;       // one partial sum of dw and dbias per CTA
 
 template <typename T> struct Chunk;             // the channels of one thread
@@ -106,22 +109,24 @@ __global__ void __launch_bounds__(kConvThreads, 6) conv_silu_fwd_kernel(int B, i
     load_row<T, CH>(x, xs, prev, b, Tn, C, t0 - 1, c0, r1);
     to_pairs<CH>(r3, xm3); to_pairs<CH>(r2, xm2); to_pairs<CH>(r1, xm1);
   }
-  // the loads of eight steps are issued before the first is used: with three dozen warps per SM that
-  // keeps enough bytes in flight to cover the latency of HBM
-  constexpr int U = 8;
+  // Loads run one batch of U steps ahead of the arithmetic (the next batch is requested before the
+  // current one is used), so that a thread always has U to 2U rows in flight: the kernel is bound
+  // by the latency of HBM, not by its arithmetic.
+  constexpr int U = kUFwd;
   using Raw = typename Chunk<T>::Raw;
   const T *xp = x + ((size_t)b * Tn + t0) * xs + c0;
   T *op = out + ((size_t)b * Tn + t0) * os + c0;
-  for (int tb = t0; tb < t1; tb += U, xp += U * xs, op += U * os) {
-    Raw raw[U];
+  Raw cur[U], nxt[U];
 #pragma unroll
-    for (int u = 0; u < U; ++u)
-      raw[u] = tb + u < t1 ? *reinterpret_cast<const Raw *>(xp + u * xs) : Raw{};
+  for (int u = 0; u < U; ++u) cur[u] = t0 + u < t1 ? *reinterpret_cast<const Raw *>(xp + u * xs) : Raw{};
+  for (int tb = t0; tb < t1; tb += U, xp += U * xs, op += U * os) {
+#pragma unroll
+    for (int u = 0; u < U; ++u) nxt[u] = tb + U + u < t1 ? *reinterpret_cast<const Raw *>(xp + (U + u) * xs) : Raw{};
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       float xr[CH], o[CH];
       float2 x0[CP];
-      Chunk<T>::unpack(raw[u], xr);
+      Chunk<T>::unpack(cur[u], xr);
       to_pairs<CH>(xr, x0);
 #pragma unroll
       for (int e = 0; e < CP; ++e) {
@@ -132,12 +137,14 @@ __global__ void __launch_bounds__(kConvThreads, 6) conv_silu_fwd_kernel(int B, i
       }
       if (tb + u < t1) Chunk<T>::store(op + u * os, o);     // (past the end: arithmetic on stale registers, nothing stored)
     }
+#pragma unroll
+    for (int u = 0; u < U; ++u) cur[u] = nxt[u];
   }
 }
 
 // partial sums of a tile: part[tile][5][C] = dw taps 0..3 and dbias
 template <typename T>
-__global__ void __launch_bounds__(kConvThreads, 4) conv_silu_bwd_kernel(int B, int Tn, int C, const T *__restrict__ x, long long xs,
+__global__ void __launch_bounds__(kConvThreads, kOccBwd) conv_silu_bwd_kernel(int B, int Tn, int C, const T *__restrict__ x, long long xs,
                                                                      const T *__restrict__ w, const T *__restrict__ bias,
                                                                      const T *__restrict__ prev, const T *__restrict__ dout, long long ds,
                                                                      T *__restrict__ dx, long long dxs, T *__restrict__ dprev,
@@ -178,18 +185,23 @@ __global__ void __launch_bounds__(kConvThreads, 4) conv_silu_bwd_kernel(int B, i
   for (int e = 0; e < CP; ++e) d3[e] = d2[e] = d1[e] = make_float2(0.f, 0.f);
   // t runs three steps past the run: dx[t'] needs dpre[t' .. t'+3].  The loads of four steps are
   // issued before the first is used.
-  constexpr int U = 4;
+  constexpr int U = kUBwd;
   using Raw = typename Chunk<T>::Raw;
   const T *xp = x + ((size_t)b * Tn + t0) * xs + c0, *gp = dout + ((size_t)b * Tn + t0) * ds + c0;
   T *dxp = dx + ((size_t)b * Tn + t0 - 3) * dxs + c0;       // three steps behind
   const int tend = min(Tn, t1 + 3);                          // steps with inputs to read
   const float2 one = make_float2(1.f, 1.f), mone = make_float2(-1.f, -1.f);
-  for (int tb = t0; tb < t1 + 3 && work; tb += U, xp += U * xs, gp += U * ds, dxp += U * dxs) {
-    Raw rx[U], rg[U];
+  Raw rx[U], rg[U], nx[U], ng[U];
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      rx[u] = tb + u < tend ? *reinterpret_cast<const Raw *>(xp + u * xs) : Raw{};
-      rg[u] = tb + u < tend ? *reinterpret_cast<const Raw *>(gp + u * ds) : Raw{};
+  for (int u = 0; u < U; ++u) {
+    rx[u] = work && t0 + u < tend ? *reinterpret_cast<const Raw *>(xp + u * xs) : Raw{};
+    rg[u] = work && t0 + u < tend ? *reinterpret_cast<const Raw *>(gp + u * ds) : Raw{};
+  }
+  for (int tb = t0; tb < t1 + 3 && work; tb += U, xp += U * xs, gp += U * ds, dxp += U * dxs) {
+#pragma unroll
+    for (int u = 0; u < U; ++u) {   // the next batch, requested before this one is used
+      nx[u] = tb + U + u < tend ? *reinterpret_cast<const Raw *>(xp + (U + u) * xs) : Raw{};
+      ng[u] = tb + U + u < tend ? *reinterpret_cast<const Raw *>(gp + (U + u) * ds) : Raw{};
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
@@ -232,6 +244,8 @@ __global__ void __launch_bounds__(kConvThreads, 4) conv_silu_bwd_kernel(int B, i
 #pragma unroll
       for (int e = 0; e < CP; ++e) { d3[e] = d2[e]; d2[e] = d1[e]; d1[e] = d0[e]; }
     }
+#pragma unroll
+    for (int u = 0; u < U; ++u) { rx[u] = nx[u]; rg[u] = ng[u]; }
   }
   // the sums, channel by channel, for the hand-over below
   float dwv[CH][4], dbv[CH];
