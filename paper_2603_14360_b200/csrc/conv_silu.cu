@@ -3,7 +3,10 @@
 //
 // HBM-bound streaming kernels.  A thread owns four channels and walks a
 // run of consecutive time steps with the last three inputs in registers, so every input row is
-// read from HBM once (a run's three-row halo comes from L2) and every output row written once.  Input, output and
+// read from HBM once (a run's three-row halo comes from L2) and every output row written once.  The
+// rows travel through a per-thread ring in shared memory filled by cp.async two or three batches
+// ahead (no registers held while they are in flight); batches that lie wholly inside the run take
+// a form without range checks.  Input, output and
 // gradient tensors take a token stride, so that the three projections can be processed in place as
 // one [tokens, Nq K + Nk K + N V] tensor whose column slices feed the scan.
 // Backward: the thread recomputes the pre-activation, forms dpre = dout SiLU'(pre), emits
@@ -11,6 +14,8 @@
 // registers; per-tile partial sums are added by a second launch in a fixed order (bitwise
 // repeatable).
 #include <cuda_bf16.h>
+
+#include <type_traits>
 
 #include "device_common.cuh"
 #include "internal.h"
@@ -23,10 +28,11 @@ namespace {
 constexpr int kLanes = 32, kSub = 4;
 constexpr int kConvThreads = kLanes * kSub;
 constexpr int kStepsFwd = 64;                    // time steps per thread of the forward kernel
-constexpr int kUFwd = 8;                         // ... of which a batch of this many is loaded ahead
+constexpr int kUFwd = 8, kGFwd = 3;              // ... fetched in batches of kUFwd steps, kGFwd batches ahead
+constexpr int kOccFwd = 6;
 constexpr int kTileFwd = kSub * kStepsFwd;       // ... per CTA
 constexpr int kStepsBwd = 64;                    // backward: longer runs, fewer halo steps
-constexpr int kUBwd = 4;                         // batch of steps loaded ahead
+constexpr int kUBwd = 4, kGBwd = 2;              // fetched in batches of kUBwd steps, kGBwd batches ahead
 constexpr int kOccBwd = 4;                       // CTAs per SM the backward kernel is compiled for
 constexpr int kTileBwd = kSub * kStepsBwd;       // one partial sum of dw and dbias per CTA
 
@@ -74,6 +80,15 @@ __device__ __forceinline__ void to_pairs(const float (&v)[CH], float2 (&p)[CH / 
   for (int e = 0; e < CH / 2; ++e) p[e] = make_float2(v[2 * e], v[2 * e + 1]);
 }
 
+// asynchronous copy of one chunk (8 or 16 bytes) from global to shared memory; groups of copies are
+// committed and waited for per thread, and a thread reads back only what it copied itself
+template <int BYTES>
+__device__ __forceinline__ void cp_async_chunk(void *dst, const void *src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], %2;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src), "n"(BYTES) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 // row t of batch entry b: x for t >= 0, the carried rows `prev` [B,3,C] for t = -3..-1 (zeros without)
 template <typename T, int CH>
 __device__ __forceinline__ void load_row(const T *x, long long xs, const T *prev, int b, int Tn, int C, int t, int c0, float (&v)[CH]) {
@@ -84,7 +99,7 @@ __device__ __forceinline__ void load_row(const T *x, long long xs, const T *prev
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kConvThreads, 6) conv_silu_fwd_kernel(int B, int Tn, int C, const T *__restrict__ x, long long xs,
+__global__ void __launch_bounds__(kConvThreads, kOccFwd) conv_silu_fwd_kernel(int B, int Tn, int C, const T *__restrict__ x, long long xs,
                                                                      const T *__restrict__ w, const T *__restrict__ bias,
                                                                      const T *__restrict__ prev, T *__restrict__ out, long long os) {
   constexpr int CH = Chunk<T>::CH;
@@ -109,37 +124,54 @@ __global__ void __launch_bounds__(kConvThreads, 6) conv_silu_fwd_kernel(int B, i
     load_row<T, CH>(x, xs, prev, b, Tn, C, t0 - 1, c0, r1);
     to_pairs<CH>(r3, xm3); to_pairs<CH>(r2, xm2); to_pairs<CH>(r1, xm1);
   }
-  // Loads run one batch of U steps ahead of the arithmetic (the next batch is requested before the
-  // current one is used), so that a thread always has U to 2U rows in flight: the kernel is bound
-  // by the latency of HBM, not by its arithmetic.
+  // The rows of a run travel through a per-thread ring in shared memory: G batches of U rows are
+  // requested ahead with cp.async (no registers held while they are in flight), so that a thread
+  // has up to G U rows outstanding: the kernel is bound by the latency of HBM, not by arithmetic.
   constexpr int U = kUFwd;
   using Raw = typename Chunk<T>::Raw;
+  constexpr int G = sizeof(Raw) == 16 ? 2 : kGFwd;
+  __shared__ Raw ring[G][U][kConvThreads];
+  const int tid = threadIdx.x;
   const T *xp = x + ((size_t)b * Tn + t0) * xs + c0;
   T *op = out + ((size_t)b * Tn + t0) * os + c0;
-  Raw cur[U], nxt[U];
+  auto fetch = [&](int slot, const T *src, int tbase) {   // always one group, possibly empty
 #pragma unroll
-  for (int u = 0; u < U; ++u) cur[u] = t0 + u < t1 ? *reinterpret_cast<const Raw *>(xp + u * xs) : Raw{};
+    for (int u = 0; u < U; ++u)
+      if (tbase + u < t1) cp_async_chunk<sizeof(Raw)>(&ring[slot][u][tid], src + u * xs);
+    cp_async_commit();
+  };
+#pragma unroll
+  for (int g = 0; g < G; ++g) fetch(g, xp + (size_t)g * U * xs, t0 + g * U);
+  int slot = 0;
   for (int tb = t0; tb < t1; tb += U, xp += U * xs, op += U * os) {
+    cp_async_wait<G - 1>();
+    auto batch = [&](auto interior) {   // interior: the whole batch lies inside the run, no range checks
+      constexpr bool IN = decltype(interior)::value;
+      Raw cur[U];
 #pragma unroll
-    for (int u = 0; u < U; ++u) nxt[u] = tb + U + u < t1 ? *reinterpret_cast<const Raw *>(xp + (U + u) * xs) : Raw{};
+      for (int u = 0; u < U; ++u) cur[u] = IN || tb + u < t1 ? ring[slot][u][tid] : Raw{};
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      float xr[CH], o[CH];
-      float2 x0[CP];
-      Chunk<T>::unpack(cur[u], xr);
-      to_pairs<CH>(xr, x0);
+      for (int u = 0; u < U; ++u) {
+        float xr[CH], o[CH];
+        float2 x0[CP];
+        Chunk<T>::unpack(cur[u], xr);
+        to_pairs<CH>(xr, x0);
 #pragma unroll
-      for (int e = 0; e < CP; ++e) {
-        const float2 pre = __ffma2_rn(w2[3][e], x0[e], __ffma2_rn(w2[2][e], xm1[e], __ffma2_rn(w2[1][e], xm2[e], __ffma2_rn(w2[0][e], xm3[e], b2[e]))));
-        const float2 r = __fmul2_rn(pre, sigmoid2<T>(pre));
-        o[2 * e] = r.x; o[2 * e + 1] = r.y;
-        xm3[e] = xm2[e]; xm2[e] = xm1[e]; xm1[e] = x0[e];
+        for (int e = 0; e < CP; ++e) {
+          const float2 pre = __ffma2_rn(w2[3][e], x0[e], __ffma2_rn(w2[2][e], xm1[e], __ffma2_rn(w2[1][e], xm2[e], __ffma2_rn(w2[0][e], xm3[e], b2[e]))));
+          const float2 r = __fmul2_rn(pre, sigmoid2<T>(pre));
+          o[2 * e] = r.x; o[2 * e + 1] = r.y;
+          xm3[e] = xm2[e]; xm2[e] = xm1[e]; xm1[e] = x0[e];
+        }
+        if (IN || tb + u < t1) Chunk<T>::store(op + u * os, o);   // (past the end: arithmetic on stale registers, nothing stored)
       }
-      if (tb + u < t1) Chunk<T>::store(op + u * os, o);     // (past the end: arithmetic on stale registers, nothing stored)
-    }
-#pragma unroll
-    for (int u = 0; u < U; ++u) cur[u] = nxt[u];
+    };
+    if (tb + U <= t1) batch(std::true_type{});
+    else batch(std::false_type{});
+    fetch(slot, xp + (size_t)G * U * xs, tb + G * U);       // refill the batch just used
+    slot = slot + 1 == G ? 0 : slot + 1;
   }
+  cp_async_wait<0>();
 }
 
 // partial sums of a tile: part[tile][5][C] = dw taps 0..3 and dbias
@@ -191,62 +223,82 @@ __global__ void __launch_bounds__(kConvThreads, kOccBwd) conv_silu_bwd_kernel(in
   T *dxp = dx + ((size_t)b * Tn + t0 - 3) * dxs + c0;       // three steps behind
   const int tend = min(Tn, t1 + 3);                          // steps with inputs to read
   const float2 one = make_float2(1.f, 1.f), mone = make_float2(-1.f, -1.f);
-  Raw rx[U], rg[U], nx[U], ng[U];
+  // x and dout travel through per-thread rings in shared memory, G batches of U rows ahead (cp.async)
+  constexpr int G = sizeof(Raw) == 16 ? 2 : kGBwd;
+  __shared__ Raw ringx[G][U][kConvThreads], ringg[G][U][kConvThreads];
+  const int tid = threadIdx.x;
+  auto fetch = [&](int slot, const T *sx, const T *sg, int tbase) {   // always one group, possibly empty
 #pragma unroll
-  for (int u = 0; u < U; ++u) {
-    rx[u] = work && t0 + u < tend ? *reinterpret_cast<const Raw *>(xp + u * xs) : Raw{};
-    rg[u] = work && t0 + u < tend ? *reinterpret_cast<const Raw *>(gp + u * ds) : Raw{};
-  }
+    for (int u = 0; u < U; ++u)
+      if (work && tbase + u < tend) {
+        cp_async_chunk<sizeof(Raw)>(&ringx[slot][u][tid], sx + u * xs);
+        cp_async_chunk<sizeof(Raw)>(&ringg[slot][u][tid], sg + u * ds);
+      }
+    cp_async_commit();
+  };
+#pragma unroll
+  for (int g = 0; g < G; ++g) fetch(g, xp + (size_t)g * U * xs, gp + (size_t)g * U * ds, t0 + g * U);
+  int slot = 0;
   for (int tb = t0; tb < t1 + 3 && work; tb += U, xp += U * xs, gp += U * ds, dxp += U * dxs) {
+    cp_async_wait<G - 1>();
+    // interior batches (every step inside the run, every dx row inside it too) take the form
+    // without the per-step range checks, which were a third of the kernel's instructions
+    auto batch = [&](auto interior) {
+      constexpr bool IN = decltype(interior)::value;
+      Raw rx[U], rg[U];
 #pragma unroll
-    for (int u = 0; u < U; ++u) {   // the next batch, requested before this one is used
-      nx[u] = tb + U + u < tend ? *reinterpret_cast<const Raw *>(xp + (U + u) * xs) : Raw{};
-      ng[u] = tb + U + u < tend ? *reinterpret_cast<const Raw *>(gp + (U + u) * ds) : Raw{};
-    }
+      for (int u = 0; u < U; ++u) {
+        rx[u] = IN || tb + u < tend ? ringx[slot][u][tid] : Raw{};
+        rg[u] = IN || tb + u < tend ? ringg[slot][u][tid] : Raw{};
+      }
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int t = tb + u;
-      float2 d0[CP];
-      if (t < tend) {
-        float xr[CH], gr[CH];
-        float2 x0[CP], g[CP];
-        Chunk<T>::unpack(rx[u], xr);
-        Chunk<T>::unpack(rg[u], gr);
-        to_pairs<CH>(xr, x0); to_pairs<CH>(gr, g);
+      for (int u = 0; u < U; ++u) {
+        const int t = tb + u;
+        float2 d0[CP];
+        if (IN || t < tend) {
+          float xr[CH], gr[CH];
+          float2 x0[CP], g[CP];
+          Chunk<T>::unpack(rx[u], xr);
+          Chunk<T>::unpack(rg[u], gr);
+          to_pairs<CH>(xr, x0); to_pairs<CH>(gr, g);
 #pragma unroll
-        for (int e = 0; e < CP; ++e) {
-          const float2 pre = __ffma2_rn(w2[3][e], x0[e], __ffma2_rn(w2[2][e], xm1[e], __ffma2_rn(w2[1][e], xm2[e], __ffma2_rn(w2[0][e], xm3[e], b2[e]))));
-          const float2 sg = sigmoid2<T>(pre);
-          // dout * SiLU'(pre),  SiLU'(x) = sg (1 + x (1 - sg))
-          d0[e] = __fmul2_rn(__fmul2_rn(g[e], sg), __ffma2_rn(pre, __ffma2_rn(sg, mone, one), one));
-          if (t < t1) {                                      // sums over this run's own steps only
-            dw2[0][e] = __ffma2_rn(d0[e], xm3[e], dw2[0][e]); dw2[1][e] = __ffma2_rn(d0[e], xm2[e], dw2[1][e]);
-            dw2[2][e] = __ffma2_rn(d0[e], xm1[e], dw2[2][e]); dw2[3][e] = __ffma2_rn(d0[e], x0[e], dw2[3][e]);
-            db2[e] = __fadd2_rn(db2[e], d0[e]);
+          for (int e = 0; e < CP; ++e) {
+            const float2 pre = __ffma2_rn(w2[3][e], x0[e], __ffma2_rn(w2[2][e], xm1[e], __ffma2_rn(w2[1][e], xm2[e], __ffma2_rn(w2[0][e], xm3[e], b2[e]))));
+            const float2 sg = sigmoid2<T>(pre);
+            // dout * SiLU'(pre),  SiLU'(x) = sg (1 + x (1 - sg))
+            d0[e] = __fmul2_rn(__fmul2_rn(g[e], sg), __ffma2_rn(pre, __ffma2_rn(sg, mone, one), one));
+            if (IN || t < t1) {                                // sums over this run's own steps only
+              dw2[0][e] = __ffma2_rn(d0[e], xm3[e], dw2[0][e]); dw2[1][e] = __ffma2_rn(d0[e], xm2[e], dw2[1][e]);
+              dw2[2][e] = __ffma2_rn(d0[e], xm1[e], dw2[2][e]); dw2[3][e] = __ffma2_rn(d0[e], x0[e], dw2[3][e]);
+              db2[e] = __fadd2_rn(db2[e], d0[e]);
+            }
+            xm3[e] = xm2[e]; xm2[e] = xm1[e]; xm1[e] = x0[e];
           }
-          xm3[e] = xm2[e]; xm2[e] = xm1[e]; xm1[e] = x0[e];
+        } else {
+#pragma unroll
+          for (int e = 0; e < CP; ++e) d0[e] = make_float2(0.f, 0.f);
         }
-      } else {
+        const int tp = t - 3;                                  // dx[tp] = w3 dpre[tp] + w2 dpre[tp+1] + w1 dpre[tp+2] + w0 dpre[tp+3]
+        if (IN || (tp >= ts && tp < t1)) {
+          float o[CH];
 #pragma unroll
-        for (int e = 0; e < CP; ++e) d0[e] = make_float2(0.f, 0.f);
-      }
-      const int tp = t - 3;                                  // dx[tp] = w3 dpre[tp] + w2 dpre[tp+1] + w1 dpre[tp+2] + w0 dpre[tp+3]
-      if (tp >= ts && tp < t1) {
-        float o[CH];
-#pragma unroll
-        for (int e = 0; e < CP; ++e) {
-          const float2 r = __ffma2_rn(w2[3][e], d3[e], __ffma2_rn(w2[2][e], d2[e], __ffma2_rn(w2[1][e], d1[e], __fmul2_rn(w2[0][e], d0[e]))));
-          o[2 * e] = r.x; o[2 * e + 1] = r.y;
+          for (int e = 0; e < CP; ++e) {
+            const float2 r = __ffma2_rn(w2[3][e], d3[e], __ffma2_rn(w2[2][e], d2[e], __ffma2_rn(w2[1][e], d1[e], __fmul2_rn(w2[0][e], d0[e]))));
+            o[2 * e] = r.x; o[2 * e + 1] = r.y;
+          }
+          if (IN || tp >= 0) Chunk<T>::store(dxp + u * dxs, o);
+          else if (dprev) Chunk<T>::store(dprev + ((size_t)b * 3 + (3 + tp)) * C + c0, o);
         }
-        if (tp >= 0) Chunk<T>::store(dxp + u * dxs, o);
-        else if (dprev) Chunk<T>::store(dprev + ((size_t)b * 3 + (3 + tp)) * C + c0, o);
+#pragma unroll
+        for (int e = 0; e < CP; ++e) { d3[e] = d2[e]; d2[e] = d1[e]; d1[e] = d0[e]; }
       }
-#pragma unroll
-      for (int e = 0; e < CP; ++e) { d3[e] = d2[e]; d2[e] = d1[e]; d1[e] = d0[e]; }
-    }
-#pragma unroll
-    for (int u = 0; u < U; ++u) { rx[u] = nx[u]; rg[u] = ng[u]; }
+    };
+    if (tb >= t0 + 3 && tb + U <= t1) batch(std::true_type{});
+    else batch(std::false_type{});
+    fetch(slot, xp + (size_t)G * U * xs, gp + (size_t)G * U * ds, tb + G * U);   // refill the batch just used
+    slot = slot + 1 == G ? 0 : slot + 1;
   }
+  cp_async_wait<0>();
   // the sums, channel by channel, for the hand-over below
   float dwv[CH][4], dbv[CH];
 #pragma unroll
