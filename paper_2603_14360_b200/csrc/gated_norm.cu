@@ -55,9 +55,19 @@ __device__ __forceinline__ float warp_sum(float v) {
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   return v;
 }
-// SiLU and its derivative
-__device__ __forceinline__ float silu(float x, float *dx) {
-  const float sg = __fdividef(1.f, 1.f + __expf(-x));   // ex2.approx + rcp.approx: ~1e-6 relative
+// SiLU and its derivative.  fp32 I/O: sigmoid through ex2.approx + rcp.approx (~1e-6 relative);
+// bf16 I/O: through one tanh.approx (~2^-11, below the rounding of the bf16 result) -- the kernels
+// are bound by the special-function unit as much as by HBM, and this halves its work
+template <typename T>
+__device__ __forceinline__ float silu_t(float x, float *dx) {
+  float sg;
+  if constexpr (sizeof(T) == 2) {
+    float th;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(0.5f * x));
+    sg = fmaf(0.5f, th, 0.5f);
+  } else {
+    sg = __fdividef(1.f, 1.f + __expf(-x));
+  }
   if (dx) *dx = sg * (1.f + x * (1.f - sg));
   return x * sg;
 }
@@ -84,7 +94,7 @@ __global__ void __launch_bounds__(kFwdWarps * 32) gated_norm_fwd_kernel(long tok
         for (int j = 0; j < CPL; ++j)
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
-            x[j][e] = a[j][e] * (use_silu ? silu(b[j][e], nullptr) : b[j][e]);
+            x[j][e] = a[j][e] * (use_silu ? silu_t<T>(b[j][e], nullptr) : b[j][e]);
             ss = fmaf(x[j][e], x[j][e], ss);
           }
       }
@@ -107,7 +117,7 @@ __global__ void __launch_bounds__(kFwdWarps * 32) gated_norm_fwd_kernel(long tok
         load8(gt + 8 * c, b);
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-          const float x = a[e] * (use_silu ? silu(b[e], nullptr) : b[e]);
+          const float x = a[e] * (use_silu ? silu_t<T>(b[e], nullptr) : b[e]);
           ss = fmaf(x, x, ss);
         }
       }
@@ -120,7 +130,7 @@ __global__ void __launch_bounds__(kFwdWarps * 32) gated_norm_fwd_kernel(long tok
         load8(gt + 8 * c, b);
         load8(w + 8 * c, wv);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) o[e] = wv[e] * (a[e] * (use_silu ? silu(b[e], nullptr) : b[e])) * s;
+        for (int e = 0; e < 8; ++e) o[e] = wv[e] * (a[e] * (use_silu ? silu_t<T>(b[e], nullptr) : b[e])) * s;
         store8(out + t * d + 8 * c, o);
       }
       if (rstd && lane == 0) rstd[t] = s;
@@ -155,7 +165,7 @@ __global__ void __launch_bounds__(kWarps * 32) gated_norm_bwd_kernel(long tokens
       load8(w + 8 * c, wv);
       load8(dot + 8 * c, dv);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) r = fmaf(wv[e] * dv[e], a[e] * (use_silu ? silu(b[e], nullptr) : b[e]), r);
+      for (int e = 0; e < 8; ++e) r = fmaf(wv[e] * dv[e], a[e] * (use_silu ? silu_t<T>(b[e], nullptr) : b[e]), r);
     }
     r = warp_sum(r);
     const float k3 = r * s * s * s / (float)d;
@@ -172,7 +182,7 @@ __global__ void __launch_bounds__(kWarps * 32) gated_norm_bwd_kernel(long tokens
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         float dsl = 1.f;
-        const float g = use_silu ? silu(b[e], &dsl) : b[e];
+        const float g = use_silu ? silu_t<T>(b[e], &dsl) : b[e];
         const float x = a[e] * g;
         const float dx = s * wv[e] * dv[e] - k3 * x;
         o1[e] = dx * g;
@@ -235,14 +245,47 @@ __global__ void __launch_bounds__(kRegWarps * 32) gated_norm_bwd_reg_kernel(long
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[j][e] = 0.f;
   }
-  for (long t = (long)blockIdx.x * kRegWarps + warp; t < tokens; t += (long)gridDim.x * kRegWarps) {
+  // bf16: the next token's three rows are on their way (cp.async into a two-slot ring of the warp, a
+  // lane copies and later reads its own chunks only) while this token is worked on; without that a
+  // warp's loads and its arithmetic took turns and the kernel ran at half of the HBM bandwidth
+  constexpr bool kRing = sizeof(T) == 2;
+  const long t_first = (long)blockIdx.x * kRegWarps + warp, t_step = (long)gridDim.x * kRegWarps;
+  uint4 *ring = reinterpret_cast<uint4 *>(acc_all + (size_t)kRegWarps * d) + (size_t)warp * (2 * 3 * CPL * 32);
+  auto fetch = [&](long t, int slot) {   // always one group, possibly empty
+    if (t < tokens) {
+      const T *src[3] = {y + t * d, g_in + t * d, dout + t * d};
+#pragma unroll
+      for (int x = 0; x < 3; ++x)
+#pragma unroll
+        for (int j = 0; j < CPL; ++j) {
+          const uint32_t dst = (uint32_t)__cvta_generic_to_shared(ring + ((slot * 3 + x) * CPL + j) * 32 + lane);
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src[x] + 8 * (lane + 32 * j)) : "memory");
+        }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  if constexpr (kRing) fetch(t_first, 0);
+  int slot = 0;
+  for (long t = t_first; t < tokens; t += t_step) {
     const T *yt = y + t * d, *gt = g_in + t * d, *dot = dout + t * d;
     Raw8<T> ar[CPL], br[CPL], dr[CPL];
+    if constexpr (kRing) {
+      fetch(t + t_step, slot ^ 1);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
 #pragma unroll
-    for (int j = 0; j < CPL; ++j) {
-      ar[j].load(yt + 8 * (lane + 32 * j));
-      br[j].load(gt + 8 * (lane + 32 * j));
-      dr[j].load(dot + 8 * (lane + 32 * j));
+      for (int j = 0; j < CPL; ++j) {
+        ar[j].v = ring[((slot * 3 + 0) * CPL + j) * 32 + lane];
+        br[j].v = ring[((slot * 3 + 1) * CPL + j) * 32 + lane];
+        dr[j].v = ring[((slot * 3 + 2) * CPL + j) * 32 + lane];
+      }
+      slot ^= 1;
+    } else {
+#pragma unroll
+      for (int j = 0; j < CPL; ++j) {
+        ar[j].load(yt + 8 * (lane + 32 * j));
+        br[j].load(gt + 8 * (lane + 32 * j));
+        dr[j].load(dot + 8 * (lane + 32 * j));
+      }
     }
     const float s = rstd[t];
     float r = 0.f;   // r = sum_j w_j dout_j x_j
@@ -251,7 +294,7 @@ __global__ void __launch_bounds__(kRegWarps * 32) gated_norm_bwd_reg_kernel(long
       float a[8], b[8], dv[8], wv[8];
       ar[j].get(a); br[j].get(b); dr[j].get(dv); wr[j].get(wv);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) r = fmaf(wv[e] * dv[e], a[e] * (use_silu ? silu(b[e], nullptr) : b[e]), r);
+      for (int e = 0; e < 8; ++e) r = fmaf(wv[e] * dv[e], a[e] * (use_silu ? silu_t<T>(b[e], nullptr) : b[e]), r);
     }
     r = warp_sum(r);
     const float k3 = r * s * s * s / (float)d;
@@ -262,7 +305,7 @@ __global__ void __launch_bounds__(kRegWarps * 32) gated_norm_bwd_reg_kernel(long
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         float dsl = 1.f;
-        const float g = use_silu ? silu(b[e], &dsl) : b[e];
+        const float g = use_silu ? silu_t<T>(b[e], &dsl) : b[e];
         const float x = a[e] * g;
         const float dx = s * wv[e] * dv[e] - k3 * x;
         o1[e] = dx * g;
@@ -273,6 +316,7 @@ __global__ void __launch_bounds__(kRegWarps * 32) gated_norm_bwd_reg_kernel(long
       store8(dg_in + t * d + 8 * (lane + 32 * j), o2);
     }
   }
+  if constexpr (kRing) asm volatile("cp.async.wait_group 0;" ::: "memory");
 #pragma unroll
   for (int j = 0; j < CPL; ++j) {
     float *p = acc_all + (size_t)warp * d + 8 * (lane + 32 * j);
@@ -361,14 +405,17 @@ cudaError_t launch_bwd_w(long tokens, int d, const void *y, const void *g, const
 // grows with CPL), so that the per-CTA prologue and partial of dw are paid once per SM slot
 int reg_grid(long tokens, int cpl) {
   const long need = (tokens + kRegWarps - 1) / kRegWarps;
-  const long slots = 148L * (cpl >= 4 ? 1 : (cpl == 2 ? 2 : 4));
+  const long slots = (long)sm_count() * (cpl >= 4 ? 1 : (cpl == 2 ? 2 : 4));
   return (int)(need < slots ? need : slots);
 }
 
 template <typename T, int CPL>
 cudaError_t launch_bwd_reg(long tokens, const void *y, const void *g, const void *w, const float *rstd, int silu_on,
                            const void *dout, void *dy, void *dg, float *dw_part, cudaStream_t s) {
-  const size_t smem = (size_t)kRegWarps * 256 * CPL * sizeof(float);
+  // the warps' dw sums, then (bf16) the warps' two-slot rings of three rows each
+  const size_t smem = (size_t)kRegWarps * 256 * CPL * sizeof(float) + (sizeof(T) == 2 ? (size_t)kRegWarps * 2 * 3 * 256 * CPL * sizeof(T) : 0);
+  cudaError_t e = cudaFuncSetAttribute(gated_norm_bwd_reg_kernel<T, CPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
   gated_norm_bwd_reg_kernel<T, CPL><<<reg_grid(tokens, CPL), kRegWarps * 32, smem, s>>>(
       tokens, static_cast<const T *>(y), static_cast<const T *>(g), static_cast<const T *>(w), rstd, silu_on,
       static_cast<const T *>(dout), static_cast<T *>(dy), static_cast<T *>(dg), dw_part);
