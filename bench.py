@@ -74,6 +74,15 @@ def profiled_traffic(workload: str, units: int):
     return None
 
 
+def profiled_traffic_sum(workload: str, parts, units: int):
+    """The same for a step made of several kernels: rows `workload:part`, added; None if one is
+    missing or stale."""
+    rows = [profiled_traffic(f"{workload}:{p}", units) for p in parts]
+    if any(r is None for r in rows):
+        return None
+    return {"bytes": sum(r["bytes"] for r in rows), "source": "; ".join(r["source"] for r in rows)}
+
+
 def workload_pass(name: str) -> str:
     return PASS_OF.get(name, "fwd+bwd")
 
@@ -457,6 +466,7 @@ def main_out_norm(args):
     peaks = measured_peaks()
     alg_bytes = tokens * ((6 * d + 4) + (10 * d + 4)) + 2 * d * 2 + d * 4
     achieved = alg_bytes / (ms_step * 1e-3) / 1e9
+    traffic = profiled_traffic_sum("out_norm", ("fwd", "bwd"), tokens)
     line = {
         "metric": METRIC, "value": whole_job_tokens_per_s(tokens, world, ms_step), "unit": "tokens/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -465,9 +475,10 @@ def main_out_norm(args):
                    "per_gpu_batch": B, "l2": f"{R} input sets cycled; bytes touched per step {int(alg_bytes / 1e6)} MB vs 126 MB L2"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": achieved / peaks["hbm_gbs"],
-                     # dram bytes of the two kernels of a step from the ncu capture in profiles/ (part of the
-                     # results is still in L2 when a kernel ends, so this is below the algorithmic bytes)
-                     "traffic": 205.7e6, "call": "m2rnn_gated_norm_fwd + m2rnn_gated_norm_bwd",
+                     # dram bytes of the two kernels of a step (part of the results is still in L2 when a
+                     # kernel ends, so this is below the algorithmic bytes)
+                     "traffic": traffic and traffic["bytes"], "traffic_source": traffic and traffic["source"],
+                     "call": "m2rnn_gated_norm_fwd + m2rnn_gated_norm_bwd",
                      "peak_source": f"{peaks['source']} HBM copy", "algorithmic_bytes_per_step": alg_bytes},
         "gpu_launches": args.steps * 3,
         "clocks": clocks.summary(),
@@ -582,6 +593,7 @@ def main_in_conv(args):
     peaks = measured_peaks()
     alg_bytes = tokens * C * 2 * (2 + 3)               # x, out | x, dout, dx (bf16)
     achieved = alg_bytes / (ms_step * 1e-3) / 1e9
+    traffic = profiled_traffic_sum("in_conv", ("fwd", "bwd", "reduce"), tokens)
     line = {
         "metric": METRIC, "value": whole_job_tokens_per_s(tokens, world, ms_step), "unit": "tokens/s", "n_gpus": world,
         "steps": steps, "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -589,7 +601,8 @@ def main_in_conv(args):
         "config": {"workload": "in_conv", "pass": "fwd+bwd of SiLU(conv1d) on the fused q/k/v projection", "B": B, "T": T, "C": C,
                    "per_gpu_batch": B, "l2": f"{R} input sets cycled; bytes touched per step {int(alg_bytes / 1e6)} MB vs 126 MB L2"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": achieved / peaks["hbm_gbs"], "traffic": None, "call": "m2rnn_conv_silu_fwd + m2rnn_conv_silu_bwd",
+                     "frac": achieved / peaks["hbm_gbs"], "traffic": traffic and traffic["bytes"],
+                     "traffic_source": traffic and traffic["source"], "call": "m2rnn_conv_silu_fwd + m2rnn_conv_silu_bwd",
                      "peak_source": f"{peaks['source']} HBM copy", "algorithmic_bytes_per_step": alg_bytes},
         "gpu_launches": steps * 3,
         "clocks": clocks.summary(),

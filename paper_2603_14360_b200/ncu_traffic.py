@@ -8,7 +8,8 @@ The row holds, for one launch of the workload's dominant kernel, the DRAM bytes 
 counted (dram__bytes_read.sum + dram__bytes_write.sum, averaged over the captured launches), the
 token-heads (B T N; decode: B N) the captured launch processed, and a digest of the kernel's sources at capture time.
 ``bench.py`` reports the figure as ``roofline.traffic``, scaled to a full launch by token-heads, and
-reports null once the sources have changed.
+reports null once the sources have changed.  A step made of several kernels (`in_conv`, `out_norm`)
+has one row per kernel, named `workload:part`; bench.py adds them.
 """
 from __future__ import annotations
 
@@ -23,7 +24,7 @@ CSRC = os.path.join(HERE, "csrc")
 TABLE = os.path.join(os.path.dirname(HERE), "profiles", "dram_traffic.txt")
 HEADER = ("# DRAM traffic of one launch of each workload's dominant kernel, from ncu captures.\n"
           "# Written by `python -m paper_2603_14360_b200.ncu_traffic`; read by bench.py (roofline.traffic).\n"
-          "# workload  kernel  source  dram_bytes_per_launch  token_heads_captured  source_digest  ncu_dram_read  ncu_dram_write  launches\n")
+          "# workload[:kernel of a step made of several]  kernel  source  dram_bytes_per_launch  units_captured (token-heads; tokens for in_conv, out_norm)  source_digest  ncu_dram_read  ncu_dram_write  launches\n")
 
 
 def source_digest(cu_file: str) -> str:
