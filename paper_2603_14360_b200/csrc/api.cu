@@ -50,6 +50,15 @@ BwdPlan plan_bwd(int B, int N, int K, int V, int io_dtype) {
   for (int cand = 32; cand <= cap; cand *= 2)
     if (K % cand == 0) KC = cand;
   while (KC > 16 && units * (K / KC) < kSMs && units * (K / (KC / 2)) <= kSMs) KC /= 2;
+  // V = 16, whole 64-row states, more units than two CTAs per SM hold (the paper's layer shape: 336
+  // units): 32-row CTAs at three per SM where that needs fewer waves, a 32-row CTA's wave counted
+  // as 0.9 of a 64-row one (measured: the step is latency, not rows; 3.50 -> 3.16 ms at that shape)
+  bool v16_split = false;
+  if (V == 16 && KC == 64 && units > 2L * kSMs) {
+    const long waves64 = (units + 2L * kSMs - 1) / (2L * kSMs), waves32 = (2 * units + 3L * kSMs - 1) / (3L * kSMs);
+    v16_split = 9 * waves32 < 10 * waves64;
+  }
+  if (v16_split) KC = 32;
   pl.KC = KC;
   // Checkpoint interval: as many steps as two chunk buffers fit in shared memory (even, <= 16)
   constexpr size_t kSmemLimit = 227 * 1024;
@@ -57,9 +66,9 @@ BwdPlan plan_bwd(int B, int N, int K, int V, int io_dtype) {
   while (c > 2 && bwd_bf16_smem_bytes(KC, V, c) > kSmemLimit) c -= 2;
   pl.C_max = c;
   // V = 16 with more CTAs than SMs (the paper's layer shape: 84 heads): a shorter chunk lets two
-  // CTAs share an SM, which saves a wave
+  // (32-row CTAs: three) CTAs share an SM, which saves a wave
   if (V == 16 && units * (K / KC) > kSMs)
-    while (c > 2 && bwd_bf16_smem_bytes(KC, V, c) > 110 * 1024) c -= 2;
+    while (c > 2 && bwd_bf16_smem_bytes(KC, V, c) > (v16_split ? 72 : 110) * 1024) c -= 2;
   pl.C = c;
   return pl;
 }

@@ -121,7 +121,7 @@ template <int V, int NWC>
 __host__ __device__ constexpr int bwd_threads() { return bwd_rebalance<V, NWC>() ? 512 : (2 * NWC + V / 16 + 2) * 32; }
 
 template <int V, int NWC>
-__global__ void __launch_bounds__(bwd_threads<V, NWC>(), V == 16 ? 2 : 1) bwd_bf16_kernel(ScanArgs a) {
+__global__ void __launch_bounds__(bwd_threads<V, NWC>(), V == 16 ? (NWC == 2 ? 3 : 2) : 1) bwd_bf16_kernel(ScanArgs a) {
   using G = TileGeom<V>;
   constexpr int NT = G::NT, KT = G::KT, SEG = G::SEG;
   constexpr int KC = 16 * NWC, NDW = V / 16;

@@ -135,12 +135,15 @@ def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
 
 def test_plans_for_small_states_with_many_units(lib):
     """V = 16 with more CTAs than SMs (the paper's layer shape, 84 heads x batch 4): the backward
-    plan shortens the chunk so that two CTAs share an SM; few units keep the long chunk."""
+    plan shortens the chunk so that several CTAs share an SM (and takes 32-row CTAs, three per SM,
+    where that needs fewer waves); few units keep the long chunk."""
     many = _p(B=4, N=84, Nq=1, Nk=1, K=64, V=16, T=64)
     few = _p(B=1, N=4, Nq=1, Nk=1, K=64, V=16, T=64)
     c_many, c_few = lib.m2rnn_ckpt_interval(ctypes.byref(many)), lib.m2rnn_ckpt_interval(ctypes.byref(few))
     assert 2 <= c_many < c_few <= 16 and c_many % 2 == 0
-    assert lib.m2rnn_bwd_row_slab(ctypes.byref(many)) == 64        # a CTA keeps the whole state
+    assert lib.m2rnn_bwd_row_slab(ctypes.byref(many)) == 32        # 672 CTAs at three per SM: two waves of the shorter kind
+    some = _p(B=2, N=84, Nq=1, Nk=1, K=64, V=16, T=64)              # 168 units: one wave at two per SM
+    assert lib.m2rnn_bwd_row_slab(ctypes.byref(some)) == 64        # a CTA keeps the whole state
     assert lib.m2rnn_bwd_row_slab(ctypes.byref(few)) == 16         # few units: spread the rows over the SMs
     # a caller may still ask for a longer chunk, up to what one CTA's shared memory holds
     assert lib.m2rnn_ckpt_interval(ctypes.byref(_p(B=4, N=84, Nq=1, Nk=1, K=64, V=16, T=64, ckpt_interval=12))) == 12

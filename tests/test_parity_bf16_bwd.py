@@ -25,6 +25,7 @@ SHAPES = [
     (40, 7, 4, 32, 128, 0, 0),    # ... and the 32-row CTAs of V = 128 (W in shared memory)
     (40, 7, 4, 32, 64, 0, 0),     # two slabs per CTA
     (40, 15, 4, 64, 16, 1, 1),    # V = 16 with more units than SMs: shorter chunks, two CTAs per SM
+    (4, 13, 84, 64, 16, 1, 1),    # the paper's layer shape (336 units): 32-row CTAs, three per SM
 ]
 
 
