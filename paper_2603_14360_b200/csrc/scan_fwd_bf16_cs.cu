@@ -37,6 +37,14 @@ struct CsSmem {
   }
 };
 
+// transpose of an 8 x 8 tile of 16-bit elements held by a warp (lane holds row lane/4, elements
+// 2 (lane%4), +1 before and after): turns half of an A fragment into half of a B fragment
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+
 // memory column (inside a part of VP columns) of MMA column m of that part
 template <int VP>
 __host__ __device__ constexpr int part_col(int m) { return (VP / 4) * ((m & 7) >> 1) + 2 * (m >> 3) + (m & 1); }
@@ -301,9 +309,18 @@ __global__ void __launch_bounds__((SP * NW + cs_service_warps(SP * NW)) * 32, OC
   auto step = [&](float (&Pc)[NTH][4], float (&Pn)[NTH][4], float f, uint32_t qrow, uint32_t ydst,
                   uint32_t krow_n, uint32_t vrow_n, int par) {
     seed(Pn, krow_n, vrow_n);
-    const float q0 = lds32(qrow + 4u * r0), q1 = lds32(qrow + 4u * (r0 + 8));
-    float part[SEGH];
-    const float2 f2 = make_float2(f, f), m1 = make_float2(-1.f, -1.f), q02 = make_float2(q0, q0), q12 = make_float2(q1, q1);
+    // Readout (Eq. 3) on the tensor cores: y^T = q^T H over the slab's 16 rows is one more product
+    // per accumulator tile, with q as row 0 of an otherwise empty A operand and the freshly packed
+    // bf16 fragments of H_t, transposed in registers, as B.  It replaces the products and the
+    // shuffle tree over the rows (39 instructions per warp and step by 8 movmatrix + 4 MMAs + a
+    // dozen others); the chain is bound by its instruction count, the tensor pipe has room.
+    uint32_t Aq[4] = {0u, 0u, 0u, 0u};
+    {
+      const float2 qa = lds64(qrow + 4u * (16 * slab + 2 * c)), qb = lds64(qrow + 4u * (16 * slab + 2 * c + 8));
+      if (g == 0) { Aq[0] = pack_bf16(qa.x, qa.y); Aq[2] = pack_bf16(qb.x, qb.y); }
+    }
+    float Y[NTH][4];
+    const float2 f2 = make_float2(f, f), m1 = make_float2(-1.f, -1.f);
     // Unit u = (accumulator tile u/2, row half u%2): Eq. 1 and 2 for two elements, and after the
     // tile's second unit its share of Eq. 3.
     auto unit = [&](int u) {
@@ -312,10 +329,6 @@ __global__ void __launch_bounds__((SP * NW + cs_service_warps(SP * NW)) * 32, OC
       const float2 d = __ffma2_rn(z, m1, make_float2(H[nt][2 * h], H[nt][2 * h + 1]));            // H - Z
       const float2 hh = __ffma2_rn(f2, d, z);                                                     // Eq. 2
       H[nt][2 * h] = hh.x; H[nt][2 * h + 1] = hh.y;
-      if (h == 1) {
-        const float2 pr = __ffma2_rn(q12, hh, __fmul2_rn(q02, make_float2(H[nt][0], H[nt][1])));  // Eq. 3, this thread's two rows
-        part[2 * nt] = pr.x; part[2 * nt + 1] = pr.y;
-      }
     };
     uint32_t Aown[KTH][4], Apar[KTP][4];
     auto pack_store = [&](int kth) {
@@ -325,6 +338,10 @@ __global__ void __launch_bounds__((SP * NW + cs_service_warps(SP * NW)) * 32, OC
       Aown[kth][3] = pack_bf16(H[2 * kth + 1][2], H[2 * kth + 1][3]);
       asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(xslot(par, hf) + 512u * kth), "r"(Aown[kth][0]), "r"(Aown[kth][1]),
                    "r"(Aown[kth][2]), "r"(Aown[kth][3]) : "memory");
+    };
+    auto readout = [&](int kth) {   // accumulator tiles 2 kth and 2 kth + 1
+      mma_bf16_16816_zero(Y[2 * kth], Aq, movmatrix_trans(Aown[kth][0]), movmatrix_trans(Aown[kth][1]));
+      mma_bf16_16816_zero(Y[2 * kth + 1], Aq, movmatrix_trans(Aown[kth][2]), movmatrix_trans(Aown[kth][3]));
     };
     // The MMAs of own k-tile kth are issued between the units of the next k-tile's two
     // accumulator tiles, so that the tensor pipe and the tanh unit work at the same time
@@ -347,13 +364,13 @@ __global__ void __launch_bounds__((SP * NW + cs_service_warps(SP * NW)) * 32, OC
     pair_sync();
     xload(par, Apar);
     mma_partner(Pn, Apar);
-    reduce_over_rows<SEGH>(part, lane);
-    // after the reduction lane (g,c) holds CNT sums starting at segment index (g >> (3-R)) * CNT
-    constexpr int R = SEGH >= 8 ? 3 : (SEGH >= 4 ? 2 : 1), CNT = SEGH >> R;
-    if (((g) & ((1 << (3 - R)) - 1)) == 0) {
-      const uint32_t dst = ydst + 4u * (col0 + (g >> (3 - R)) * CNT);
-      if constexpr (CNT == 2) sts64(dst, make_float2(part[0], part[1]));
-      else sts32(dst, part[0]);
+#pragma unroll
+    for (int kth = 0; kth < KTH; ++kth) readout(kth);
+    // row 0 of the products: lanes 0-3 hold the slab's sums over its 16 rows, two adjacent memory
+    // columns per accumulator tile
+    if (g == 0) {
+#pragma unroll
+      for (int nt = 0; nt < NTH; ++nt) sts64(ydst + 4u * (col0 + 2 * nt), make_float2(Y[nt][0], Y[nt][1]));
     }
   };
 
