@@ -272,6 +272,12 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
     }
   };
 
+  // transpose of an 8 x 8 tile of 16-bit elements held by a warp: half of an A fragment -> half of a B fragment
+  auto movmatrix_trans = [](uint32_t x) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(x));
+    return d;
+  };
   // One step, software-pipelined by hand: while the MUFU works through tanh of step t, column
   // tile pair by column tile pair, the tensor pipe already runs the k tiles of step t+1 that
   // depend only on the pairs finished so far.  The body is branch-free (one basic block) so the
@@ -284,6 +290,17 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
     seed(Pn, krow_n, vrow_n);
     const float2 qq = lds64(qrow + 4 * row0);
     float part[SEG];
+    // packed path: the readout (Eq. 3) on the tensor cores, y^T = q^T H over the slab's 16 rows as
+    // one more product per accumulator tile: q is row 0 of an otherwise empty A operand (MMA row m
+    // <-> memory row 2m, m + 8 <-> 2m + 1), the packed bf16 fragments of H_t, transposed in
+    // registers, are B.  It replaces the products and the shuffle tree over the rows, which were
+    // half of a V = 16 step's instructions.
+    uint32_t Aq[4] = {0u, 0u, 0u, 0u};
+    float Y[NT][4];
+    if constexpr (kPacked) {
+      const float4 q4 = lds128(qrow + 4 * (16 * warp + 4 * c));
+      if (g == 0) { Aq[0] = pack_bf16(q4.x, q4.z); Aq[2] = pack_bf16(q4.y, q4.w); }
+    }
 #pragma unroll
     for (int kt = 0; kt < KT; ++kt) {
 #pragma unroll
@@ -299,8 +316,6 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
             hh[h] = __ffma2_rn(make_float2(f, f), dd, z);                                                          // Eq. 2
             H[nt][2 * h] = hh[h].x; H[nt][2 * h + 1] = hh[h].y;
           }
-          const float2 pr = __ffma2_rn(make_float2(qq.y, qq.y), hh[1], __fmul2_rn(make_float2(qq.x, qq.x), hh[0]));   // Eq. 3
-          part[2 * nt] = pr.x; part[2 * nt + 1] = pr.y;
         } else {
 #pragma unroll
           for (int r = 0; r < 4; ++r) {
@@ -319,14 +334,27 @@ __global__ void __launch_bounds__((MAXW + 1) * 32, OCC) fwd_bf16_kernel(ScanArgs
       Ak[2] = pack_bf16(H[2 * kt + 1][0], H[2 * kt + 1][1]);
       Ak[3] = pack_bf16(H[2 * kt + 1][2], H[2 * kt + 1][3]);
       mma_ktile(Pn, Ak, kt);
+      if constexpr (kPacked) {   // Eq. 3 for accumulator tiles 2 kt and 2 kt + 1
+        mma_bf16_16816_zero(Y[2 * kt], Aq, movmatrix_trans(Ak[0]), movmatrix_trans(Ak[1]));
+        mma_bf16_16816_zero(Y[2 * kt + 1], Aq, movmatrix_trans(Ak[2]), movmatrix_trans(Ak[3]));
+      }
     }
-    reduce_over_rows<SEG>(part, lane);
-    using RO = RowReduceOut<V>;
-    if (RO::owner(lane)) {
-      const uint32_t dst = ydst + 4 * RO::first_col(lane);
-      if constexpr (RO::CNT == 4) sts128(dst, make_float4(part[0], part[1], part[2], part[3]));
-      else if constexpr (RO::CNT == 2) sts64(dst, make_float2(part[0], part[1]));
-      else sts32(dst, part[0]);
+    if constexpr (kPacked) {
+      // row 0 of the products: lanes 0-3 hold the sums over the slab's rows for their SEG columns
+      if (g == 0) {
+#pragma unroll
+        for (int x = 0; x < SEG / 4; ++x)
+          sts128(ydst + 4 * (SEG * c + 4 * x), make_float4(Y[2 * x][0], Y[2 * x][1], Y[2 * x + 1][0], Y[2 * x + 1][1]));
+      }
+    } else {
+      reduce_over_rows<SEG>(part, lane);
+      using RO = RowReduceOut<V>;
+      if (RO::owner(lane)) {
+        const uint32_t dst = ydst + 4 * RO::first_col(lane);
+        if constexpr (RO::CNT == 4) sts128(dst, make_float4(part[0], part[1], part[2], part[3]));
+        else if constexpr (RO::CNT == 2) sts64(dst, make_float2(part[0], part[1]));
+        else sts32(dst, part[0]);
+      }
     }
   };
 
