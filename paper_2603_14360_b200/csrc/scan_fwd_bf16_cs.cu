@@ -359,13 +359,12 @@ __global__ void __launch_bounds__((SP * NW + cs_service_warps(SP * NW)) * 32, OC
           for (int u = 4 * nt / NTH; u < 4 * (nt + 1) / NTH; ++u) unit(4 * (kth + 1) + u);
         }
       }
+      readout(kth);
       if (kth + 1 < KTH) pack_store(kth + 1);
     }
     pair_sync();
     xload(par, Apar);
     mma_partner(Pn, Apar);
-#pragma unroll
-    for (int kth = 0; kth < KTH; ++kth) readout(kth);
     // row 0 of the products: lanes 0-3 hold the slab's sums over its 16 rows, two adjacent memory
     // columns per accumulator tile
     if (g == 0) {
