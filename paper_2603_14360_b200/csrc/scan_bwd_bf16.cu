@@ -63,6 +63,10 @@ __device__ __forceinline__ void load_wt_fragment(const __nv_bfloat16 *__restrict
   b1 = (uint32_t)w[l * V + j2] | ((uint32_t)w[l * V + j3] << 16);
 }
 
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+
 // Register re-balancing between warpgroups (4 aligned warps): the kernel is compiled for an even
 // split (128 per thread here), then the chain warps take registers that the dW and service warps
 // give up.  An increase waits until the CTA's own pool holds enough released registers, so the
@@ -98,8 +102,8 @@ __host__ __device__ inline BwdLayout bwd_layout(int KC, int C, bool w_in_smem) {
   off += 2u * C * L.state_stride;
   L.dx = off;                                  // [2] dX tiles (bf16)
   off += 2u * KC * V * 2;
-  L.hfin = off;                                // H after the last step, as a tile (dq of step T-1)
-  off += (uint32_t)KC * V * 2;
+  L.hfin = off;                                // [2] H_t of a chunk's last step, as a tile (dq of that step): chunk j reads tile j & 1
+  off += 2u * KC * V * 2;
   L.ring = off;
   const uint32_t Cp = (uint32_t)((C + 3) & ~3);  // keeps every array of a slot 16-byte aligned
   L.oQ = 0; L.oK = L.oQ + C * KC; L.oV = L.oK + C * KC; L.oDY = L.oV + C * V; L.oF = L.oDY + C * V;
@@ -135,6 +139,11 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), V == 16 ? (NWC == 2 ? 3
   // packed fp32x2 element-wise arithmetic where it measured faster (elsewhere its register pairs spill)
   constexpr bool kPacked = V <= 32 || (V == 64 && NWC == 4);
   constexpr int NSET = 1;   // accumulator sets of the state x W product, as in the forward kernel
+  // Who computes dq = H_t dy and dk = dX v (small MMAs): the dW warps from the tiles, where they have
+  // the time (more dW warps than row slabs: sweep64 backward 7.13 -> 5.76 ms, sweep32 2.65 -> 2.43),
+  // else the reverse warps from the fragments they hold (with as many slabs as dW warps the dW
+  // warps would set the pace: bptt_bf16 8.37 -> 9.00 ms, the paper's layer shape 3.13 -> 3.41)
+  constexpr bool kDqDw = NDW >= 2 * NWC || (NDW == 1 && NWC == 1), kDkDw = kDqDw;
   extern __shared__ __align__(128) unsigned char smem[];
 
   const int K = a.K, N = a.N, C = a.C;
@@ -450,7 +459,7 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), V == 16 ? (NWC == 2 ? 3
       const int len = chunk_len(j);
       if (!mbar_wait(&in_full[j & (kRing - 1)], (j / kRing) & 1)) { report_timeout(a.dev_status); return; }
       if (!mbar_wait(&st_ready[j & 1], (j >> 1) & 1)) { report_timeout(a.dev_status); return; }
-      if (j == 0) tile_load_at(sm0 + L.hfin, w, toff, hn);
+      if constexpr (!kDqDw) { if (j == 0) tile_load_at(sm0 + L.hfin, w, toff, hn); }
       const uint32_t sl = slot_sa(j);
       // addresses of the step's operands: walked backwards (one add per step) or worked out from s
       struct Ptrs { uint32_t st, f, q, dyb, vb, dy, dfp, dq, dk; };
@@ -480,10 +489,14 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), V == 16 ? (NWC == 2 ? 3
         const float omf = 1.f - f;
         // dq = H_t dy on the tensor cores (Algorithm 2, query-gradient line)
         float dqd[2][4], dkd[2][4];
-        {
+        if constexpr (!kDqDw) {
           uint32_t dyp[NT];
           load_pairs(pDYB, dyp);
           matvec(hn, dyp, dqd);
+        } else {
+          // H_{t-1} of a chunk's first step is H_t of the last step of the chunk swept next; its
+          // state buffer may be overwritten by then, so it is kept as a tile for the dW warps
+          if (s == 0) tile_store_at(sm0 + L.hfin + (uint32_t)((j + 1) & 1) * (KC * V * 2), w, toff, hp);
         }
         float df = 0.f;
         float2 df2 = make_float2(0.f, 0.f);   // packed path: even and odd elements summed apart
@@ -563,7 +576,7 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), V == 16 ? (NWC == 2 ? 3
           }
         }
         // dk = dX v on the tensor cores (Algorithm 2, key-gradient line)
-        {
+        if constexpr (!kDkDw) {
           uint32_t vp[NT];
           load_pairs(pVB, vp);
           matvec(xp, vp, dkd);
@@ -576,11 +589,13 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), V == 16 ? (NWC == 2 ? 3
         }
         sts32(pDFP, df);   // summed by the service warp
         if (c == 0) {
-          sts32(pDQ, dqd[0][0] + dqd[1][0]); sts32(pDQ + 32u, dqd[0][2] + dqd[1][2]);
-          sts32(pDK, dkd[0][0] + dkd[1][0]); sts32(pDK + 32u, dkd[0][2] + dkd[1][2]);
+          if constexpr (!kDqDw) { sts32(pDQ, dqd[0][0] + dqd[1][0]); sts32(pDQ + 32u, dqd[0][2] + dqd[1][2]); }
+          if constexpr (!kDkDw) { sts32(pDK, dkd[0][0] + dkd[1][0]); sts32(pDK + 32u, dkd[0][2] + dkd[1][2]); }
         }
+        if constexpr (!kDqDw) {
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) { hn[nt][0] = hp[nt][0]; hn[nt][1] = hp[nt][1]; }
+          for (int nt = 0; nt < NT; ++nt) { hn[nt][0] = hp[nt][0]; hn[nt][1] = hp[nt][1]; }
+        }
         if constexpr (kWalk) {
           run.st -= L.state_stride; run.f -= 4u; run.q -= 4u * KC; run.dyb -= 2u * V; run.vb -= 2u * V;
           run.dy -= 4u * V; run.dfp -= 4u * NWC * 32; run.dq -= 4u * KC; run.dk -= 4u * KC;
@@ -676,6 +691,43 @@ __global__ void __launch_bounds__(bwd_threads<V, NWC>(), V == 16 ? (NWC == 2 ? 3
           const uint32_t dst = slot_sa(j) + 4u * (L.oDV + s * V + 16 * d + 2 * c);
           sts64(dst, make_float2(dvacc[0][0], dvacc[0][1]));
           sts64(dst + 32u, make_float2(dvacc[1][0], dvacc[1][1]));
+        }
+        // dq = H_t dy and dk = dX v (Algorithm 2, query- and key-gradient lines) for the 16-row
+        // slabs this warp takes in turn: A fragments by ldmatrix from the H_t tile (the H_{t-1} tile
+        // of the step after this one; for a chunk's last step the tile the reverse warps kept) and
+        // from the dX tile, B = the vector as bf16 pairs in every column, so that every column of
+        // the result holds the product
+        if constexpr (kDqDw || kDkDw) {
+          const uint32_t hnext = s + 1 < len ? state_sa(j, s + 1) : sm0 + L.hfin + (uint32_t)(j & 1) * (KC * V * 2);
+          const uint32_t dyb = slot_sa(j) + 4u * (L.oDYB + s * (V / 2)), vb = slot_sa(j) + 4u * (L.oVB + s * (V / 2));
+          auto pair_of = [&](uint32_t vec_sa, int kt, uint32_t &b0, uint32_t &b1) {
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(b0) : "r"(vec_sa + 4u * (8 * kt + c)));
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(b1) : "r"(vec_sa + 4u * (8 * kt + 4 + c)));
+          };
+          for (int mt = d; mt < NWC; mt += NDW) {
+            float dq[4] = {0.f, 0.f, 0.f, 0.f}, dk[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int kt = 0; kt < KT; ++kt) {
+              // matrices (rows 0-7, chunk 2kt), (rows 8-15, 2kt), (rows 0-7, 2kt+1), (rows 8-15, 2kt+1)
+              const uint32_t off = tile_off<V>(16 * mt + mr + 8 * (mi & 1), 2 * kt + (mi >> 1));
+              uint32_t A[4], b0, b1;
+              if constexpr (kDqDw) {
+                ldmatrix_x4(hnext + off, A);
+                pair_of(dyb, kt, b0, b1);
+                mma_bf16_16816(dq, A, b0, b1);
+              }
+              if constexpr (kDkDw) {
+                ldmatrix_x4(xt + off, A);
+                pair_of(vb, kt, b0, b1);
+                mma_bf16_16816(dk, A, b0, b1);
+              }
+            }
+            if (c == 0) {
+              const uint32_t o = slot_sa(j) + 4u * (s * KC + 16 * mt + g);
+              if constexpr (kDqDw) { sts32(o + 4u * L.oDQ, dq[0]); sts32(o + 4u * (L.oDQ + 8), dq[2]); }
+              if constexpr (kDkDw) { sts32(o + 4u * L.oDK, dk[0]); sts32(o + 4u * (L.oDK + 8), dk[2]); }
+            }
+          }
         }
         __syncwarp();
         if (lane == 0) asm volatile("red.release.cta.shared.add.u32 [%0], 1;" ::"r"(smem_u32(dx_read)) : "memory");
